@@ -1,0 +1,243 @@
+/*
+ * argus.h — C-ABI of the region-trace synthesis hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library turns raw per-(CTA, warp) begin/end region-marker event buffers into
+ * nested, attributed region intervals, attribution-ambiguity records, per-(region,
+ * execution-scope) statistics and per-SM producer/consumer overlap time.
+ *
+ * Paper passages the operations follow (arxiv 2609.12299, "Argus"):
+ *   - Section 3.2 "Region Semantics and Identity": a region is a code span delimited by
+ *     begin(id)/end(id) markers with stable ids; the transitions update a nested region
+ *     context stack per warp and the innermost active region owns what happens;
+ *     temporal traces recover region-labelled intervals.
+ *   - Section 3.2 "Region and scope": a scope selects dynamic executions (warp role,
+ *     iteration window, SM subset); here scopes are the aggregation keys warp/CTA/SM/kernel.
+ *   - Section 3.1 / 3.3: the `duration` signal is the elapsed time of a region.
+ *   - Section 3.5 "Synthesizing Qualified Region Reports": evidence is joined by region
+ *     identity and dynamic execution context, and attribution ambiguity is reported, not
+ *     hidden.
+ *
+ * Conventions
+ *   - All structs are plain little-endian PODs, naturally aligned, with no padding.
+ *   - Every pointer named "device" below is a CUDA device pointer on the current device;
+ *     `cuda_stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *   - The caller owns every buffer. The three operations allocate nothing, keep no state
+ *     between calls, enqueue their kernels on `cuda_stream` and return without
+ *     synchronising; results are valid once the stream reaches that point, so
+ *     pair -> aggregate -> overlap on one stream needs no host synchronisation.
+ *   - Return value: host-detectable errors (ARGUS_OK, ARGUS_ERR_INVALID_ARG,
+ *     ARGUS_ERR_WORKSPACE, ARGUS_ERR_CUDA). Conditions found on the device are written to
+ *     `status->code` (first error wins); on a device error the output arrays are
+ *     unspecified, but the GPU is never trapped or hung.
+ */
+#ifndef ARGUS_H_
+#define ARGUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ARGUS_NONE        0xFFFFFFFFu /* parent_region of a top-level interval */
+#define ARGUS_MAX_DEPTH   64          /* max simultaneously open frames per stream */
+#define ARGUS_MAX_REGIONS 65536       /* upper bound of num_regions */
+#define ARGUS_HIST_BINS   64
+
+/* return / status codes */
+enum {
+  ARGUS_OK = 0,
+  ARGUS_ERR_INVALID_ARG = 1, /* host: null pointer, bad sizes, misaligned buffer          */
+  ARGUS_ERR_WORKSPACE = 2,   /* host: workspace_bytes smaller than the *_workspace_bytes query */
+  ARGUS_ERR_CUDA = 3,        /* host: a CUDA runtime call failed                          */
+  ARGUS_ERR_CAPACITY = 4,    /* device: interval/ambiguity capacity too small; see *_required */
+  ARGUS_ERR_DEPTH = 5,       /* device: a stream would hold more than ARGUS_MAX_DEPTH open frames */
+  ARGUS_ERR_BAD_REGION = 6,  /* device: tag>>1 >= num_regions                             */
+  ARGUS_ERR_BAD_OFFSETS = 7, /* device: stream_offsets / interval_offsets not non-decreasing */
+  ARGUS_ERR_TIMEOUT = 8,     /* device: a bounded wait expired (reserved)                 */
+  ARGUS_ERR_RANGE = 9        /* device: a timestamp is outside the range overlap supports  */
+};
+
+/* One marker event, 16 bytes. tag = region_id << 1 | is_end. ts = globaltimer ns.
+ * ctx = dynamic execution context (iteration / tile / token coordinate). */
+typedef struct {
+  uint64_t ts;
+  uint32_t tag;
+  uint32_t ctx;
+} argus_event_t;
+
+/* interval flags */
+#define ARGUS_FLAG_CTX_MISMATCH  1u /* end.ctx != begin.ctx (interval keeps begin's ctx)     */
+#define ARGUS_FLAG_TIME_REVERSED 2u /* t_end < t_begin; inclusive saturated to 0             */
+#define ARGUS_FLAG_CHILD_CLAMPED 4u /* children sum > inclusive; exclusive saturated to 0    */
+
+/* One matched region occurrence, 48 bytes. depth = stack height before the push
+ * (top level = 0); parent_region = region on top of the stack at the push or ARGUS_NONE;
+ * begin_idx = index of the begin marker within its stream. */
+typedef struct {
+  uint64_t t_begin;
+  uint64_t inclusive;
+  uint64_t exclusive;
+  uint32_t region;
+  uint32_t ctx;
+  uint32_t stream;
+  uint32_t parent_region;
+  uint32_t begin_idx;
+  uint16_t depth;
+  uint16_t flags;
+} argus_interval_t;
+
+/* ambiguity kinds */
+#define ARGUS_AMBIG_UNMATCHED_END   1u /* end with no open frame of its region; depth = stack height */
+#define ARGUS_AMBIG_BEGIN_MISNESTED 2u /* begin force-closed by an enclosing region's end            */
+#define ARGUS_AMBIG_BEGIN_EOS       3u /* begin still open at the end of its stream                  */
+
+/* One marker that could not be attributed to an interval, 32 bytes. */
+typedef struct {
+  uint64_t ts;
+  uint32_t tag;
+  uint32_t ctx;
+  uint32_t stream;
+  uint32_t event_idx; /* index of the marker within its stream */
+  uint32_t kind;
+  uint32_t depth;
+} argus_ambiguity_t;
+
+/* Statistics of one (scope key, region) cell, 576 bytes. min/max/hist use the inclusive
+ * duration; hist bin = d ? 63 - clz64(d) : 0. An empty cell is all zero except
+ * min_incl = UINT64_MAX. */
+typedef struct {
+  uint64_t count;
+  uint64_t sum_incl;
+  uint64_t min_incl;
+  uint64_t max_incl;
+  uint64_t sum_excl;
+  uint64_t n_unmatched_begin; /* ambiguity kinds 2 and 3 at this (key, region) */
+  uint64_t n_unmatched_end;   /* ambiguity kind 1 */
+  uint64_t n_flagged;         /* intervals with flags != 0 */
+  uint64_t hist[ARGUS_HIST_BINS];
+} argus_agg_t;
+
+/* Overlap of one (producer, consumer) pair on one SM, 32 bytes; all in ns. */
+typedef struct {
+  uint64_t overlap_ns;  /* |U_P  ∩ U_C| */
+  uint64_t producer_ns; /* |U_P|       */
+  uint64_t consumer_ns; /* |U_C|       */
+  uint64_t either_ns;   /* |U_P ∪ U_C| */
+} argus_overlap_t;
+
+/* Device-resident status block, 64 bytes. */
+typedef struct {
+  uint32_t code;       /* ARGUS_OK or the first device error                     */
+  uint32_t bad_stream; /* stream where the first error was seen                  */
+  uint64_t bad_event;  /* event index within that stream (or offending count)    */
+  uint64_t intervals_required;
+  uint64_t ambig_required;
+  uint64_t n_ctx_mismatch;
+  uint64_t n_time_reversed;
+  uint64_t n_child_clamped;
+  uint64_t reserved;
+} argus_status_t;
+
+/* ---------------------------------------------------------------------------------------
+ * argus_pair_intervals — Section 3.2 (per-warp nested region stack; innermost region owns).
+ *
+ * For every stream s (events[stream_offsets[s] .. stream_offsets[s+1]), in buffer order,
+ * never re-sorted by time):
+ *   begin(r): push a frame (depth = current height, parent = region on top or ARGUS_NONE);
+ *             more than ARGUS_MAX_DEPTH open frames -> ARGUS_ERR_DEPTH.
+ *   end(r):   search the stack from the top for the innermost frame of region r.
+ *             none  -> ambiguity record UNMATCHED_END (depth = height), stack unchanged.
+ *             found -> frames above it are force-closed as BEGIN_MISNESTED (their
+ *                      accumulated child time moves to the new top); the found frame
+ *                      becomes an interval: inclusive = t_end - t_begin (0 + TIME_REVERSED
+ *                      if negative), exclusive = inclusive - sum of inclusive of its
+ *                      children among matched intervals (0 + CHILD_CLAMPED if negative),
+ *                      ctx from the begin (CTX_MISMATCH if the end's differs).
+ *   end of stream: every open frame -> BEGIN_EOS.
+ * Outputs (device): intervals ordered by (stream, position of the end marker) with
+ * interval_offsets[S+1]; ambiguity records ordered by (stream, event_idx) with
+ * ambig_offsets[S+1]. interval_capacity >= floor(N/2) and ambig_capacity >= N always
+ * suffice; otherwise ARGUS_ERR_CAPACITY reports the required counts in `status`.
+ * Requirements: events 16-byte aligned; num_regions in [1, ARGUS_MAX_REGIONS];
+ * every stream shorter than 2^32 events; workspace 256-byte aligned and at least
+ * argus_pair_workspace_bytes(N, S, ambig_capacity) bytes. `status` (device, 64 B) is
+ * overwritten. Empty streams and num_streams == 0 are legal.
+ * ------------------------------------------------------------------------------------- */
+size_t argus_pair_workspace_bytes(uint64_t num_events, uint32_t num_streams,
+                                  uint64_t ambig_capacity);
+
+int argus_pair_intervals(const argus_event_t* events /*device*/,
+                         const uint64_t* stream_offsets /*device [S+1]*/,
+                         uint32_t num_streams, uint32_t num_regions,
+                         argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
+                         uint64_t* interval_offsets /*device [S+1] out*/,
+                         argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
+                         uint64_t* ambig_offsets /*device [S+1] out*/,
+                         argus_status_t* status /*device*/, void* workspace /*device*/,
+                         size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
+ * argus_aggregate — Section 3.2 "Region and scope" + the `duration` signal (Section 3.1).
+ *
+ * Reduces intervals (and, if given, ambiguity records) into dense tables of argus_agg_t,
+ * one per scope level: warp_tab[S][R] (key = stream), cta_tab[C][R] (key = stream /
+ * warps_per_cta, C = S / warps_per_cta), sm_tab[M][R] (key = cta_sm[cta]) and
+ * kernel_tab[R]. Any table pointer may be NULL (that level is skipped). Every cell of a
+ * requested table is written (empty cells: zero, min_incl = UINT64_MAX).
+ * num_streams must be a multiple of warps_per_cta; cta_sm values must be < num_sms.
+ * Event-derived ambiguity counters are added at the marker's (region, key).
+ * ------------------------------------------------------------------------------------- */
+size_t argus_aggregate_workspace_bytes(uint64_t num_intervals, uint32_t num_streams,
+                                       uint32_t num_regions);
+
+int argus_aggregate(const argus_interval_t* intervals /*device*/,
+                    const uint64_t* interval_offsets /*device [S+1]*/,
+                    const argus_ambiguity_t* ambig /*device, nullable*/,
+                    const uint64_t* ambig_offsets /*device [S+1], nullable*/,
+                    uint32_t num_streams, uint32_t warps_per_cta,
+                    const uint32_t* cta_sm /*device [C]*/, uint32_t num_sms,
+                    uint32_t num_regions, argus_agg_t* warp_tab /*device [S][R], nullable*/,
+                    argus_agg_t* cta_tab /*device [C][R], nullable*/,
+                    argus_agg_t* sm_tab /*device [M][R], nullable*/,
+                    argus_agg_t* kernel_tab /*device [R], nullable*/,
+                    argus_status_t* status /*device*/, void* workspace /*device*/,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
+ * argus_overlap — producer/consumer overlap per SM (the overlap diagnosis the paper
+ * motivates in Sections 1 and 4; scope = SM subset, Section 3.2).
+ *
+ * For every pair k = (producer region P, consumer region Cn) and SM m: take the half-open
+ * spans [t_begin, t_begin + inclusive) of all intervals of region P (resp. Cn) in streams
+ * whose CTA maps to m (all depths and contexts, flagged ones included, empty spans
+ * dropped); U_P, U_C = their unions. out[k][m] = { |U_P ∩ U_C|, |U_P|, |U_C|, |U_P ∪ U_C| }.
+ * Timestamps must satisfy t_begin + inclusive < 2^62, else ARGUS_ERR_RANGE.
+ * ------------------------------------------------------------------------------------- */
+size_t argus_overlap_workspace_bytes(uint64_t num_intervals, uint32_t num_streams,
+                                     uint32_t num_pairs, uint32_t num_sms);
+
+int argus_overlap(const argus_interval_t* intervals /*device*/,
+                  const uint64_t* interval_offsets /*device [S+1]*/, uint32_t num_streams,
+                  uint32_t warps_per_cta, const uint32_t* cta_sm /*device [C]*/,
+                  uint32_t num_sms, const uint32_t* pairs /*device [K][2]*/,
+                  uint32_t num_pairs, argus_overlap_t* out /*device [K][M]*/,
+                  argus_status_t* status /*device*/, void* workspace /*device*/,
+                  size_t workspace_bytes, void* cuda_stream);
+
+/* Copies the device status block to host memory and synchronises `cuda_stream`.
+ * Returns ARGUS_OK or ARGUS_ERR_CUDA; the device-side code is in host_copy->code. */
+int argus_status_fetch(const argus_status_t* dev_status, argus_status_t* host_copy,
+                       void* cuda_stream);
+
+/* Static, NUL-terminated description of a code; never NULL. */
+const char* argus_strerror(int code);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int argus_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARGUS_H_ */

@@ -1,0 +1,118 @@
+"""ctypes loader of the CPU oracle (test infrastructure only).
+
+Only the tests, the smoke check and the CPU-baseline leg of the benchmark may import this
+package; the product never does. Record layouts are retyped here, independently of the CUDA
+binding. See oracle.h for what each function computes and which paper passages it follows.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+
+EVENT = np.dtype([("ts", "<u8"), ("tag", "<u4"), ("ctx", "<u4")])
+INTERVAL = np.dtype([("t_begin", "<u8"), ("inclusive", "<u8"), ("exclusive", "<u8"), ("region", "<u4"),
+                     ("ctx", "<u4"), ("stream", "<u4"), ("parent_region", "<u4"), ("begin_idx", "<u4"),
+                     ("depth", "<u2"), ("flags", "<u2")])
+AMBIG = np.dtype([("ts", "<u8"), ("tag", "<u4"), ("ctx", "<u4"), ("stream", "<u4"), ("event_idx", "<u4"),
+                  ("kind", "<u4"), ("depth", "<u4")])
+AGG = np.dtype([("count", "<u8"), ("sum_incl", "<u8"), ("min_incl", "<u8"), ("max_incl", "<u8"),
+                ("sum_excl", "<u8"), ("n_unmatched_begin", "<u8"), ("n_unmatched_end", "<u8"),
+                ("n_flagged", "<u8"), ("hist", "<u8", (64,))])
+OVERLAP = np.dtype([("overlap_ns", "<u8"), ("producer_ns", "<u8"), ("consumer_ns", "<u8"), ("either_ns", "<u8")])
+STATUS = np.dtype([("code", "<u4"), ("bad_stream", "<u4"), ("bad_event", "<u8"), ("intervals_required", "<u8"),
+                   ("ambig_required", "<u8"), ("n_ctx_mismatch", "<u8"), ("n_time_reversed", "<u8"),
+                   ("n_child_clamped", "<u8"), ("reserved", "<u8")])
+assert (EVENT.itemsize, INTERVAL.itemsize, AMBIG.itemsize, AGG.itemsize, OVERLAP.itemsize, STATUS.itemsize) == \
+    (16, 48, 32, 576, 32, 64)
+
+NONE = 0xFFFFFFFF
+
+
+def build(force: bool = False) -> str:
+    """Compiles oracle.cpp into liboracle.so next to it (g++, -O2)."""
+    src = os.path.join(_HERE, "oracle.cpp")
+    out = os.path.join(_HERE, "liboracle.so")
+    if force or not os.path.exists(out) or os.path.getmtime(out) < max(
+            os.path.getmtime(src), os.path.getmtime(os.path.join(_HERE, "oracle.h"))):
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", out, src])
+    return out
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, u32, u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
+        lib.oracle_pair.argtypes = [vp, vp, u32, u32, vp, u64, vp, vp, u64, vp, vp]
+        lib.oracle_aggregate.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp]
+        lib.oracle_overlap.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp]
+        for f in (lib.oracle_pair, lib.oracle_aggregate, lib.oracle_overlap):
+            f.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data
+
+
+def pair(events: np.ndarray, stream_offsets: np.ndarray, num_regions: int, interval_cap: int | None = None,
+         ambig_cap: int | None = None):
+    """Returns (rc, intervals, interval_offsets, ambig, ambig_offsets, status)."""
+    events = np.ascontiguousarray(events, dtype=EVENT)
+    offs = np.ascontiguousarray(stream_offsets, dtype=np.uint64)
+    S = len(offs) - 1
+    n = len(events)
+    icap = n // 2 if interval_cap is None else interval_cap
+    acap = n if ambig_cap is None else ambig_cap
+    iv = np.zeros(icap, dtype=INTERVAL)
+    am = np.zeros(acap, dtype=AMBIG)
+    ioffs = np.zeros(S + 1, dtype=np.uint64)
+    aoffs = np.zeros(S + 1, dtype=np.uint64)
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_pair(_ptr(events), _ptr(offs), S, num_regions, _ptr(iv), icap, _ptr(ioffs), _ptr(am), acap,
+                             _ptr(aoffs), _ptr(st))
+    ni = min(int(ioffs[S]), icap)
+    na = min(int(aoffs[S]), acap)
+    return rc, iv[:ni], ioffs, am[:na], aoffs, st[0]
+
+
+def aggregate(intervals, interval_offsets, ambig, ambig_offsets, warps_per_cta, cta_sm, num_sms, num_regions,
+              levels=("warp", "cta", "sm", "kernel")):
+    """Returns (rc, {level: table [keys, R]}, status)."""
+    iv = np.ascontiguousarray(intervals, dtype=INTERVAL)
+    ioffs = np.ascontiguousarray(interval_offsets, dtype=np.uint64)
+    S = len(ioffs) - 1
+    am = None if ambig is None else np.ascontiguousarray(ambig, dtype=AMBIG)
+    aoffs = None if ambig_offsets is None else np.ascontiguousarray(ambig_offsets, dtype=np.uint64)
+    cs = np.ascontiguousarray(cta_sm, dtype=np.uint32)
+    C = S // warps_per_cta if warps_per_cta else 0
+    keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1}
+    tabs = {lv: (np.zeros((keys[lv], num_regions), dtype=AGG) if lv in levels else None) for lv in keys}
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_aggregate(_ptr(iv), _ptr(ioffs), _ptr(am), _ptr(aoffs), S, warps_per_cta, _ptr(cs), num_sms,
+                                  num_regions, _ptr(tabs["warp"]), _ptr(tabs["cta"]), _ptr(tabs["sm"]),
+                                  _ptr(tabs["kernel"]), _ptr(st))
+    return rc, {k: v for k, v in tabs.items() if v is not None}, st[0]
+
+
+def overlap(intervals, interval_offsets, warps_per_cta, cta_sm, num_sms, pairs):
+    """Returns (rc, out [K, M], status)."""
+    iv = np.ascontiguousarray(intervals, dtype=INTERVAL)
+    ioffs = np.ascontiguousarray(interval_offsets, dtype=np.uint64)
+    S = len(ioffs) - 1
+    cs = np.ascontiguousarray(cta_sm, dtype=np.uint32)
+    pr = np.ascontiguousarray(pairs, dtype=np.uint32).reshape(-1, 2)
+    out = np.zeros((len(pr), num_sms), dtype=OVERLAP)
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_overlap(_ptr(iv), _ptr(ioffs), S, warps_per_cta, _ptr(cs), num_sms, _ptr(pr), len(pr),
+                                _ptr(out), _ptr(st))
+    return rc, out, st[0]

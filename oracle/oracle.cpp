@@ -1,0 +1,263 @@
+// oracle.cpp — single-threaded CPU oracle (test infrastructure; see oracle.h).
+//
+// Written from the sequential definition, not from the CUDA path: an explicit std::vector
+// stack per stream, std::map aggregates, sort + two-pointer sweep for overlap. No blocking,
+// no fusion, no reordering beyond what the definition states.
+#include "oracle.h"
+
+#include <algorithm>
+#include <cstring>
+#include <map>
+#include <tuple>
+#include <utility>
+#include <vector>
+
+namespace {
+
+constexpr uint32_t kNone = 0xFFFFFFFFu;
+constexpr size_t kMaxDepth = 64;
+enum { OK = 0, ERR_INVALID = 1, ERR_CAPACITY = 4, ERR_DEPTH = 5, ERR_BAD_REGION = 6, ERR_BAD_OFFSETS = 7 };
+enum { FLAG_CTX = 1, FLAG_REV = 2, FLAG_CLAMP = 4 };
+enum { AMB_END = 1, AMB_MISNESTED = 2, AMB_EOS = 3 };
+
+struct Frame {
+  uint32_t region, ctx;
+  uint64_t ts;
+  uint32_t idx;
+  uint32_t depth;
+  uint32_t parent;
+  uint64_t child;  // sum of inclusive time of matched intervals directly below this frame
+};
+
+void fail(OStatus* st, uint32_t code, uint32_t stream, uint64_t ev) {
+  if (st->code == OK) { st->code = code; st->bad_stream = stream; st->bad_event = ev; }
+}
+
+}  // namespace
+
+extern "C" int oracle_pair(const OEvent* events, const uint64_t* stream_offsets, uint32_t num_streams,
+                           uint32_t num_regions, OInterval* intervals, uint64_t interval_cap,
+                           uint64_t* interval_offsets, OAmbig* ambig, uint64_t ambig_cap,
+                           uint64_t* ambig_offsets, OStatus* st) {
+  if (!stream_offsets || !interval_offsets || !ambig_offsets || !st) return ERR_INVALID;
+  if (num_regions == 0 || num_regions > 65536) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  uint64_t n_int = 0, n_amb = 0;
+  interval_offsets[0] = 0;
+  ambig_offsets[0] = 0;
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    const uint64_t lo = stream_offsets[s], hi = stream_offsets[s + 1];
+    if (hi < lo) { fail(st, ERR_BAD_OFFSETS, s, 0); return OK; }
+    const uint64_t n = hi - lo;
+    std::vector<Frame> stack;
+    std::vector<OAmbig> amb;  // this stream's records, sorted by event index at the end
+    auto note = [&](uint32_t kind, uint64_t ts, uint32_t tag, uint32_t ctx, uint32_t idx, uint32_t depth) {
+      amb.push_back(OAmbig{ts, tag, ctx, s, idx, kind, depth});
+    };
+    for (uint64_t i = 0; i < n; ++i) {
+      const OEvent& e = events[lo + i];
+      const uint32_t region = e.tag >> 1;
+      const bool is_end = (e.tag & 1u) != 0;
+      if (region >= num_regions) { fail(st, ERR_BAD_REGION, s, i); return OK; }
+      if (!is_end) {
+        if (stack.size() == kMaxDepth) { fail(st, ERR_DEPTH, s, i); return OK; }
+        Frame f;
+        f.region = region; f.ctx = e.ctx; f.ts = e.ts; f.idx = static_cast<uint32_t>(i);
+        f.depth = static_cast<uint32_t>(stack.size());
+        f.parent = stack.empty() ? kNone : stack.back().region;
+        f.child = 0;
+        stack.push_back(f);
+        continue;
+      }
+      // end marker: innermost open frame of the same region, searching down from the top
+      long k = static_cast<long>(stack.size()) - 1;
+      while (k >= 0 && stack[static_cast<size_t>(k)].region != region) --k;
+      if (k < 0) {
+        note(AMB_END, e.ts, e.tag, e.ctx, static_cast<uint32_t>(i), static_cast<uint32_t>(stack.size()));
+        continue;
+      }
+      while (static_cast<long>(stack.size()) - 1 > k) {  // force-close mis-nested frames
+        Frame f = stack.back();
+        stack.pop_back();
+        note(AMB_MISNESTED, f.ts, f.region << 1, f.ctx, f.idx, f.depth);
+        stack.back().child += f.child;  // grandchildren time moves up
+      }
+      Frame f = stack.back();
+      stack.pop_back();
+      uint16_t flags = 0;
+      uint64_t incl, excl;
+      if (e.ctx != f.ctx) { flags |= FLAG_CTX; st->n_ctx_mismatch++; }
+      if (e.ts < f.ts) { incl = 0; flags |= FLAG_REV; st->n_time_reversed++; } else { incl = e.ts - f.ts; }
+      if (f.child > incl) { excl = 0; flags |= FLAG_CLAMP; st->n_child_clamped++; } else { excl = incl - f.child; }
+      if (n_int < interval_cap && intervals) {
+        OInterval& o = intervals[n_int];
+        o.t_begin = f.ts; o.inclusive = incl; o.exclusive = excl;
+        o.region = f.region; o.ctx = f.ctx; o.stream = s; o.parent_region = f.parent;
+        o.begin_idx = f.idx; o.depth = static_cast<uint16_t>(f.depth); o.flags = flags;
+      }
+      ++n_int;
+      if (!stack.empty()) stack.back().child += incl;
+    }
+    for (const Frame& f : stack) note(AMB_EOS, f.ts, f.region << 1, f.ctx, f.idx, f.depth);
+    std::sort(amb.begin(), amb.end(), [](const OAmbig& a, const OAmbig& b) { return a.event_idx < b.event_idx; });
+    for (const OAmbig& a : amb) {
+      if (n_amb < ambig_cap && ambig) ambig[n_amb] = a;
+      ++n_amb;
+    }
+    interval_offsets[s + 1] = n_int;
+    ambig_offsets[s + 1] = n_amb;
+  }
+  st->intervals_required = n_int;
+  st->ambig_required = n_amb;
+  if (n_int > interval_cap) fail(st, ERR_CAPACITY, 0, n_int);
+  else if (n_amb > ambig_cap) fail(st, ERR_CAPACITY, 0, n_amb);
+  return OK;
+}
+
+namespace {
+
+int bin_of(uint64_t d) {  // floor(log2 d), with d in {0, 1} -> 0
+  int b = 0;
+  while (d > 1) { d >>= 1; ++b; }
+  return b;
+}
+
+struct Cell {
+  OAgg a;
+  Cell() { std::memset(&a, 0, sizeof(a)); a.min_incl = ~0ull; }
+};
+
+using Key = std::tuple<int, uint32_t, uint32_t>;  // (level, scope key, region)
+
+void materialise(const std::map<Key, Cell>& m, int level, uint32_t nkeys, uint32_t R, OAgg* tab) {
+  if (!tab) return;
+  Cell empty;
+  for (uint64_t i = 0; i < static_cast<uint64_t>(nkeys) * R; ++i) tab[i] = empty.a;
+  for (const auto& kv : m) {
+    if (std::get<0>(kv.first) != level) continue;
+    tab[static_cast<uint64_t>(std::get<1>(kv.first)) * R + std::get<2>(kv.first)] = kv.second.a;
+  }
+}
+
+}  // namespace
+
+extern "C" int oracle_aggregate(const OInterval* intervals, const uint64_t* interval_offsets,
+                                const OAmbig* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                                uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                                uint32_t num_regions, OAgg* warp_tab, OAgg* cta_tab, OAgg* sm_tab,
+                                OAgg* kernel_tab, OStatus* st) {
+  if (!interval_offsets || !st || warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ERR_INVALID;
+  if (num_regions == 0 || num_regions > 65536) return ERR_INVALID;
+  if ((sm_tab != nullptr) && (!cta_sm || num_sms == 0)) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  const uint32_t num_ctas = num_streams / warps_per_cta;
+  std::map<Key, Cell> m;
+  auto keys_of = [&](uint32_t s, uint32_t keys[4]) {
+    keys[0] = s;
+    keys[1] = s / warps_per_cta;
+    keys[2] = cta_sm ? cta_sm[s / warps_per_cta] : 0;
+    keys[3] = 0;
+  };
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    uint32_t keys[4];
+    keys_of(s, keys);
+    if (cta_sm && keys[2] >= num_sms && sm_tab) return ERR_INVALID;
+    for (uint64_t i = interval_offsets[s]; i < interval_offsets[s + 1]; ++i) {
+      const OInterval& v = intervals[i];
+      if (v.region >= num_regions) { fail(st, ERR_BAD_REGION, s, i); return OK; }
+      for (int level = 0; level < 4; ++level) {
+        OAgg& a = m[Key(level, keys[level], v.region)].a;
+        a.count++;
+        a.sum_incl += v.inclusive;
+        a.min_incl = std::min(a.min_incl, v.inclusive);
+        a.max_incl = std::max(a.max_incl, v.inclusive);
+        a.sum_excl += v.exclusive;
+        a.n_flagged += (v.flags != 0);
+        a.hist[bin_of(v.inclusive)]++;
+      }
+    }
+    if (ambig && ambig_offsets) {
+      for (uint64_t i = ambig_offsets[s]; i < ambig_offsets[s + 1]; ++i) {
+        const OAmbig& r = ambig[i];
+        const uint32_t region = r.tag >> 1;
+        if (region >= num_regions) { fail(st, ERR_BAD_REGION, s, i); return OK; }
+        for (int level = 0; level < 4; ++level) {
+          OAgg& a = m[Key(level, keys[level], region)].a;
+          if (r.kind == AMB_END) a.n_unmatched_end++; else a.n_unmatched_begin++;
+        }
+      }
+    }
+  }
+  materialise(m, 0, num_streams, num_regions, warp_tab);
+  materialise(m, 1, num_ctas, num_regions, cta_tab);
+  materialise(m, 2, num_sms, num_regions, sm_tab);
+  materialise(m, 3, 1, num_regions, kernel_tab);
+  return OK;
+}
+
+namespace {
+
+using Span = std::pair<uint64_t, uint64_t>;  // half-open [first, second)
+
+std::vector<Span> merged_union(std::vector<Span> v) {
+  std::sort(v.begin(), v.end());
+  std::vector<Span> u;
+  for (const Span& s : v) {
+    if (!u.empty() && s.first <= u.back().second) u.back().second = std::max(u.back().second, s.second);
+    else u.push_back(s);
+  }
+  return u;
+}
+
+uint64_t measure(const std::vector<Span>& u) {
+  uint64_t t = 0;
+  for (const Span& s : u) t += s.second - s.first;
+  return t;
+}
+
+}  // namespace
+
+extern "C" int oracle_overlap(const OInterval* intervals, const uint64_t* interval_offsets,
+                              uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,
+                              uint32_t num_sms, const uint32_t* pairs, uint32_t num_pairs, OOverlap* out,
+                              OStatus* st) {
+  if (!interval_offsets || !cta_sm || !st || warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ERR_INVALID;
+  if (num_pairs && (!pairs || !out)) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  std::vector<std::vector<uint32_t>> streams_of_sm(num_sms);  // which streams ran on each SM
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    const uint32_t m = cta_sm[s / warps_per_cta];
+    if (m >= num_sms) return ERR_INVALID;
+    streams_of_sm[m].push_back(s);
+  }
+  for (uint32_t k = 0; k < num_pairs; ++k) {
+    const uint32_t P = pairs[2 * k], Cn = pairs[2 * k + 1];
+    for (uint32_t m = 0; m < num_sms; ++m) {
+      std::vector<Span> p, c;
+      for (uint32_t s : streams_of_sm[m]) {
+        for (uint64_t i = interval_offsets[s]; i < interval_offsets[s + 1]; ++i) {
+          const OInterval& v = intervals[i];
+          if (v.inclusive == 0) continue;  // empty span
+          const Span sp(v.t_begin, v.t_begin + v.inclusive);
+          if (v.region == P) p.push_back(sp);
+          if (v.region == Cn) c.push_back(sp);
+        }
+      }
+      const std::vector<Span> up = merged_union(p), uc = merged_union(c);
+      uint64_t both = 0;
+      size_t a = 0, b = 0;
+      while (a < up.size() && b < uc.size()) {  // two-pointer sweep over disjoint sorted spans
+        const uint64_t lo = std::max(up[a].first, uc[b].first);
+        const uint64_t hi = std::min(up[a].second, uc[b].second);
+        if (hi > lo) both += hi - lo;
+        if (up[a].second < uc[b].second) ++a; else ++b;
+      }
+      OOverlap& o = out[static_cast<uint64_t>(k) * num_sms + m];
+      o.producer_ns = measure(up);
+      o.consumer_ns = measure(uc);
+      o.overlap_ns = both;
+      o.either_ns = o.producer_ns + o.consumer_ns - both;
+    }
+  }
+  return OK;
+}

@@ -1,0 +1,62 @@
+/*
+ * oracle.h — record layouts and entry points of the CPU oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY. This is a plain, slow, single-threaded restatement of what the
+ * hot path computes, used by the tests, the smoke check and the CPU-baseline leg of the
+ * benchmark. It shares no code with the CUDA library: the layouts below are retyped here
+ * on purpose and nothing in the product may include or link this.
+ *
+ * Every function follows the sequential definition of the per-warp nested region context
+ * stack (paper Section 3.2, "Region Semantics and Identity") and of scopes as selections
+ * of executions (Section 3.2, "Region and scope"). All arithmetic is unsigned 64-bit.
+ * Parity status: every function here is pinned by tests (hand-worked examples, brute-force
+ * pairing enumeration, closed forms and invariants); nothing is "parity unpinned".
+ */
+#ifndef ORACLE_H_
+#define ORACLE_H_
+#include <cstddef>
+#include <cstdint>
+
+extern "C" {
+
+struct OEvent { uint64_t ts; uint32_t tag; uint32_t ctx; };                     // 16 B
+struct OInterval {                                                               // 48 B
+  uint64_t t_begin, inclusive, exclusive;
+  uint32_t region, ctx, stream, parent_region, begin_idx;
+  uint16_t depth, flags;
+};
+struct OAmbig { uint64_t ts; uint32_t tag, ctx, stream, event_idx, kind, depth; };  // 32 B
+struct OAgg {                                                                    // 576 B
+  uint64_t count, sum_incl, min_incl, max_incl, sum_excl;
+  uint64_t n_unmatched_begin, n_unmatched_end, n_flagged;
+  uint64_t hist[64];
+};
+struct OOverlap { uint64_t overlap_ns, producer_ns, consumer_ns, either_ns; };   // 32 B
+struct OStatus {                                                                 // 64 B
+  uint32_t code, bad_stream;
+  uint64_t bad_event, intervals_required, ambig_required;
+  uint64_t n_ctx_mismatch, n_time_reversed, n_child_clamped, reserved;
+};
+
+// Step 1-3: stack matching, durations, ambiguity records. Host pointers throughout.
+// Returns 0 or a host-detectable code; device-class conditions go to st->code, as the
+// library does. interval_cap / ambig_cap: capacity of the output arrays in records.
+int oracle_pair(const OEvent* events, const uint64_t* stream_offsets, uint32_t num_streams,
+                uint32_t num_regions, OInterval* intervals, uint64_t interval_cap,
+                uint64_t* interval_offsets, OAmbig* ambig, uint64_t ambig_cap,
+                uint64_t* ambig_offsets, OStatus* st);
+
+// Step 4: per-(region, scope) statistics. Any table may be null.
+int oracle_aggregate(const OInterval* intervals, const uint64_t* interval_offsets,
+                     const OAmbig* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                     uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                     uint32_t num_regions, OAgg* warp_tab, OAgg* cta_tab, OAgg* sm_tab,
+                     OAgg* kernel_tab, OStatus* st);
+
+// Step 4 (second half): per-SM overlap of producer/consumer region pairs.
+int oracle_overlap(const OInterval* intervals, const uint64_t* interval_offsets,
+                   uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,
+                   uint32_t num_sms, const uint32_t* pairs, uint32_t num_pairs, OOverlap* out,
+                   OStatus* st);
+}
+#endif
