@@ -55,8 +55,7 @@ enum {
   ARGUS_ERR_DEPTH = 5,       /* device: a stream would hold more than ARGUS_MAX_DEPTH open frames */
   ARGUS_ERR_BAD_REGION = 6,  /* device: tag>>1 >= num_regions                             */
   ARGUS_ERR_BAD_OFFSETS = 7, /* device: stream_offsets / interval_offsets not non-decreasing */
-  ARGUS_ERR_TIMEOUT = 8,     /* device: a bounded wait expired (reserved)                 */
-  ARGUS_ERR_RANGE = 9        /* device: a timestamp is outside the range overlap supports  */
+  ARGUS_ERR_TIMEOUT = 8      /* device: a bounded wait expired (reserved)                 */
 };
 
 /* One marker event, 16 bytes. tag = region_id << 1 | is_end. ts = globaltimer ns.
@@ -160,15 +159,17 @@ typedef struct {
  * interval_offsets[S+1]; ambiguity records ordered by (stream, event_idx) with
  * ambig_offsets[S+1]. interval_capacity >= floor(N/2) and ambig_capacity >= N always
  * suffice; otherwise ARGUS_ERR_CAPACITY reports the required counts in `status`.
- * Requirements: events 16-byte aligned; num_regions in [1, ARGUS_MAX_REGIONS];
- * every stream shorter than 2^32 events; workspace 256-byte aligned and at least
- * argus_pair_workspace_bytes(N, S, ambig_capacity) bytes. `status` (device, 64 B) is
+ * Requirements: events 16-byte aligned; num_events = length of `events` (every
+ * stream_offsets value must be <= num_events, else ARGUS_ERR_BAD_OFFSETS);
+ * num_regions in [1, ARGUS_MAX_REGIONS]; every stream shorter than 2^32 events;
+ * num_events < 2^48; workspace 256-byte aligned and at least
+ * argus_pair_workspace_bytes(num_events, S, ambig_capacity) bytes. `status` (device, 64 B) is
  * overwritten. Empty streams and num_streams == 0 are legal.
  * ------------------------------------------------------------------------------------- */
 size_t argus_pair_workspace_bytes(uint64_t num_events, uint32_t num_streams,
                                   uint64_t ambig_capacity);
 
-int argus_pair_intervals(const argus_event_t* events /*device*/,
+int argus_pair_intervals(const argus_event_t* events /*device*/, uint64_t num_events,
                          const uint64_t* stream_offsets /*device [S+1]*/,
                          uint32_t num_streams, uint32_t num_regions,
                          argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
@@ -177,6 +178,20 @@ int argus_pair_intervals(const argus_event_t* events /*device*/,
                          uint64_t* ambig_offsets /*device [S+1] out*/,
                          argus_status_t* status /*device*/, void* workspace /*device*/,
                          size_t workspace_bytes, void* cuda_stream);
+
+/* Same operation with an explicit kernel choice, for tests and profiling:
+ * kernel_choice 0 = automatic, 1 = one thread per stream (sequential stack, any input),
+ * 2 = tiled kernel (one CTA walks a stream tile by tile; falls back to the sequential stack
+ * inside tiles that are not well-nested). All choices produce identical output. */
+int argus_pair_intervals_ex(const argus_event_t* events /*device*/, uint64_t num_events,
+                            const uint64_t* stream_offsets /*device [S+1]*/,
+                            uint32_t num_streams, uint32_t num_regions,
+                            argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
+                            uint64_t* interval_offsets /*device [S+1] out*/,
+                            argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
+                            uint64_t* ambig_offsets /*device [S+1] out*/,
+                            argus_status_t* status /*device*/, void* workspace /*device*/,
+                            size_t workspace_bytes, void* cuda_stream, int kernel_choice);
 
 /* ---------------------------------------------------------------------------------------
  * argus_aggregate — Section 3.2 "Region and scope" + the `duration` signal (Section 3.1).
@@ -213,12 +228,14 @@ int argus_aggregate(const argus_interval_t* intervals /*device*/,
  * spans [t_begin, t_begin + inclusive) of all intervals of region P (resp. Cn) in streams
  * whose CTA maps to m (all depths and contexts, flagged ones included, empty spans
  * dropped); U_P, U_C = their unions. out[k][m] = { |U_P ∩ U_C|, |U_P|, |U_C|, |U_P ∪ U_C| }.
- * Timestamps must satisfy t_begin + inclusive < 2^62, else ARGUS_ERR_RANGE.
+ * max_intervals is an upper bound of interval_offsets[S] known on the host (for instance
+ * the capacity given to argus_pair_intervals); it sizes the workspace. If more spans are
+ * selected than the workspace holds, status->code = ARGUS_ERR_CAPACITY.
  * ------------------------------------------------------------------------------------- */
-size_t argus_overlap_workspace_bytes(uint64_t num_intervals, uint32_t num_streams,
+size_t argus_overlap_workspace_bytes(uint64_t max_intervals, uint32_t num_streams,
                                      uint32_t num_pairs, uint32_t num_sms);
 
-int argus_overlap(const argus_interval_t* intervals /*device*/,
+int argus_overlap(const argus_interval_t* intervals /*device*/, uint64_t max_intervals,
                   const uint64_t* interval_offsets /*device [S+1]*/, uint32_t num_streams,
                   uint32_t warps_per_cta, const uint32_t* cta_sm /*device [C]*/,
                   uint32_t num_sms, const uint32_t* pairs /*device [K][2]*/,

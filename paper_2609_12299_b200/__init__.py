@@ -1,0 +1,17 @@
+"""B200-native region-trace synthesis: marker events -> intervals -> scope statistics -> overlap.
+
+Thin binding over the C-ABI library `libargus.so` (see include/argus.h). Every step of the path runs
+in the library's CUDA kernels; this module only marshals arguments and uses PyTorch for device
+memory and streams. There is no CPU fallback: if the library has not been built, every call raises.
+"""
+from .binding import (AGG_DTYPE, AMBIG_DTYPE, EVENT_DTYPE, INTERVAL_DTYPE, OVERLAP_DTYPE, STATUS_DTYPE, ArgusError,
+                      AggregateResult, PairResult, argus_aggregate, argus_aggregate_workspace_bytes, argus_overlap,
+                      argus_overlap_workspace_bytes, argus_pair_intervals, argus_pair_workspace_bytes,
+                      argus_status_fetch, argus_strerror, argus_version, library_path, load_library, pair_aggregate_host)
+
+__all__ = [
+    "AGG_DTYPE", "AMBIG_DTYPE", "EVENT_DTYPE", "INTERVAL_DTYPE", "OVERLAP_DTYPE", "STATUS_DTYPE", "ArgusError",
+    "AggregateResult", "PairResult", "argus_aggregate", "argus_aggregate_workspace_bytes", "argus_overlap",
+    "argus_overlap_workspace_bytes", "argus_pair_intervals", "argus_pair_workspace_bytes", "argus_status_fetch",
+    "argus_strerror", "argus_version", "library_path", "load_library", "pair_aggregate_host",
+]

@@ -1,0 +1,266 @@
+"""ctypes binding of libargus.so: same names as the C-ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+
+EVENT_DTYPE = np.dtype([("ts", "<u8"), ("tag", "<u4"), ("ctx", "<u4")])
+INTERVAL_DTYPE = np.dtype([("t_begin", "<u8"), ("inclusive", "<u8"), ("exclusive", "<u8"), ("region", "<u4"),
+                           ("ctx", "<u4"), ("stream", "<u4"), ("parent_region", "<u4"), ("begin_idx", "<u4"),
+                           ("depth", "<u2"), ("flags", "<u2")])
+AMBIG_DTYPE = np.dtype([("ts", "<u8"), ("tag", "<u4"), ("ctx", "<u4"), ("stream", "<u4"), ("event_idx", "<u4"),
+                        ("kind", "<u4"), ("depth", "<u4")])
+AGG_DTYPE = np.dtype([("count", "<u8"), ("sum_incl", "<u8"), ("min_incl", "<u8"), ("max_incl", "<u8"),
+                      ("sum_excl", "<u8"), ("n_unmatched_begin", "<u8"), ("n_unmatched_end", "<u8"),
+                      ("n_flagged", "<u8"), ("hist", "<u8", (64,))])
+OVERLAP_DTYPE = np.dtype([("overlap_ns", "<u8"), ("producer_ns", "<u8"), ("consumer_ns", "<u8"), ("either_ns", "<u8")])
+STATUS_DTYPE = np.dtype([("code", "<u4"), ("bad_stream", "<u4"), ("bad_event", "<u8"), ("intervals_required", "<u8"),
+                         ("ambig_required", "<u8"), ("n_ctx_mismatch", "<u8"), ("n_time_reversed", "<u8"),
+                         ("n_child_clamped", "<u8"), ("reserved", "<u8")])
+
+KERNEL_AUTO, KERNEL_THREAD_PER_STREAM, KERNEL_TILED = 0, 1, 2
+
+
+class ArgusError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {argus_strerror(code)} (code {code})")
+        self.code = code
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libargus.so")
+
+
+_lib = None
+
+
+def load_library():
+    """Loads libargus.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} not found: build it with `python -c 'import __graft_entry__ as g; g.build()'`; "
+                           "this package has no CPU fallback")
+    lib = ctypes.CDLL(path)
+    vp, u32, u64, sz, ci = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_size_t, ctypes.c_int
+    lib.argus_pair_workspace_bytes.argtypes = [u64, u32, u64]
+    lib.argus_pair_workspace_bytes.restype = sz
+    pair_args = [vp, u64, vp, u32, u32, vp, u64, vp, vp, u64, vp, vp, vp, sz, vp]
+    lib.argus_pair_intervals.argtypes = pair_args
+    lib.argus_pair_intervals.restype = ci
+    lib.argus_pair_intervals_ex.argtypes = pair_args + [ci]
+    lib.argus_pair_intervals_ex.restype = ci
+    lib.argus_aggregate_workspace_bytes.argtypes = [u64, u32, u32]
+    lib.argus_aggregate_workspace_bytes.restype = sz
+    lib.argus_aggregate.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.argus_aggregate.restype = ci
+    lib.argus_overlap_workspace_bytes.argtypes = [u64, u32, u32, u32]
+    lib.argus_overlap_workspace_bytes.restype = sz
+    lib.argus_overlap.argtypes = [vp, u64, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp, sz, vp]
+    lib.argus_overlap.restype = ci
+    lib.argus_status_fetch.argtypes = [vp, vp, vp]
+    lib.argus_status_fetch.restype = ci
+    lib.argus_strerror.argtypes = [ci]
+    lib.argus_strerror.restype = ctypes.c_char_p
+    lib.argus_version.argtypes = []
+    lib.argus_version.restype = ci
+    _lib = lib
+    return lib
+
+
+def argus_strerror(code: int) -> str:
+    return load_library().argus_strerror(int(code)).decode()
+
+
+def argus_version() -> int:
+    return load_library().argus_version()
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(device):
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _bytes(n: int, device) -> torch.Tensor:
+    return torch.empty(max(int(n), 1), dtype=torch.uint8, device=device)
+
+
+def argus_pair_workspace_bytes(num_events: int, num_streams: int, ambig_capacity: int) -> int:
+    return load_library().argus_pair_workspace_bytes(num_events, num_streams, ambig_capacity)
+
+
+def argus_aggregate_workspace_bytes(num_intervals: int, num_streams: int, num_regions: int) -> int:
+    return load_library().argus_aggregate_workspace_bytes(num_intervals, num_streams, num_regions)
+
+
+def argus_overlap_workspace_bytes(max_intervals: int, num_streams: int, num_pairs: int, num_sms: int) -> int:
+    return load_library().argus_overlap_workspace_bytes(max_intervals, num_streams, num_pairs, num_sms)
+
+
+def argus_status_fetch(status: torch.Tensor) -> np.void:
+    """Synchronises the current stream and returns the status block as a numpy record."""
+    host = np.zeros(1, dtype=STATUS_DTYPE)
+    rc = load_library().argus_status_fetch(status.data_ptr(), host.ctypes.data, _stream_ptr(status.device))
+    if rc != 0:
+        raise ArgusError(rc, "argus_status_fetch")
+    return host[0]
+
+
+@dataclass
+class PairResult:
+    intervals: torch.Tensor          # uint8 [interval_capacity * 48]
+    interval_offsets: torch.Tensor   # int64 [S + 1]
+    ambig: torch.Tensor              # uint8 [ambig_capacity * 32]
+    ambig_offsets: torch.Tensor      # int64 [S + 1]
+    status: torch.Tensor             # uint8 [64]
+    interval_capacity: int
+    ambig_capacity: int
+    workspace: torch.Tensor
+
+    def fetch_status(self):
+        return argus_status_fetch(self.status)
+
+    def intervals_numpy(self) -> np.ndarray:
+        n = min(int(self.interval_offsets[-1].item()), self.interval_capacity)
+        return self.intervals[: n * 48].cpu().numpy().view(INTERVAL_DTYPE)
+
+    def ambig_numpy(self) -> np.ndarray:
+        n = min(int(self.ambig_offsets[-1].item()), self.ambig_capacity)
+        return self.ambig[: n * 32].cpu().numpy().view(AMBIG_DTYPE)
+
+
+def argus_pair_intervals(events: torch.Tensor, stream_offsets: torch.Tensor, num_regions: int,
+                         interval_capacity: int | None = None, ambig_capacity: int | None = None,
+                         out: PairResult | None = None, kernel: int = KERNEL_AUTO) -> PairResult:
+    """events: device tensor holding N 16-byte records; stream_offsets: device int64 [S+1].
+    Enqueues on the current stream of the events' device and returns device tensors (no sync)."""
+    lib = load_library()
+    dev = events.device
+    if dev.type != "cuda":
+        raise ValueError("events must be a CUDA tensor")
+    n = events.numel() * events.element_size() // 16
+    S = stream_offsets.numel() - 1
+    icap = n // 2 if interval_capacity is None else int(interval_capacity)
+    acap = n if ambig_capacity is None else int(ambig_capacity)
+    if out is None:
+        ws_bytes = lib.argus_pair_workspace_bytes(n, S, acap)
+        out = PairResult(_bytes(icap * 48, dev), torch.empty(S + 1, dtype=torch.int64, device=dev),
+                         _bytes(acap * 32, dev), torch.empty(S + 1, dtype=torch.int64, device=dev),
+                         _bytes(64, dev), icap, acap, _bytes(ws_bytes, dev))
+    rc = lib.argus_pair_intervals_ex(_ptr(events), n, _ptr(stream_offsets), S, num_regions, _ptr(out.intervals),
+                                     out.interval_capacity, _ptr(out.interval_offsets), _ptr(out.ambig),
+                                     out.ambig_capacity, _ptr(out.ambig_offsets), _ptr(out.status),
+                                     _ptr(out.workspace), out.workspace.numel(), _stream_ptr(dev), kernel)
+    if rc != 0:
+        raise ArgusError(rc, "argus_pair_intervals")
+    return out
+
+
+@dataclass
+class AggregateResult:
+    warp: torch.Tensor | None    # uint8 [S * R * 576]
+    cta: torch.Tensor | None
+    sm: torch.Tensor | None
+    kernel: torch.Tensor | None
+    status: torch.Tensor
+    workspace: torch.Tensor
+    shape: dict
+
+    def table_numpy(self, level: str) -> np.ndarray:
+        t = getattr(self, level)
+        return t.cpu().numpy().view(AGG_DTYPE).reshape(self.shape[level])
+
+
+def argus_aggregate(intervals: torch.Tensor, interval_offsets: torch.Tensor, ambig: torch.Tensor | None,
+                    ambig_offsets: torch.Tensor | None, warps_per_cta: int, cta_sm: torch.Tensor, num_sms: int,
+                    num_regions: int, levels=("warp", "cta", "sm", "kernel"),
+                    out: AggregateResult | None = None) -> AggregateResult:
+    lib = load_library()
+    dev = intervals.device
+    S = interval_offsets.numel() - 1
+    C = S // warps_per_cta if warps_per_cta else 0
+    keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1}
+    if out is None:
+        tabs = {lv: (_bytes(keys[lv] * num_regions * 576, dev) if lv in levels else None) for lv in keys}
+        ws = _bytes(lib.argus_aggregate_workspace_bytes(intervals.numel() // 48, S, num_regions), dev)
+        out = AggregateResult(tabs["warp"], tabs["cta"], tabs["sm"], tabs["kernel"], _bytes(64, dev), ws,
+                              {lv: (keys[lv], num_regions) for lv in keys})
+    rc = lib.argus_aggregate(_ptr(intervals), _ptr(interval_offsets), _ptr(ambig), _ptr(ambig_offsets), S,
+                             warps_per_cta, _ptr(cta_sm), num_sms, num_regions, _ptr(out.warp), _ptr(out.cta),
+                             _ptr(out.sm), _ptr(out.kernel), _ptr(out.status), _ptr(out.workspace),
+                             out.workspace.numel(), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_aggregate")
+    return out
+
+
+def argus_overlap(intervals: torch.Tensor, max_intervals: int, interval_offsets: torch.Tensor, warps_per_cta: int,
+                  cta_sm: torch.Tensor, num_sms: int, pairs: torch.Tensor, workspace: torch.Tensor | None = None,
+                  workspace_bytes: int | None = None):
+    """pairs: device int32/uint32 [K, 2]. Returns (out uint8 [K * M * 32], status uint8 [64])."""
+    lib = load_library()
+    dev = intervals.device
+    S = interval_offsets.numel() - 1
+    K = pairs.numel() // 2
+    if workspace is None:
+        need = workspace_bytes if workspace_bytes is not None else lib.argus_overlap_workspace_bytes(max_intervals, S, K, num_sms)
+        workspace = _bytes(need, dev)
+    out = _bytes(K * num_sms * 32, dev)
+    status = _bytes(64, dev)
+    rc = lib.argus_overlap(_ptr(intervals), max_intervals, _ptr(interval_offsets), S, warps_per_cta, _ptr(cta_sm),
+                           num_sms, _ptr(pairs), K, _ptr(out), _ptr(status), _ptr(workspace), workspace.numel(),
+                           _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_overlap")
+    return out, status
+
+
+def pair_aggregate_host(events: np.ndarray, stream_offsets: np.ndarray, num_regions: int, warps_per_cta: int,
+                        cta_sm: np.ndarray, num_sms: int, device="cuda:0", state: dict | None = None):
+    """End-to-end call with HOST buffers: copies the events (and offsets) to the device, runs
+    argus_pair_intervals + argus_aggregate, and copies the kernel-, SM- and CTA-scope tables, the
+    interval offsets and the status block back. `state` (a dict the caller keeps) caches pinned staging
+    and device buffers between calls. Returns (tables dict of numpy arrays, interval_offsets, status)."""
+    dev = torch.device(device)
+    st = state if state is not None else {}
+    n = len(events)
+    S = len(stream_offsets) - 1
+    key = (n, S, num_regions)
+    if st.get("key") != key:
+        st.clear()
+        st["key"] = key
+        st["pin_ev"] = torch.empty(max(n, 1) * 16, dtype=torch.uint8).pin_memory()
+        st["pin_off"] = torch.empty(S + 1, dtype=torch.int64).pin_memory()
+        st["dev_ev"] = torch.empty(max(n, 1) * 16, dtype=torch.uint8, device=dev)
+        st["dev_off"] = torch.empty(S + 1, dtype=torch.int64, device=dev)
+        st["cta_sm"] = torch.from_numpy(np.ascontiguousarray(cta_sm, dtype=np.uint32).view(np.int32)).to(dev)
+        st["pair"] = None
+        st["agg"] = None
+    ev_bytes = np.ascontiguousarray(events).view(np.uint8).reshape(-1)
+    if ev_bytes.ctypes.data != st["pin_ev"].data_ptr():
+        st["pin_ev"][: n * 16].numpy()[:] = ev_bytes
+    st["pin_off"].numpy()[:] = np.ascontiguousarray(stream_offsets, dtype=np.uint64).view(np.int64)
+    with torch.cuda.device(dev):
+        st["dev_ev"][: n * 16].copy_(st["pin_ev"][: n * 16], non_blocking=True)
+        st["dev_off"].copy_(st["pin_off"], non_blocking=True)
+        st["pair"] = argus_pair_intervals(st["dev_ev"][: n * 16], st["dev_off"], num_regions, out=st["pair"],
+                                          ambig_capacity=max(n // 64, 4096) if st["pair"] is None else None)
+        p = st["pair"]
+        st["agg"] = argus_aggregate(p.intervals, p.interval_offsets, p.ambig, p.ambig_offsets, warps_per_cta,
+                                    st["cta_sm"], num_sms, num_regions, out=st["agg"])
+        a = st["agg"]
+        tables = {lv: a.table_numpy(lv) for lv in ("kernel", "sm", "cta")}
+        ioffs = p.interval_offsets.cpu().numpy().view(np.uint64)
+        status = p.fetch_status()
+    return tables, ioffs, status

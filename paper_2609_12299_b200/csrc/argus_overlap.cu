@@ -1,0 +1,297 @@
+// argus_overlap.cu — argus_overlap: per-SM overlap time of producer/consumer region pairs.
+//
+// Segment = (pair k, SM m, role) with role 0 = producer, 1 = consumer.
+//   k_ov_count   : spans selected per segment
+//   k_ov_scan    : segment bases; capacity check
+//   k_ov_scatter : spans (start, end) copied into their segment (order irrelevant)
+//   k_ov_sort    : one CTA per segment: sort by (start, end); then turn the sorted spans into the
+//                  disjoint pieces of their union, piece i = [max(start_i, E_{i-1}), E_i) with
+//                  E_i = max end of spans 0..i, and the running length before each piece
+//   k_ov_measure : one CTA per (k, m): |U_P|, |U_C|, and |U_P ∩ U_C| = sum over producer pieces of
+//                  F_C(b) - F_C(a), F_C(t) = covered length of U_C before t (binary search in C pieces)
+#include "argus_common.cuh"
+
+namespace {
+
+constexpr int kOvThreads = 1024;
+constexpr u32 kMaxPairs = 256;
+
+struct OvArgs {
+  const argus_interval_t* intervals;
+  const u64* interval_offsets;
+  u32 num_streams, warps_per_cta, num_sms, num_pairs;
+  const u32* cta_sm;
+  const u32* pairs;
+  argus_overlap_t* out;
+  argus_status_t* status;
+  u64* seg_count;   // [nseg]     (zeroed)
+  u64* seg_cursor;  // [nseg]     (zeroed)
+  u64* seg_base;    // [nseg + 1]
+  ulonglong2* spans;  // [capacity] (start, end) -> after k_ov_sort (piece begin, piece end)
+  u64* cum;           // [capacity] covered length before piece i within its segment
+  u64 capacity;
+  u32 nseg;
+};
+
+__global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatter) {
+  __shared__ u32 sh_pairs[2 * kMaxPairs];
+  for (u32 i = threadIdx.x; i < 2 * a.num_pairs; i += blockDim.x) sh_pairs[i] = a.pairs[i];
+  __syncthreads();
+  if (scatter && a.status->code != 0) return;
+  for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
+    const u32 m = a.cta_sm[s / a.warps_per_cta];
+    if (m >= a.num_sms) {
+      if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
+      continue;
+    }
+    const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
+    if (hi < lo) {
+      if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
+      continue;
+    }
+    for (u64 i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+      const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
+      const uint4 q0 = __ldg(p), q1 = __ldg(p + 1);
+      const u64 t0 = (u64)q0.x | ((u64)q0.y << 32);
+      const u64 incl = (u64)q0.z | ((u64)q0.w << 32);
+      const u32 region = q1.z;
+      if (incl == 0) continue;
+      for (u32 k = 0; k < a.num_pairs; ++k) {
+#pragma unroll
+        for (u32 role = 0; role < 2; ++role) {
+          if (sh_pairs[2 * k + role] != region) continue;
+          const u32 seg = (k * a.num_sms + m) * 2 + role;
+          if (!scatter) {
+            atomicAdd(&a.seg_count[seg], 1ull);
+          } else {
+            const u64 slot = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], 1ull);
+            if (slot < a.capacity) a.spans[slot] = make_ulonglong2(t0, t0 + incl);
+          }
+        }
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kOvThreads) k_ov_scan(OvArgs a) {
+  __shared__ u64 sh[33];
+  u64 carry = 0;
+  for (u32 g0 = 0; g0 < a.nseg; g0 += kOvThreads) {
+    const u32 g = g0 + threadIdx.x;
+    const u64 c = g < a.nseg ? a.seg_count[g] : 0;
+    u64 total;
+    const u64 ex = argus_block_exclusive_scan<u64>(c, sh, &total);
+    if (g < a.nseg) a.seg_base[g] = carry + ex;
+    carry += total;
+  }
+  if (threadIdx.x == 0) {
+    a.seg_base[a.nseg] = carry;
+    if (carry > a.capacity) {
+      argus_set_error(a.status, ARGUS_ERR_CAPACITY, 0, carry);
+      a.status->intervals_required = carry;
+    }
+  }
+}
+
+__device__ __forceinline__ bool span_less(const ulonglong2& x, const ulonglong2& y) {
+  return x.x < y.x || (x.x == y.x && x.y < y.y);
+}
+
+__device__ __forceinline__ void cmp_swap(ulonglong2* d, u64 i, u64 l) {
+  const ulonglong2 x = d[i], y = d[l];
+  if (span_less(y, x)) { d[i] = y; d[l] = x; }
+}
+
+__global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
+  __shared__ u64 sh[33];
+  __shared__ u64 sh_carry_e, sh_carry_len;
+  if (a.status->code != 0) return;
+  const u32 seg = blockIdx.x;
+  const u64 base = a.seg_base[seg];
+  const u64 n = a.seg_base[seg + 1] - base;
+  if (n == 0) return;
+  ulonglong2* d = a.spans + base;
+  u64 p = 1;
+  while (p < n) p <<= 1;
+  // bitonic network whose comparators all sort ascending; slots >= n act as +infinity and never move
+  for (u64 k = 2; k <= p; k <<= 1) {
+    for (u64 i = threadIdx.x; i < p; i += blockDim.x) {
+      const u64 l = i ^ (k - 1);
+      if (l > i && l < n) cmp_swap(d, i, l);
+    }
+    __syncthreads();
+    for (u64 j = k >> 2; j > 0; j >>= 1) {
+      for (u64 i = threadIdx.x; i < p; i += blockDim.x) {
+        const u64 l = i ^ j;
+        if (l > i && l < n) cmp_swap(d, i, l);
+      }
+      __syncthreads();
+    }
+  }
+  // pieces of the union and running covered length
+  if (threadIdx.x == 0) { sh_carry_e = 0; sh_carry_len = 0; }
+  __syncthreads();
+  const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (u64 i0 = 0; i0 < n; i0 += blockDim.x) {
+    const u64 i = i0 + threadIdx.x;
+    const bool live = i < n;
+    const ulonglong2 sp = live ? d[i] : make_ulonglong2(0, 0);
+    // inclusive prefix max of span ends (0 is the identity: ends are > starts >= 0)
+    u64 e = live ? sp.y : 0;
+#pragma unroll
+    for (int dd = 1; dd < 32; dd <<= 1) {
+      const u64 o = __shfl_up_sync(0xffffffffu, e, dd);
+      if (lane >= (u32)dd && o > e) e = o;
+    }
+    if (lane == 31) sh[warp] = e;
+    __syncthreads();
+    if (warp == 0) {
+      u64 w = sh[lane];
+#pragma unroll
+      for (int dd = 1; dd < 32; dd <<= 1) {
+        const u64 o = __shfl_up_sync(0xffffffffu, w, dd);
+        if (lane >= (u32)dd && o > w) w = o;
+      }
+      sh[lane] = w;
+    }
+    __syncthreads();
+    const u64 carry_e = sh_carry_e;
+    u64 before = carry_e;  // max end of all earlier spans
+    if (warp > 0 && sh[warp - 1] > before) before = sh[warp - 1];
+    {
+      const u64 own_excl = __shfl_up_sync(0xffffffffu, e, 1);
+      if (lane > 0 && own_excl > before) before = own_excl;
+    }
+    u64 e_incl = e > before ? e : before;
+    const u64 pa = sp.x > before ? sp.x : before;
+    const u64 pb = e_incl > pa ? e_incl : pa;
+    const u64 len = live ? pb - pa : 0;
+    __syncthreads();
+    u64 total;
+    const u64 ex = argus_block_exclusive_scan<u64>(len, sh, &total);
+    const u64 carry_len = sh_carry_len;
+    if (live) {
+      d[i] = make_ulonglong2(pa, pb);
+      a.cum[base + i] = carry_len + ex;
+    }
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) {
+      sh_carry_e = e_incl > carry_e ? e_incl : carry_e;
+      sh_carry_len = carry_len + total;
+    }
+    __syncthreads();
+  }
+}
+
+// covered length of the pieces [pc, cum) of one segment strictly before time t
+__device__ __forceinline__ u64 covered_before(const ulonglong2* pc, const u64* cum, u64 n, u64 t) {
+  // number of pieces whose begin is < t
+  u64 lo = 0, hi = n;
+  while (lo < hi) {
+    const u64 mid = lo + ((hi - lo) >> 1);
+    if (pc[mid].x < t) lo = mid + 1; else hi = mid;
+  }
+  if (lo == 0) return 0;
+  const ulonglong2 last = pc[lo - 1];
+  const u64 upto = t < last.y ? t : last.y;
+  return cum[lo - 1] + (upto - last.x);
+}
+
+__global__ void __launch_bounds__(256) k_ov_measure(OvArgs a) {
+  __shared__ u64 sh[8];
+  if (a.status->code != 0) return;
+  const u32 km = blockIdx.x;  // k * M + m
+  const u64 bp = a.seg_base[2 * km], bc = a.seg_base[2 * km + 1], be = a.seg_base[2 * km + 2];
+  const u64 np = bc - bp, nc = be - bc;
+  const ulonglong2* pp = a.spans + bp;
+  const ulonglong2* pc = a.spans + bc;
+  const u64* cum_c = a.cum + bc;
+  u64 acc = 0;
+  if (nc) {
+    for (u64 i = threadIdx.x; i < np; i += blockDim.x) {
+      const ulonglong2 piece = pp[i];
+      if (piece.y > piece.x) acc += covered_before(pc, cum_c, nc, piece.y) - covered_before(pc, cum_c, nc, piece.x);
+    }
+  }
+#pragma unroll
+  for (int dd = 16; dd > 0; dd >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, dd);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u64 both = 0;
+    for (u32 w = 0; w < (blockDim.x >> 5); ++w) both += sh[w];
+    const u64 p_ns = np ? a.cum[bp + np - 1] + (pp[np - 1].y - pp[np - 1].x) : 0;
+    const u64 c_ns = nc ? a.cum[bc + nc - 1] + (pc[nc - 1].y - pc[nc - 1].x) : 0;
+    argus_overlap_t o;
+    o.overlap_ns = both; o.producer_ns = p_ns; o.consumer_ns = c_ns; o.either_ns = p_ns + c_ns - both;
+    a.out[km] = o;
+  }
+}
+
+struct OvLayout { size_t seg_count, seg_cursor, seg_base, spans, total_fixed; };
+
+OvLayout ov_layout(uint32_t nseg) {
+  OvLayout L;
+  size_t o = 0;
+  L.seg_count = o; o += argus_align_up((size_t)nseg * 8, 256);
+  L.seg_cursor = o; o += argus_align_up((size_t)nseg * 8, 256);
+  L.seg_base = o; o += argus_align_up(((size_t)nseg + 1) * 8, 256);
+  L.spans = o;
+  L.total_fixed = o;
+  return L;
+}
+
+}  // namespace
+
+extern "C" size_t argus_overlap_workspace_bytes(uint64_t max_intervals, uint32_t /*num_streams*/, uint32_t num_pairs,
+                                                uint32_t num_sms) {
+  const OvLayout L = ov_layout(num_pairs * num_sms * 2);
+  // worst case: every interval selected in both roles of every pair; 24 bytes per selected span
+  return L.total_fixed + argus_align_up((size_t)max_intervals * 2 * num_pairs * 24 + 256, 256);
+}
+
+extern "C" int argus_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                             uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                             const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!interval_offsets || !cta_sm || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
+  if (warps_per_cta == 0 || num_streams % warps_per_cta != 0 || num_sms == 0) return ARGUS_ERR_INVALID_ARG;
+  if (num_pairs > kMaxPairs || (num_pairs && (!pairs || !out))) return ARGUS_ERR_INVALID_ARG;
+  if ((max_intervals && !intervals) || ((uintptr_t)intervals & 15) || ((uintptr_t)workspace & 255) || ((uintptr_t)out & 7))
+    return ARGUS_ERR_INVALID_ARG;
+  if ((uint64_t)num_pairs * num_sms * 2 > 0x7fffffffull) return ARGUS_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
+  if (num_pairs == 0) return ARGUS_OK;
+  const u32 nseg = num_pairs * num_sms * 2;
+  const OvLayout L = ov_layout(nseg);
+  if (workspace_bytes < L.total_fixed + 256) return ARGUS_ERR_WORKSPACE;
+  char* ws = (char*)workspace;
+  OvArgs a;
+  a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets; a.num_streams = num_streams;
+  a.warps_per_cta = warps_per_cta; a.num_sms = num_sms; a.num_pairs = num_pairs; a.cta_sm = cta_sm; a.pairs = pairs;
+  a.out = out; a.status = status;
+  a.seg_count = (u64*)(ws + L.seg_count); a.seg_cursor = (u64*)(ws + L.seg_cursor); a.seg_base = (u64*)(ws + L.seg_base);
+  a.capacity = (workspace_bytes - L.total_fixed) / 24;
+  a.spans = (ulonglong2*)(ws + L.spans);
+  a.cum = (u64*)(ws + L.spans + argus_align_up((size_t)a.capacity * 16, 16));
+  a.nseg = nseg;
+  ARGUS_CUDA_TRY(cudaMemsetAsync(ws, 0, L.seg_base, stream));
+  ARGUS_CUDA_TRY(cudaMemsetAsync(out, 0, (size_t)num_pairs * num_sms * sizeof(argus_overlap_t), stream));
+  if (num_streams) {
+    k_ov_count_or_scatter<<<num_streams < 2368 ? num_streams : 2368, 256, 0, stream>>>(a, 0);
+    ARGUS_CHECK_LAUNCH();
+  }
+  k_ov_scan<<<1, kOvThreads, 0, stream>>>(a);
+  ARGUS_CHECK_LAUNCH();
+  if (num_streams) {
+    k_ov_count_or_scatter<<<num_streams < 2368 ? num_streams : 2368, 256, 0, stream>>>(a, 1);
+    ARGUS_CHECK_LAUNCH();
+  }
+  k_ov_sort<<<nseg, kOvThreads, 0, stream>>>(a);
+  ARGUS_CHECK_LAUNCH();
+  k_ov_measure<<<nseg / 2, 256, 0, stream>>>(a);
+  ARGUS_CHECK_LAUNCH();
+  (void)max_intervals;
+  return ARGUS_OK;
+}

@@ -1,0 +1,247 @@
+"""Parity of the CUDA path (through the C-ABI) against the CPU oracle: bit-exact, element by element.
+Everything here needs a GPU."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_12299_b200 as argus
+from helpers import load_example, make_events, random_wellformed
+from paper_2609_12299_b200 import tracegen as tg
+from paper_2609_12299_b200.binding import KERNEL_THREAD_PER_STREAM, KERNEL_TILED
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+KERNELS = [KERNEL_THREAD_PER_STREAM, KERNEL_TILED]
+
+
+def to_dev(ev, offs):
+    d_ev = torch.from_numpy(np.ascontiguousarray(ev).view(np.uint8).reshape(-1).copy()).to(DEV)
+    d_off = torch.from_numpy(np.ascontiguousarray(offs, dtype=np.uint64).view(np.int64).copy()).to(DEV)
+    return d_ev, d_off
+
+
+def run_pair(ev, offs, R, kernel, **kw):
+    d_ev, d_off = to_dev(ev, offs)
+    pr = argus.argus_pair_intervals(d_ev, d_off, R, kernel=kernel, **kw)
+    return pr, pr.fetch_status()
+
+
+def assert_pair_matches(ev, offs, R, kernel, **kw):
+    pr, st = run_pair(ev, offs, R, kernel, **kw)
+    rc, o_iv, o_ioffs, o_am, o_aoffs, o_st = oracle.pair(ev, offs, R)
+    assert rc == 0 and int(o_st["code"]) == 0
+    assert int(st["code"]) == 0, f"device status {st}"
+    assert np.array_equal(pr.interval_offsets.cpu().numpy().view(np.uint64), o_ioffs)
+    assert np.array_equal(pr.ambig_offsets.cpu().numpy().view(np.uint64), o_aoffs)
+    g_iv, g_am = pr.intervals_numpy(), pr.ambig_numpy()
+    if g_iv.tobytes() != o_iv.tobytes():
+        bad = np.nonzero(g_iv != o_iv)[0]
+        raise AssertionError(f"{len(bad)} intervals differ; first at {bad[0]}: gpu {g_iv[bad[0]]} oracle {o_iv[bad[0]]}")
+    if g_am.tobytes() != o_am.tobytes():
+        bad = np.nonzero(g_am != o_am)[0]
+        raise AssertionError(f"{len(bad)} ambiguity records differ; first at {bad[0]}: gpu {g_am[bad[0]]} oracle {o_am[bad[0]]}")
+    for f in ("intervals_required", "ambig_required", "n_ctx_mismatch", "n_time_reversed", "n_child_clamped"):
+        assert int(st[f]) == int(o_st[f]), f
+    return pr, (o_iv, o_ioffs, o_am, o_aoffs)
+
+
+EXAMPLES = ["example_a_wellformed.txt", "example_b_dropped_end.txt", "example_c_dup_stray_trunc.txt",
+            "example_e_ctx_ignored.txt", "example_f_greedy.txt", "example_g_boundary.txt", "example_h_flags.txt"]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("name", EXAMPLES)
+def test_hand_worked_examples(name, kernel):
+    ev, _, _ = load_example(name)
+    assert_pair_matches(ev, np.array([0, len(ev)], np.uint64), 8, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_tracegen_host_equals_device_and_config0(kernel):
+    spec = tg.config(0)
+    ev, offs = tg.generate_host(spec)
+    d_ev, d_off = tg.generate_cuda(spec, DEV)
+    assert d_ev.cpu().numpy().tobytes() == ev.tobytes()
+    assert np.array_equal(d_off.cpu().numpy().view(np.uint64), offs)
+    assert_pair_matches(ev, offs, spec.num_regions, kernel)
+
+
+@pytest.mark.parametrize("idx,ctas,iters", [(1, 5, 60), (2, 3, 2), (3, 2, 3), (4, 6, 80)])
+def test_tracegen_host_equals_device_scaled(idx, ctas, iters):
+    spec = tg.config(idx).scaled(ctas, iters)
+    ev, offs = tg.generate_host(spec)
+    d_ev, d_off = tg.generate_cuda(spec, DEV)
+    assert np.array_equal(d_off.cpu().numpy().view(np.uint64), offs)
+    assert d_ev.cpu().numpy().tobytes() == ev.tobytes()
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("idx,ctas,iters", [(1, 7, 300), (2, 3, 3), (3, 3, 9), (4, 9, 400)])
+def test_scaled_configs_full_pipeline(idx, ctas, iters, kernel):
+    """Pair + aggregate + overlap on scaled-down versions of configs 1-4 (several tiles per stream and a ragged tail)."""
+    spec = tg.config(idx).scaled(ctas, iters)
+    ev, offs = tg.generate_host(spec)
+    pr, (o_iv, o_ioffs, o_am, o_aoffs) = assert_pair_matches(ev, offs, spec.num_regions, kernel)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    ag = argus.argus_aggregate(pr.intervals, pr.interval_offsets, pr.ambig, pr.ambig_offsets, spec.warps_per_cta, cta_sm,
+                               spec.num_sms, spec.num_regions)
+    assert int(argus.argus_status_fetch(ag.status)["code"]) == 0
+    _, o_tabs, _ = oracle.aggregate(o_iv, o_ioffs, o_am, o_aoffs, spec.warps_per_cta, spec.cta_sm, spec.num_sms,
+                                    spec.num_regions)
+    for lv in ("warp", "cta", "sm", "kernel"):
+        assert ag.table_numpy(lv).tobytes() == o_tabs[lv].tobytes(), lv
+    pairs_np = np.concatenate([spec.overlap_pairs, spec.overlap_pairs[:, ::-1], [[0, 0]]]).astype(np.uint32)
+    pairs = torch.from_numpy(pairs_np.view(np.int32)).to(DEV)
+    ov, ov_st = argus.argus_overlap(pr.intervals, pr.interval_capacity, pr.interval_offsets, spec.warps_per_cta, cta_sm,
+                                    spec.num_sms, pairs)
+    assert int(argus.argus_status_fetch(ov_st)["code"]) == 0
+    _, o_ov, _ = oracle.overlap(o_iv, o_ioffs, spec.warps_per_cta, spec.cta_sm, spec.num_sms, pairs_np)
+    assert ov.cpu().numpy().view(argus.OVERLAP_DTYPE).reshape(o_ov.shape).tobytes() == o_ov.tobytes()
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_random_malformed_streams(kernel):
+    rng = np.random.default_rng(11)
+    evs, offs = [], [0]
+    for s in range(96):
+        n_pairs = int(rng.integers(0, 3000 if s % 7 == 0 else 200))
+        ev = random_wellformed(rng, n_pairs, 6, max_height=int(rng.integers(1, 12))) if n_pairs else make_events([])
+        mode = s % 4
+        if mode == 1 and len(ev):
+            ev = ev[rng.random(len(ev)) > 0.02]              # drop markers of either kind
+        elif mode == 2 and len(ev):
+            ev = np.repeat(ev, 1 + (rng.random(len(ev)) < 0.02))  # duplicate markers
+        elif mode == 3 and len(ev) > 2:
+            ev = ev[int(rng.integers(0, len(ev))):]            # cut the head: leading unmatched ends
+            if rng.random() < 0.5:
+                ev = ev.copy()
+                ev["ts"][rng.random(len(ev)) < 0.05] -= 500   # timestamps that run backwards
+                ev["ctx"][rng.random(len(ev)) < 0.05] += 1
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    ev = np.concatenate(evs)
+    assert_pair_matches(ev, np.array(offs, np.uint64), 6, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_deep_and_adversarial_streams(kernel):
+    rows = [(i, "B", i % 3, 0) for i in range(64)] + [(100 + i, "E", (63 - i) % 3, 0) for i in range(64)]
+    deep = make_events(rows)                                           # full depth, well formed
+    only_ends = make_events([(i, "E", i % 4, 1) for i in range(5000)])  # every marker ambiguous
+    only_begins = make_events([(i, "B", 0, 1) for i in range(64)])
+    sawtooth = make_events([(i, "BE"[i % 2], 0, i) for i in range(6001)])  # ctx mismatch on every interval, odd length
+    wide = make_events([(7 * i, "B", 1, 0) for i in range(40)] + [(1000, "E", 0, 0)] +
+                       [(2000 + i, "E", 1, 0) for i in range(40)])    # stray end under a deep stack
+    evs = [deep, only_ends, only_begins, sawtooth, wide, make_events([])]
+    offs = np.cumsum([0] + [len(e) for e in evs]).astype(np.uint64)
+    assert_pair_matches(np.concatenate(evs), offs, 4, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_edges_and_error_codes(kernel):
+    ev = make_events([(1, "B", 0, 0), (2, "E", 0, 0), (5, "B", 1, 3), (9, "E", 1, 3)])
+    # offsets that do not start at zero, empty streams
+    assert_pair_matches(ev, np.array([2, 2, 4, 4], np.uint64), 2, kernel)
+    # no events at all, but streams exist
+    assert_pair_matches(ev[:0], np.array([0, 0, 0], np.uint64), 2, kernel)
+    # bad region id
+    pr, st = run_pair(ev, np.array([0, 4], np.uint64), 1, kernel)
+    assert int(st["code"]) == 6 and int(st["bad_stream"]) == 0 and int(st["bad_event"]) == 2
+    # 65 open frames
+    deep = make_events([(i, "B", 0, 0) for i in range(65)])
+    pr, st = run_pair(deep, np.array([0, 65], np.uint64), 1, kernel)
+    assert int(st["code"]) == 5 and int(st["bad_event"]) == 64
+    # interval capacity too small: required count reported
+    many = make_events([(i, "BE"[i % 2], 0, 0) for i in range(200)])
+    pr, st = run_pair(many, np.array([0, 200], np.uint64), 1, kernel, interval_capacity=10)
+    assert int(st["code"]) == 4 and int(st["intervals_required"]) == 100
+    # ambiguity capacity too small
+    ends = make_events([(i, "E", 0, 0) for i in range(100)])
+    pr, st = run_pair(ends, np.array([0, 100], np.uint64), 1, kernel, ambig_capacity=7)
+    assert int(st["code"]) == 4 and int(st["ambig_required"]) == 100
+    # decreasing offsets, offsets beyond the buffer
+    pr, st = run_pair(ev, np.array([0, 3, 2], np.uint64), 2, kernel)
+    assert int(st["code"]) == 7
+    pr, st = run_pair(ev, np.array([0, 9], np.uint64), 2, kernel)
+    assert int(st["code"]) == 7
+    # the context stays usable after every error
+    assert_pair_matches(ev, np.array([0, 4], np.uint64), 2, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_exact_capacity_with_malformed_trace(kernel):
+    """Capacity equal to the true interval count: provisional positions overflow, the second pass fixes them."""
+    spec = tg.config(4).scaled(3, 120)
+    ev, offs = tg.generate_host(spec)
+    _, o_iv, _, o_am, _, _ = oracle.pair(ev, offs, spec.num_regions)
+    assert_pair_matches(ev, offs, spec.num_regions, kernel, interval_capacity=len(o_iv), ambig_capacity=len(o_am))
+
+
+def test_invalid_arguments_raise():
+    ev = make_events([(1, "B", 0, 0), (2, "E", 0, 0)])
+    d_ev, d_off = to_dev(ev, np.array([0, 2], np.uint64))
+    with pytest.raises(argus.ArgusError):
+        argus.argus_pair_intervals(d_ev, d_off, 0)
+    with pytest.raises(argus.ArgusError):
+        argus.argus_pair_intervals(d_ev, d_off, 70000)
+    pr = argus.argus_pair_intervals(d_ev, d_off, 1)
+    cta_sm = torch.zeros(1, dtype=torch.int32, device=DEV)
+    with pytest.raises(argus.ArgusError):
+        argus.argus_aggregate(pr.intervals, pr.interval_offsets, None, None, 2, cta_sm, 1, 1)  # S % W != 0
+    small_ws = torch.empty(256, dtype=torch.uint8, device=DEV)
+    with pytest.raises(argus.ArgusError) as e:
+        argus.argus_pair_intervals(d_ev, d_off, 1, out=argus.PairResult(pr.intervals, pr.interval_offsets, pr.ambig,
+                                   pr.ambig_offsets, pr.status, 1, 2, small_ws))
+    assert e.value.code == 2
+
+
+def test_aggregate_large_region_count_and_null_tables():
+    """num_regions too large for a shared-memory table (global-row path) and nullable outputs."""
+    rng = np.random.default_rng(5)
+    R = 600
+    evs, offs = [], [0]
+    for s in range(8):
+        ev = random_wellformed(rng, 500, R, max_height=5)
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    ev, offs = np.concatenate(evs), np.array(offs, np.uint64)
+    pr, (o_iv, o_ioffs, o_am, o_aoffs) = assert_pair_matches(ev, offs, R, KERNEL_THREAD_PER_STREAM)
+    cta_sm_np = np.array([1, 0, 1, 2], np.uint32)
+    cta_sm = torch.from_numpy(cta_sm_np.view(np.int32)).to(DEV)
+    _, o_tabs, _ = oracle.aggregate(o_iv, o_ioffs, o_am, o_aoffs, 2, cta_sm_np, 3, R)
+    ag = argus.argus_aggregate(pr.intervals, pr.interval_offsets, pr.ambig, pr.ambig_offsets, 2, cta_sm, 3, R)
+    for lv in ("warp", "cta", "sm", "kernel"):
+        assert ag.table_numpy(lv).tobytes() == o_tabs[lv].tobytes(), lv
+    ag2 = argus.argus_aggregate(pr.intervals, pr.interval_offsets, None, None, 2, cta_sm, 3, R, levels=("kernel",))
+    assert ag2.table_numpy("kernel").tobytes() == o_tabs["kernel"].tobytes()
+    ag3 = argus.argus_aggregate(pr.intervals, pr.interval_offsets, None, None, 2, cta_sm, 3, R, levels=("sm",))
+    assert ag3.table_numpy("sm").tobytes() == o_tabs["sm"].tobytes()
+
+
+def test_overlap_random_spans_and_capacity():
+    rng = np.random.default_rng(8)
+    S, W, M, R = 24, 3, 4, 5
+    cta_sm_np = rng.integers(0, M, S // W).astype(np.uint32)
+    rows = []
+    for s in range(S):
+        for _ in range(int(rng.integers(0, 3000 if s % 5 == 0 else 50))):
+            rows.append((s, int(rng.integers(0, R)), int(rng.integers(0, 1 << 40)) + (1 << 60), int(rng.integers(0, 1 << 30))))
+    rows.sort(key=lambda r: r[0])
+    iv = np.zeros(len(rows), argus.INTERVAL_DTYPE)
+    arr = np.array(rows, dtype=np.uint64)
+    iv["stream"], iv["region"], iv["t_begin"], iv["inclusive"] = arr[:, 0], arr[:, 1], arr[:, 2], arr[:, 3]
+    ioffs = np.zeros(S + 1, np.uint64)
+    ioffs[1:] = np.cumsum(np.bincount(arr[:, 0].astype(np.int64), minlength=S))
+    pairs_np = np.array([(0, 1), (1, 0), (2, 2), (3, 4), (4, 0)], np.uint32)
+    _, o_ov, _ = oracle.overlap(iv, ioffs, W, cta_sm_np, M, pairs_np)
+    d_iv = torch.from_numpy(iv.view(np.uint8).reshape(-1).copy()).to(DEV)
+    d_off = torch.from_numpy(ioffs.view(np.int64).copy()).to(DEV)
+    cta_sm = torch.from_numpy(cta_sm_np.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(pairs_np.view(np.int32)).to(DEV)
+    ov, st = argus.argus_overlap(d_iv, len(iv), d_off, W, cta_sm, M, pairs)
+    assert int(argus.argus_status_fetch(st)["code"]) == 0
+    assert ov.cpu().numpy().view(argus.OVERLAP_DTYPE).reshape(o_ov.shape).tobytes() == o_ov.tobytes()
+    # a workspace too small for the selected spans is reported, not overrun
+    ov, st = argus.argus_overlap(d_iv, len(iv), d_off, W, cta_sm, M, pairs, workspace_bytes=64 * 1024)
+    assert int(argus.argus_status_fetch(st)["code"]) == 4

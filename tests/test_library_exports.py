@@ -1,0 +1,52 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import paper_2609_12299_b200 as argus
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "argus.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(argus_[a-z_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported():
+    names = _declared_functions()
+    assert {"argus_pair_intervals", "argus_aggregate", "argus_overlap", "argus_status_fetch", "argus_strerror",
+            "argus_version", "argus_pair_workspace_bytes", "argus_aggregate_workspace_bytes",
+            "argus_overlap_workspace_bytes"} <= set(names)
+    lib = ctypes.CDLL(argus.library_path())
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in argus.h but not exported"
+
+
+def test_host_only_calls():
+    assert argus.argus_version() >= 100
+    assert argus.argus_strerror(0) == "ok"
+    assert "capacity" in argus.argus_strerror(4)
+    assert argus.argus_strerror(12345) == "unknown error code"
+    a = argus.argus_pair_workspace_bytes(1 << 20, 64, 1 << 10)
+    b = argus.argus_pair_workspace_bytes(1 << 21, 64, 1 << 10)
+    assert 0 < a < b and a % 256 == 0
+    assert argus.argus_aggregate_workspace_bytes(1000, 16, 8) >= 2 * 16 * 8 * 576
+    assert argus.argus_overlap_workspace_bytes(1000, 16, 2, 4) >= 1000 * 2 * 2 * 24
+
+
+def test_struct_sizes_match_header():
+    assert (argus.EVENT_DTYPE.itemsize, argus.INTERVAL_DTYPE.itemsize, argus.AMBIG_DTYPE.itemsize,
+            argus.AGG_DTYPE.itemsize, argus.OVERLAP_DTYPE.itemsize, argus.STATUS_DTYPE.itemsize) == (16, 48, 32, 576, 32, 64)
+
+
+def test_host_argument_validation_needs_no_gpu():
+    lib = argus.load_library()
+    # null pointers and bad sizes are rejected on the host before any CUDA call
+    rc = lib.argus_pair_intervals(None, 0, None, 0, 1, None, 0, None, None, 0, None, None, None, 0, None)
+    assert rc == 1
+    rc = lib.argus_aggregate(None, None, None, None, 4, 0, None, 1, 1, None, None, None, None, None, None, 0, None)
+    assert rc == 1
+    rc = lib.argus_overlap(None, 0, None, 4, 0, None, 1, None, 0, None, None, None, 0, None)
+    assert rc == 1
