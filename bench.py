@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the region-trace hot path: marker events/s for one pass of
+pair -> aggregate -> overlap over one synthetic trace, and the HBM roofline fraction of the
+dominant (pairing) kernel.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload I]
+
+One process per GPU (torchrun for N > 1); every rank processes its own trace of the same shape
+(weak scaling, no data-path collective). Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "marker events/sec (pair+aggregate+overlap, whole hot path)"
+UNIT = "events/s"
+ALG_BYTES_PER_EVENT = 40.0  # 16 B event read + 48 B interval written per 2 events
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock, power and clock-event reasons of one GPU through NVML while running."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, torch_device):
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            props = torch.cuda.get_device_properties(torch_device)
+            h = None
+            uuid = getattr(props, "uuid", None)
+            if uuid is not None:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+                except Exception:
+                    try:
+                        h = pynvml.nvmlDeviceGetHandleByUUID("GPU-" + str(uuid))
+                    except Exception:
+                        h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(torch_device.index or 0)
+            self._h = h
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # NVML missing: report that clocks were not sampled
+            self.error = repr(e)
+
+    def _loop(self):
+        nv, h = self._nv, self._h
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0,
+                    "note": getattr(self, "error", "no samples")}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples), "power_w_max": max(self.power) if self.power else None}
+
+
+def oracle_step(oracle, ev, offs, spec, cta_sm, num_sms):
+    rc, iv, ioffs, am, aoffs, st = oracle.pair(ev, offs, spec.num_regions, ambig_cap=max(len(ev) // 64, 4096))
+    assert rc == 0 and int(st["code"]) == 0
+    rc, tabs, st = oracle.aggregate(iv, ioffs, am, aoffs, spec.warps_per_cta, cta_sm, num_sms, spec.num_regions)
+    assert rc == 0
+    rc, ov, st = oracle.overlap(iv, ioffs, spec.warps_per_cta, cta_sm, num_sms, spec.overlap_pairs)
+    assert rc == 0
+    return tabs, ov
+
+
+def oracle_sample(tg, spec, num_ctas):
+    """Host copy of the first `num_ctas` CTAs of the workload (bit-identical to the device trace)."""
+    offs = tg.host_offsets(spec)
+    S = num_ctas * spec.warps_per_cta
+    ev = tg.host_streams(spec, offs, 0, S)
+    sub = (offs[: S + 1] - offs[0]).astype(np.uint64)
+    cta_sm = spec.cta_sm[:num_ctas].copy()
+    return ev, sub, cta_sm, int(cta_sm.max()) + 1
+
+
+def run_reference(args, spec, tg):
+    """The oracle as it stands, on the host cores, on a bounded sample of the workload per step."""
+    import oracle
+    oracle.build()
+    num_ctas = 1
+    ev, offs, cta_sm, num_sms = oracle_sample(tg, spec, num_ctas)
+    for _ in range(args.warmup):
+        oracle_step(oracle, ev, offs, spec, cta_sm, num_sms)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, ev, offs, spec, cta_sm, num_sms)
+    dt = time.perf_counter() - t0
+    value = len(ev) * args.steps / dt
+    sample = f"first {num_ctas} CTA(s) = {num_ctas * spec.warps_per_cta} streams, {len(ev)} events per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": spec.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, help="config index 0..4 (default 3: decode megakernel, the largest)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-ctas", type=int, default=6, help="CTAs of the workload the CPU baseline is timed on")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2609_12299_b200 import tracegen as tg
+    spec = tg.config(args.workload)
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, spec, tg)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_12299_b200 as argus
+
+    argus.load_library()  # raises if the CUDA library was not built: there is no fallback
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    # every rank its own trace of the same shape (weak scaling)
+    from dataclasses import replace
+    spec = replace(spec, seed=spec.seed + 1000 * rank)
+    d_ev, d_off = tg.generate_cuda(spec, dev)
+    n_events = d_ev.numel() // 16
+    S = spec.num_streams
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(dev)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(dev)
+    icap = n_events // 2
+    acap = max(n_events // 64, 4096)
+    ov_ws = torch.empty(min(argus.argus_overlap_workspace_bytes(icap, S, len(spec.overlap_pairs), spec.num_sms),
+                            2 << 30), dtype=torch.uint8, device=dev)
+    state = {"pair": None, "agg": None}
+
+    def step():
+        state["pair"] = p = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions, interval_capacity=icap,
+                                                       ambig_capacity=acap, out=state["pair"])
+        state["agg"] = argus.argus_aggregate(p.intervals, p.interval_offsets, p.ambig, p.ambig_offsets,
+                                             spec.warps_per_cta, cta_sm, spec.num_sms, spec.num_regions, out=state["agg"])
+        state["ov"] = argus.argus_overlap(p.intervals, icap, p.interval_offsets, spec.warps_per_cta, cta_sm, spec.num_sms,
+                                          pairs, workspace=ov_ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    st = state["pair"].fetch_status()
+    if int(st["code"]) != 0:
+        raise RuntimeError(f"device status after warm-up: {st}")
+
+    sampler = ClockSampler(dev)
+    argus.argus_profile_read()
+    argus.argus_profile_enable(True)
+    launches0 = argus.argus_launch_count()
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    sampler.stop()
+    launches = argus.argus_launch_count() - launches0
+    argus.argus_profile_enable(False)
+    prof_ms, prof_n = argus.argus_profile_read()
+    ms_total = e0.elapsed_time(e1)
+    for name in ("pair", "agg"):
+        code = int(argus.argus_status_fetch(state[name].status)["code"])
+        if code != 0:
+            raise RuntimeError(f"device status {code} in {name} after the timed region")
+    if int(argus.argus_status_fetch(state["ov"][1])["code"]) != 0:
+        raise RuntimeError("device status in overlap after the timed region")
+
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = n_events * world / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel (the pairing kernel): algorithmic bytes / its own launch time
+    peak, peak_src = load_peaks()
+    pair_ms = prof_ms["pair"] / max(prof_n["pair"], 1)
+    achieved = ALG_BYTES_PER_EVENT * n_events / (pair_ms * 1e-3) / 1e9 if pair_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "pairing kernel of argus_pair_intervals", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "peak_source": peak_src,
+                "traffic": None, "ms_per_launch": pair_ms, "algorithmic_bytes_per_event": ALG_BYTES_PER_EVENT,
+                "pipeline_frac": ALG_BYTES_PER_EVENT * n_events / (ms_per_step * 1e-3) / 1e9 / peak}
+    kernel_ms = {k: prof_ms[k] / max(prof_n[k], 1) for k in ("pair", "aggregate", "overlap")}
+
+    # end to end with HOST buffers: pinned events -> device, the three calls, result tables -> host
+    e2e = None
+    if not args.no_e2e:
+        pin_ev = torch.empty(n_events * 16, dtype=torch.uint8, pin_memory=True)
+        pin_ev.copy_(d_ev)
+        pin_off = torch.empty(S + 1, dtype=torch.int64, pin_memory=True)
+        pin_off.copy_(d_off)
+        agg = state["agg"]
+        outs = [agg.kernel, agg.sm, agg.cta, state["ov"][0], state["pair"].interval_offsets, state["pair"].status]
+        pin_out = [torch.empty(o.numel(), dtype=o.dtype, pin_memory=True) for o in outs]
+        torch.cuda.synchronize(dev)
+
+        def e2e_step():
+            d_ev.copy_(pin_ev, non_blocking=True)
+            d_off.copy_(pin_off, non_blocking=True)
+            step()
+            for o, p in zip(outs, pin_out):
+                p.copy_(o.reshape(-1), non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        assert int(pin_out[-1].numpy().view(argus.STATUS_DTYPE)[0]["code"]) == 0
+        e2e = {"value": n_events * world / (ms / args.e2e_steps * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(pin_ev.numel() + pin_off.numel() * 8),
+               "d2h_bytes_per_step": int(sum(p.numel() * p.element_size() for p in pin_out)),
+               "steps": args.e2e_steps, "ms_per_step": ms / args.e2e_steps}
+        del pin_ev
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        ev, offs, csm, nsm = oracle_sample(tg, spec, args.cpu_ctas)
+        t0 = time.perf_counter()
+        oracle_step(oracle, ev, offs, spec, csm, nsm)
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": len(ev) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "host_cores": os.cpu_count(),
+                        "seconds": dt,
+                        "sample": f"first {args.cpu_ctas} CTAs = {args.cpu_ctas * spec.warps_per_cta} streams, {len(ev)} events, one pass"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
+            "data": "synthetic",
+            "config": {"workload": spec.name, "events_per_gpu": n_events, "streams": S, "regions": spec.num_regions,
+                       "input_bytes_per_gpu": n_events * 16, "l2": "inputs (>= 1 GB) are larger than the 126 MB L2",
+                       "step": "argus_pair_intervals + argus_aggregate + argus_overlap on one trace per GPU"},
+            "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "kernel_ms": kernel_ms,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -254,6 +254,17 @@ const char* argus_strerror(int code);
 /* Library version: major * 10000 + minor * 100 + patch. */
 int argus_version(void);
 
+/* Measurement helpers (host-side bookkeeping only; they change no result).
+ * argus_launch_count: kernels this library has launched since it was loaded.
+ * argus_profile_enable(1): from now on each operation records a CUDA event pair on its stream
+ * around its dominant kernel (slot 0 = pairing kernel of argus_pair_intervals, 1 = per-stream
+ * accumulation kernel of argus_aggregate, 2 = sort kernel of argus_overlap, 3 = reserved).
+ * argus_profile_read: waits for the recorded events, writes per slot the summed kernel time in
+ * milliseconds and the number of recorded launches (arrays of 4), and forgets them. */
+unsigned long long argus_launch_count(void);
+void argus_profile_enable(int on);
+int argus_profile_read(double* ms_total /*host [4]*/, unsigned long long* launches /*host [4]*/);
+
 #ifdef __cplusplus
 }
 #endif

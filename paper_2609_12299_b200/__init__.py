@@ -7,11 +7,13 @@ memory and streams. There is no CPU fallback: if the library has not been built,
 from .binding import (AGG_DTYPE, AMBIG_DTYPE, EVENT_DTYPE, INTERVAL_DTYPE, OVERLAP_DTYPE, STATUS_DTYPE, ArgusError,
                       AggregateResult, PairResult, argus_aggregate, argus_aggregate_workspace_bytes, argus_overlap,
                       argus_overlap_workspace_bytes, argus_pair_intervals, argus_pair_workspace_bytes,
-                      argus_status_fetch, argus_strerror, argus_version, library_path, load_library, pair_aggregate_host)
+                      argus_launch_count, argus_profile_enable, argus_profile_read, argus_status_fetch, argus_strerror,
+                      argus_version, library_path, load_library, pair_aggregate_host)
 
 __all__ = [
     "AGG_DTYPE", "AMBIG_DTYPE", "EVENT_DTYPE", "INTERVAL_DTYPE", "OVERLAP_DTYPE", "STATUS_DTYPE", "ArgusError",
     "AggregateResult", "PairResult", "argus_aggregate", "argus_aggregate_workspace_bytes", "argus_overlap",
     "argus_overlap_workspace_bytes", "argus_pair_intervals", "argus_pair_workspace_bytes", "argus_status_fetch",
-    "argus_strerror", "argus_version", "library_path", "load_library", "pair_aggregate_host",
+    "argus_strerror", "argus_version", "library_path", "load_library", "pair_aggregate_host", "argus_launch_count",
+    "argus_profile_enable", "argus_profile_read",
 ]

@@ -72,8 +72,33 @@ def load_library():
     lib.argus_strerror.restype = ctypes.c_char_p
     lib.argus_version.argtypes = []
     lib.argus_version.restype = ci
+    lib.argus_launch_count.argtypes = []
+    lib.argus_launch_count.restype = ctypes.c_ulonglong
+    lib.argus_profile_enable.argtypes = [ci]
+    lib.argus_profile_enable.restype = None
+    lib.argus_profile_read.argtypes = [vp, vp]
+    lib.argus_profile_read.restype = ci
     _lib = lib
     return lib
+
+
+def argus_launch_count() -> int:
+    return int(load_library().argus_launch_count())
+
+
+def argus_profile_enable(on: bool) -> None:
+    load_library().argus_profile_enable(1 if on else 0)
+
+
+def argus_profile_read():
+    """Returns ({slot: total ms}, {slot: launches}) for the slots pair / aggregate / overlap."""
+    ms = (ctypes.c_double * 4)()
+    n = (ctypes.c_ulonglong * 4)()
+    rc = load_library().argus_profile_read(ctypes.addressof(ms), ctypes.addressof(n))
+    if rc != 0:
+        raise ArgusError(rc, "argus_profile_read")
+    names = ("pair", "aggregate", "overlap", "reserved")
+    return {k: ms[i] for i, k in enumerate(names)}, {k: int(n[i]) for i, k in enumerate(names)}
 
 
 def argus_strerror(code: int) -> str:

@@ -175,8 +175,10 @@ extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t
   a.use_smem = smem <= kAggSmemLimit;
   if (a.use_smem && smem > 48 * 1024)
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 0);
   k_agg_streams<<<num_streams, kAggThreads, a.use_smem ? smem : 0, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
+  argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 1);
   if (cta_tab || sm_tab || kernel_tab) {
     k_agg_cta<<<1184, 256, 0, stream>>>(a);
     ARGUS_CHECK_LAUNCH();

@@ -23,9 +23,15 @@ static_assert(sizeof(argus_status_t) == 64, "status layout");
     if (e__ != cudaSuccess) return ARGUS_ERR_CUDA;    \
   } while (0)
 
+// host-side bookkeeping implemented in argus_api.cu
+void argus_count_launch();                                      // one more kernel launched by this library
+void argus_prof_mark(int slot, cudaStream_t stream, int end);   // CUDA events around a dominant kernel (if enabled)
+enum { ARGUS_PROF_PAIR = 0, ARGUS_PROF_AGGREGATE = 1, ARGUS_PROF_OVERLAP = 2, ARGUS_PROF_SLOTS = 4 };
+
 #define ARGUS_CHECK_LAUNCH()                                      \
   do {                                                            \
     if (cudaGetLastError() != cudaSuccess) return ARGUS_ERR_CUDA; \
+    argus_count_launch();                                         \
   } while (0)
 
 static inline size_t argus_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -288,8 +288,10 @@ extern "C" int argus_overlap(const argus_interval_t* intervals, uint64_t max_int
     k_ov_count_or_scatter<<<num_streams < 2368 ? num_streams : 2368, 256, 0, stream>>>(a, 1);
     ARGUS_CHECK_LAUNCH();
   }
+  argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 0);
   k_ov_sort<<<nseg, kOvThreads, 0, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
+  argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 1);
   k_ov_measure<<<nseg / 2, 256, 0, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   (void)max_intervals;

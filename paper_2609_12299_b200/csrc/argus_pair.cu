@@ -241,6 +241,7 @@ extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num
   for (int pass = 0; pass < 2; ++pass) {
     a.redo = pass;
     if (num_streams) {
+      if (pass == 0) argus_prof_mark(ARGUS_PROF_PAIR, stream, 0);
       if (tiled) {
         const int rc = argus_launch_pair_tiled(a, stream);
         if (rc != ARGUS_OK) return rc;
@@ -248,6 +249,7 @@ extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num
         k_pair_thread_per_stream<<<(num_streams + 127) / 128, 128, 0, stream>>>(a);
         ARGUS_CHECK_LAUNCH();
       }
+      if (pass == 0) argus_prof_mark(ARGUS_PROF_PAIR, stream, 1);
     }
     if (pass == 0) {
       k_pair_offsets<<<1, kScanThreads, 0, stream>>>(a);
