@@ -136,7 +136,7 @@ typedef struct {
   uint64_t n_ctx_mismatch;
   uint64_t n_time_reversed;
   uint64_t n_child_clamped;
-  uint64_t reserved;
+  uint64_t n_sequential_tiles; /* diagnostic: tiles the tiled kernel redid with the sequential stack */
 } argus_status_t;
 
 /* ---------------------------------------------------------------------------------------

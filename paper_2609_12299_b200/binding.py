@@ -22,7 +22,7 @@ AGG_DTYPE = np.dtype([("count", "<u8"), ("sum_incl", "<u8"), ("min_incl", "<u8")
 OVERLAP_DTYPE = np.dtype([("overlap_ns", "<u8"), ("producer_ns", "<u8"), ("consumer_ns", "<u8"), ("either_ns", "<u8")])
 STATUS_DTYPE = np.dtype([("code", "<u4"), ("bad_stream", "<u4"), ("bad_event", "<u8"), ("intervals_required", "<u8"),
                          ("ambig_required", "<u8"), ("n_ctx_mismatch", "<u8"), ("n_time_reversed", "<u8"),
-                         ("n_child_clamped", "<u8"), ("reserved", "<u8")])
+                         ("n_child_clamped", "<u8"), ("n_sequential_tiles", "<u8")])
 
 KERNEL_AUTO, KERNEL_THREAD_PER_STREAM, KERNEL_TILED = 0, 1, 2
 

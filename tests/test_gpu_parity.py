@@ -43,6 +43,7 @@ def assert_pair_matches(ev, offs, R, kernel, **kw):
         raise AssertionError(f"{len(bad)} ambiguity records differ; first at {bad[0]}: gpu {g_am[bad[0]]} oracle {o_am[bad[0]]}")
     for f in ("intervals_required", "ambig_required", "n_ctx_mismatch", "n_time_reversed", "n_child_clamped"):
         assert int(st[f]) == int(o_st[f]), f
+    pr.last_status = st
     return pr, (o_iv, o_ioffs, o_am, o_aoffs)
 
 
@@ -83,6 +84,9 @@ def test_scaled_configs_full_pipeline(idx, ctas, iters, kernel):
     spec = tg.config(idx).scaled(ctas, iters)
     ev, offs = tg.generate_host(spec)
     pr, (o_iv, o_ioffs, o_am, o_aoffs) = assert_pair_matches(ev, offs, spec.num_regions, kernel)
+    if kernel == KERNEL_TILED and spec.well_formed:
+        # well-formed traces must stay on the parallel path of the tiled kernel
+        assert int(pr.last_status["n_sequential_tiles"]) == 0
     cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
     ag = argus.argus_aggregate(pr.intervals, pr.interval_offsets, pr.ambig, pr.ambig_offsets, spec.warps_per_cta, cta_sm,
                                spec.num_sms, spec.num_regions)
