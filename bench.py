@@ -156,6 +156,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3, help="config index 0..4 (default 3: decode megakernel, the largest)")
+    ap.add_argument("--iters", type=int, default=0, help="override the workload's iteration count (smaller trace for profiler captures)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-ctas", type=int, default=6, help="CTAs of the workload the CPU baseline is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -169,6 +170,8 @@ def main():
 
     from paper_2609_12299_b200 import tracegen as tg
     spec = tg.config(args.workload)
+    if args.iters:
+        spec = spec.scaled(iters=args.iters)
 
     if args.impl == "reference":
         if rank == 0:
@@ -181,6 +184,9 @@ def main():
     import paper_2609_12299_b200 as argus
 
     argus.load_library()  # raises if the CUDA library was not built: there is no fallback
+    if os.environ.get("ARGUS_TILE_VARIANT"):
+        from paper_2609_12299_b200.binding import argus_set_tile_variant
+        argus_set_tile_variant(int(os.environ["ARGUS_TILE_VARIANT"]))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device")
     dev = torch.device("cuda", local_rank)

@@ -82,6 +82,14 @@ def load_library():
     return lib
 
 
+def argus_set_tile_variant(v: int) -> None:
+    """Tuning aid: selects an alternative tile shape of the tiled pairing kernel (0 = default)."""
+    lib = load_library()
+    lib.argus_set_tile_variant.argtypes = [ctypes.c_int]
+    lib.argus_set_tile_variant.restype = None
+    lib.argus_set_tile_variant(int(v))
+
+
 def argus_launch_count() -> int:
     return int(load_library().argus_launch_count())
 

@@ -1,9 +1,9 @@
 // argus_pair_tiled.cu — tiled pairing kernel for sm_100a.
 //
 // One CTA walks one stream tile by tile (T = NT * E events per tile); tiles arrive in shared
-// memory by TMA bulk copies (double buffered, mbarrier completion) and the tile's intervals leave
-// through a shared-memory staging buffer and one TMA bulk store. The per-stream region stack is
-// carried from tile to tile in shared memory, so CTAs never wait on one another.
+// memory by TMA bulk copies (double buffered, mbarrier completion) and interval records leave with
+// coalesced 16-byte stores, one thread per record. The per-stream region stack is carried from tile
+// to tile in shared memory, so CTAs never wait on one another.
 //
 // Inside a tile every thread owns E consecutive events (E odd: conflict-free 16-byte shared loads)
 // and the stack height before each event comes from a block-wide prefix sum of +1/-1. With heights
@@ -28,7 +28,6 @@ __device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
@@ -46,13 +45,6 @@ __device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void tma_store_1d(void* dst, const void* src, u32 bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void tma_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // Bounded wait: gives up after ~2^22 polls (seconds); the caller then reports ARGUS_ERR_TIMEOUT.
 __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
@@ -64,23 +56,31 @@ __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
 }
 
 constexpr int kLevelWindow = 32;  // levels [lbase, lbase + 32) may hold open begins of a tile
+constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 1 sink for "no parent", padding
+constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
 
+// Shared memory of one CTA. Events of the two tile buffers and the frames carried from earlier tiles
+// share one index space, so that "the frame an end closes" and "its parent" are plain indices:
+//   ev0[0..T) | car0[0..80) | car1[0..80) | ev1[0..T)
+// A tile in buffer 0 addresses carried level L as T + L (car0); a tile in buffer 1 as L - 80 (car1).
+// The tile in buffer b reads car_b and writes the stack it leaves behind into car_{b^1}.
 template <int NT, int E>
 struct TileSmem {
   static constexpr int T = NT * E;
   static constexpr int NW = NT / 32;
   static constexpr int MAXI = T / 2 + ARGUS_MAX_DEPTH;  // intervals a well-nested tile can emit
-  uint4 ev[2][T];                  // two event tiles (TMA destinations)
-  uint4 stage[MAXI * 3];           // interval records of the current tile (TMA source)
-  u64 fchild[T];                   // per begin: inclusive time of its finished children
-  ArgusFrame cstack[2][ARGUS_MAX_DEPTH];  // carried stack, double buffered across the carry update
-  u64 cacc[ARGUS_MAX_DEPTH];       // this tile's child time for frames of the carried stack
+  static constexpr int NI = (MAXI + NT - 1) / NT;       // intervals per thread in the emission phases
+  uint4 evall[2 * T + 2 * kCar];
+  u64 accall[T + 2 * kCar];        // child time per frame, same index space shifted by kCar
+  uint2 desc[MAXI];                // per end, in end order: {end idx | partner << 16, parent | depth << 16}
+  u32 cidx[2][ARGUS_MAX_DEPTH];    // begin index (within the stream) of each carried frame
+  u64 cchild[2][ARGUS_MAX_DEPTH];  // child time of each carried frame as the tile found it (for the redo path)
+  ArgusFrame fstk[ARGUS_MAX_DEPTH];  // stack in the layout the sequential redo path uses
   u64 opens[NT];                   // per thread: local indices of begins left open (top = low nibble)
   int hend[NT];                    // per thread: stack height after its last event
-  u32 fix[E][NT];                  // per thread: staged intervals that still need their child time
   u32 mask[kLevelWindow][NW];      // per level: threads that leave a begin open at that level
   u32 wmask[kLevelWindow];         // per level: warps with a non-zero mask word
-  u32 scan_ws[36];
+  u32 warp_tot[32];
   u64 bar[2];
   u64 cur_stream;
   u64 n_int;                       // written by the sequential redo path
@@ -111,9 +111,10 @@ __device__ __forceinline__ int tile_lookup(const TileSmem<NT, E>& sm, int L, int
 template <int NT, int E>
 __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
   using SM = TileSmem<NT, E>;
-  constexpr int T = SM::T, NW = SM::NW, MAXI = SM::MAXI;
-  static_assert(E % 2 == 1 && E <= 15, "E must be odd (bank-conflict-free) and fit 4-bit indices");
-  static_assert(NW <= 16, "warp masks are 16 bits wide at most");
+  constexpr int T = SM::T, NW = SM::NW, MAXI = SM::MAXI, NI = SM::NI;
+  constexpr int kBad = 0x3fff;  // reference that marks a tile as not well nested
+  static_assert(E % 2 == 1 && E <= 15, "E must be odd and fit 4-bit indices");
+  static_assert(NW <= 16 && NT % 32 == 0 && NT >= ARGUS_MAX_DEPTH && T + kCar < kBad, "block shape");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   SM& sm = *reinterpret_cast<SM*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -128,7 +129,6 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
   u32 ph0 = 0, ph1 = 0;  // mbarrier phase parities
   const u64 off0 = a.stream_offsets[0];
   u32 tot_ctx = 0, tot_rev = 0, tot_clamp = 0;
-  bool stores_pending = false;  // thread 0: a bulk store group may still be reading `stage`
 
   for (;;) {
     if (tid == 0) sm.cur_stream = atomicAdd(a.redo ? &a.ctl->ticket2 : &a.ctl->ticket, 1ull);
@@ -152,23 +152,29 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
     const u32 ntiles = (n + T - 1) / T;
     int ch = 0;          // carried stack height (uniform)
     u64 n_int = 0;       // intervals of this stream so far (uniform)
-    int cs = 0;          // which carried-stack buffer is current
     bool stream_failed = false;
     if (tid == 0 && ntiles > 0) {
       const u32 bytes = (n < (u32)T ? n : (u32)T) * 16u;
       mbar_expect_tx(&sm.bar[0], bytes);
-      tma_load_1d(sm.ev[0], src, bytes, &sm.bar[0]);
+      tma_load_1d(sm.evall, src, bytes, &sm.bar[0]);
     }
 
     for (u32 ti = 0; ti < ntiles; ++ti) {
       const int b = ti & 1;
       const u32 tile_start = ti * (u32)T;
       const int tn = (int)((n - tile_start) < (u32)T ? (n - tile_start) : (u32)T);
+      uint4* const ev0 = sm.evall;
+      uint4* const ev1 = sm.evall + T + 2 * kCar;
+      const uint4* evb = b ? ev1 : ev0;                  // evb[ref] for every reference of this tile
+      u64* accb = sm.accall + kCar;                      // accb[ref]
+      const int cbase = b ? -kCar : T;                   // carried level L of this tile -> reference cbase + L
+      const int nbase = b ? T : -kCar;                   // same for the next tile (other buffer)
+      uint4* const car_next = sm.evall + T + (b ? 0 : kCar);
       if (tid == 0 && ti + 1 < ntiles) {  // prefetch the next tile into the other buffer
         const u32 nstart = tile_start + T;
         const u32 bytes = ((n - nstart) < (u32)T ? (n - nstart) : (u32)T) * 16u;
         mbar_expect_tx(&sm.bar[b ^ 1], bytes);
-        tma_load_1d(sm.ev[b ^ 1], src + nstart, bytes, &sm.bar[b ^ 1]);
+        tma_load_1d(b ? ev0 : ev1, src + nstart, bytes, &sm.bar[b ^ 1]);
       }
       {
         const bool ok = mbar_wait_bounded(&sm.bar[b], b ? ph1 : ph0);
@@ -177,14 +183,14 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
       }
 
       // ---------------- phase A: local shape, prefix sums, open-level masks ----------------
-      const uint4* evb = sm.ev[b];
-      uint4 r[E];
+      u32 tags[E];
       u32 valid = 0;
 #pragma unroll
       for (int k = 0; k < E; ++k) {
         const int e = tid * E + k;
-        if (e < tn) { r[k] = evb[e]; valid |= 1u << k; } else { r[k] = make_uint4(0, 0, 0, 0); }
-        sm.fchild[e] = 0;
+        tags[k] = reinterpret_cast<const u32*>(evb + e)[2];
+        if (e < tn) valid |= 1u << k;
+        accb[e] = 0;
       }
       u64 stk = 0;
       int lsp = 0, npend = 0, nb = 0, ne = 0, rel = 0, maxrel = 0;
@@ -192,8 +198,8 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
 #pragma unroll
       for (int k = 0; k < E; ++k) {
         if (valid & (1u << k)) {
-          if ((r[k].z >> 1) >= a.num_regions) bad = true;
-          if (r[k].z & 1u) {
+          if ((tags[k] >> 1) >= a.num_regions) bad = true;
+          if (tags[k] & 1u) {
             ++ne; --rel;
             if (lsp > 0) { stk >>= 4; --lsp; } else { ++npend; }
           } else {
@@ -203,13 +209,28 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
           }
         }
       }
-      // zero the per-tile tables before the scan's barriers
+      // zero the per-tile tables before the scan's barrier
       sm.mask[tid / NW][tid % NW] = 0;
       if (tid < kLevelWindow) sm.wmask[tid] = 0;
-      if (tid < ARGUS_MAX_DEPTH) sm.cacc[tid] = 0;
-      if (tid == 0) { sm.bad = 0; sm.failed = 0; if (stores_pending) { tma_wait_read0(); stores_pending = false; } }
-      u32 tot;
-      const u32 ex = argus_block_exclusive_scan<u32>((u32)nb | ((u32)ne << 16), sm.scan_ws, &tot);
+      if (tid == 0) { sm.bad = 0; sm.failed = 0; accb[cbase + kSink] = 0; }
+      // block prefix sum of (begins, ends), 16 bits each: one barrier
+      const u32 mine_cnt = (u32)nb | ((u32)ne << 16);
+      u32 incl_cnt = mine_cnt;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const u32 o = __shfl_up_sync(0xffffffffu, incl_cnt, d);
+        if (lane >= d) incl_cnt += o;
+      }
+      if (lane == 31) sm.warp_tot[warp] = incl_cnt;
+      __syncthreads();
+      u32 before = 0, tot = 0;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const u32 t = sm.warp_tot[w];
+        if (w < warp) before += t;
+        tot += t;
+      }
+      const u32 ex = before + incl_cnt - mine_cnt;
       const int tile_nb = (int)(tot & 0xffffu), tile_ne = (int)(tot >> 16);
       const int h0 = ch + (int)(ex & 0xffffu) - (int)(ex >> 16);
       const int rank0 = (int)(ex >> 16);
@@ -238,141 +259,139 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
       if (bad) sm.bad = 1;
       __syncthreads();
 
-      // ---------------- phase B: match, emit to staging, feed parent accumulators ----------------
-      u32 t_ctx = 0, t_rev = 0, t_clamp = 0;
-      int nfix = 0;
-      const ArgusFrame* cst = sm.cstack[cs];
+      // ---------------- phase B1: one descriptor per end marker (who is my begin, who is my parent) -------------
+      const int nmax = __reduce_max_sync(0xffffffffu, npend);  // warp-wide, outside any divergent branch
       if (!bad) {
-        int h = h0, rank = rank0;
+        // frames below this thread's floor, outermost needed first: level h0-1-j for j = 0..npend, 15 bits each
+        u64 outer_lo = 0, outer_hi = 0;
+        for (int j = 0; j <= nmax; ++j) {
+          const int L = h0 - 1 - j;
+          int ref;
+          if (j > npend) ref = 0;
+          else if (L < 0) ref = cbase + kSink;
+          else {
+            ref = tile_lookup<NT, E>(sm, L, lbase, warp, lane);
+            if (ref < 0) ref = L < ch ? cbase + L : kBad;
+          }
+          const u64 v = (u64)((u32)ref & 0x7fffu);
+          if (j < 4) outer_lo |= v << (15 * j); else outer_hi |= v << (15 * ((j - 4) & 3));
+          if (j >= 8 && j <= npend) bad = true;  // more than 8 frames closed from outside: leave it to the redo path
+        }
+        int h = h0, rank = rank0, pi = 0;
         stk = 0; lsp = 0;
-        int outer_e = h > 0 ? tile_lookup<NT, E>(sm, h - 1, lbase, warp, lane) : -1;  // frame at level floor-1
+        auto outer_at = [&](int j) -> int {
+          const u64 w = j < 4 ? outer_lo : outer_hi;
+          int r = (int)((w >> (15 * (j & 3))) & 0x7fffull);
+          return (r & 0x4000) ? r - 0x8000 : r;  // sign-extend 15 bits (carried references of buffer 1 are negative)
+        };
 #pragma unroll
         for (int k = 0; k < E; ++k) {
           if (!(valid & (1u << k))) continue;
-          const u32 tag = r[k].z;
-          if (!(tag & 1u)) {
+          if (!(tags[k] & 1u)) {
             stk = (stk << 4) | (u64)k; ++lsp; ++h;
             continue;
           }
           --h;  // level of the frame this end closes
-          const u64 ts = (u64)r[k].x | ((u64)r[k].y << 32);
-          u64 bts = 0, child = 0;
-          u32 bregion = 0xffffffffu, bctx = 0, bidx = 0;
-          int parent_e, pref = -1;
-          bool cross = false;
+          int partner, parent;
           if (lsp > 0) {
-            const int ej = tid * E + (int)(stk & 15ull);
+            partner = tid * E + (int)(stk & 15ull);
             stk >>= 4; --lsp;
-            const uint4 pe = evb[ej];
-            bts = (u64)pe.x | ((u64)pe.y << 32); bregion = pe.z >> 1; bctx = pe.w; bidx = tile_start + (u32)ej;
-            child = sm.fchild[ej];
-            parent_e = lsp > 0 ? tid * E + (int)(stk & 15ull) : outer_e;
+            parent = lsp > 0 ? tid * E + (int)(stk & 15ull) : outer_at(pi);
           } else {
-            cross = true;
-            pref = outer_e;
-            if (pref >= 0) {
-              const uint4 pe = evb[pref];
-              bts = (u64)pe.x | ((u64)pe.y << 32); bregion = pe.z >> 1; bctx = pe.w; bidx = tile_start + (u32)pref;
-            } else if (h >= 0 && h < ch) {
-              const ArgusFrame& f = cst[h];
-              bts = f.ts; bregion = f.region; bctx = f.ctx; bidx = f.idx;
-            }
-            outer_e = h > 0 ? tile_lookup<NT, E>(sm, h - 1, lbase, warp, lane) : -1;
-            parent_e = outer_e;
+            partner = outer_at(pi);
+            ++pi;
+            parent = outer_at(pi);
+            if (h < 0) bad = true;
           }
-          if (bregion != (tag >> 1)) { bad = true; break; }
-          u32 flags = 0;
-          u64 incl;
-          if (r[k].w != bctx) { flags |= ARGUS_FLAG_CTX_MISMATCH; ++t_ctx; }
-          if (ts < bts) { incl = 0; flags |= ARGUS_FLAG_TIME_REVERSED; ++t_rev; } else { incl = ts - bts; }
-          u64 excl = 0;
-          if (!cross) {
-            if (child > incl) { flags |= ARGUS_FLAG_CHILD_CLAMPED; ++t_clamp; } else { excl = incl - child; }
-          } else {
-            sm.fix[nfix++][tid] = (u32)rank | ((u32)(pref + 1) << 16);
-          }
-          u32 preg = ARGUS_NONE;
-          if (parent_e >= 0) {
-            preg = evb[parent_e].z >> 1;
-            if (incl) atomicAdd(&sm.fchild[parent_e], incl);
-          } else if (h > 0) {
-            if (h - 1 < ch) { preg = cst[h - 1].region; if (incl) atomicAdd(&sm.cacc[h - 1], incl); } else { bad = true; break; }
-          }
-          uint4* q = sm.stage + rank * 3;
-          q[0] = make_uint4((u32)bts, (u32)(bts >> 32), (u32)incl, (u32)(incl >> 32));
-          q[1] = make_uint4((u32)excl, (u32)(excl >> 32), bregion, bctx);
-          q[2] = make_uint4(s, preg, bidx, ((u32)h & 0xffffu) | (flags << 16));
-          ++rank;
+          if (partner == kBad || parent == kBad) bad = true;
+          sm.desc[rank++] = make_uint2((u32)(tid * E + k) | ((u32)partner << 16), ((u32)parent & 0xffffu) | ((u32)h << 16));
         }
         if (bad) sm.bad = 1;
       }
       __syncthreads();
+
+      // ---------------- phase B2a: one thread per end marker: inclusive time feeds the parent frame -------------
+      if (!sm.bad) {
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int rk = tid + i * NT;
+          if (rk < tile_ne) {
+            const uint2 d = sm.desc[rk];
+            const uint4 ee = evb[d.x & 0xffffu];
+            const uint4 pe = evb[(int)(short)(d.x >> 16)];
+            if ((pe.z >> 1) != (ee.z >> 1) || (pe.z & 1u)) sm.bad = 1;
+            const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
+            if (ts > bts) atomicAdd(&accb[(int)(short)(d.y & 0xffffu)], ts - bts);
+          }
+        }
+      }
+      __syncthreads();
       const bool tile_bad = sm.bad != 0;
       if (sm.dead) {  // a bulk copy never arrived: report and leave (uniform decision)
-        if (tid == 0) { argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start); tma_wait_all0(); }
+        if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
         return;
       }
 
       if (!tile_bad) {
-        // ---------------- phase C: finish cross-thread intervals, update the carried stack ----------------
-        for (int f = 0; f < nfix; ++f) {
-          const u32 fx = sm.fix[f][tid];
-          const int slot = (int)(fx & 0xffffu), pref = (int)(fx >> 16) - 1;
-          uint4* q = sm.stage + slot * 3;
-          const uint4 q0 = q[0];
-          uint4 q2 = q[2];
-          const u64 incl = (u64)q0.z | ((u64)q0.w << 32);
-          const int level = (int)(q2.w & 0xffffu);
-          const u64 child = pref >= 0 ? sm.fchild[pref] : cst[level].child + sm.cacc[level];
-          u64 excl = 0;
-          if (child > incl) { q2.w |= ARGUS_FLAG_CHILD_CLAMPED << 16; ++t_clamp; q[2] = q2; } else { excl = incl - child; }
-          uint4 q1 = q[1];
-          q1.x = (u32)excl; q1.y = (u32)(excl >> 32);
-          q[1] = q1;
+        // ---------------- phase B2b: exclusive time, parent region, interval records; carried stack -------------
+        const u64 pos0 = out_base + n_int;
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int rk = tid + i * NT;
+          if (rk < tile_ne) {
+            const uint2 d = sm.desc[rk];
+            const int partner = (int)(short)(d.x >> 16), parent = (int)(short)(d.y & 0xffffu);
+            const uint4 ee = evb[d.x & 0xffffu];
+            const uint4 pe = evb[partner];
+            const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
+            const u64 child = accb[partner];
+            u32 flags = 0;
+            u64 incl = 0, excl = 0;
+            if (ee.w != pe.w) { flags |= ARGUS_FLAG_CTX_MISMATCH; ++tot_ctx; }
+            if (ts < bts) { flags |= ARGUS_FLAG_TIME_REVERSED; ++tot_rev; } else { incl = ts - bts; }
+            if (child > incl) { flags |= ARGUS_FLAG_CHILD_CLAMPED; ++tot_clamp; } else { excl = incl - child; }
+            const bool carried = (u32)partner >= (u32)T;
+            const u32 bidx = carried ? sm.cidx[b][partner - cbase] : tile_start + (u32)partner;
+            const u32 preg = parent == cbase + kSink ? ARGUS_NONE : (reinterpret_cast<const u32*>(evb + parent)[2] >> 1);
+            const u64 pos = pos0 + (u64)rk;
+            if (pos < a.interval_capacity) {
+              uint4* q = reinterpret_cast<uint4*>(a.intervals + pos);
+              q[0] = make_uint4(pe.x, pe.y, (u32)incl, (u32)(incl >> 32));
+              q[1] = make_uint4((u32)excl, (u32)(excl >> 32), pe.z >> 1, pe.w);
+              q[2] = make_uint4(s, preg, bidx, (d.y >> 16) | (flags << 16));
+            } else if (!a.redo) {
+              a.ctl->spec_overflow = 1;
+            }
+          }
         }
         const int new_ch = ch + tile_nb - tile_ne;
-        if (tid < ARGUS_MAX_DEPTH && tid < new_ch) {
+        if (tid < new_ch) {  // the stack this tile leaves behind, in the next tile's index space
           const int e = tile_lookup<NT, E>(sm, tid, lbase, NW, 0);
-          ArgusFrame f;
-          if (e >= 0) {
-            const uint4 pe = evb[e];
-            f.ts = (u64)pe.x | ((u64)pe.y << 32); f.child = sm.fchild[e]; f.region = pe.z >> 1; f.ctx = pe.w;
-            f.idx = tile_start + (u32)e; f.pad = 0;
-          } else {
-            f = cst[tid];
-            f.child += sm.cacc[tid];
-          }
-          sm.cstack[cs ^ 1][tid] = f;
-        }
-        tot_ctx += t_ctx; tot_rev += t_rev; tot_clamp += t_clamp;
-        fence_proxy_async();
-        __syncthreads();
-        if (tid == 0 && tile_ne > 0) {
-          const u64 pos = out_base + n_int;
-          u64 fit = (u64)tile_ne;
-          if (pos + fit > a.interval_capacity) {
-            fit = pos < a.interval_capacity ? a.interval_capacity - pos : 0;
-            if (!a.redo) a.ctl->spec_overflow = 1;
-          }
-          if (fit) {
-            tma_store_1d(a.intervals + pos, sm.stage, (u32)fit * 48u);
-            tma_commit();
-            stores_pending = true;
-          }
+          const int from = e >= 0 ? e : cbase + tid;
+          car_next[tid] = evb[from];
+          accb[nbase + tid] = accb[from];
+          sm.cidx[b ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[b][tid];
+          sm.cchild[b ^ 1][tid] = accb[from];
         }
         ch = new_ch;
         n_int += (u64)tile_ne;
-        cs ^= 1;
+        __syncthreads();
       } else {
         // ---------------- redo this tile with the sequential stack machine ----------------
+        if (tid < ch) {
+          const uint4 f = evb[cbase + tid];
+          ArgusFrame& o = sm.fstk[tid];
+          o.ts = (u64)f.x | ((u64)f.y << 32); o.child = sm.cchild[b][tid]; o.region = f.z >> 1; o.ctx = f.w;
+          o.idx = sm.cidx[b][tid]; o.pad = 0;
+        }
+        __syncthreads();
         if (tid == 0) {
           ArgusSeqState st;
           st.h = ch; st.n_int = n_int; st.n_ctx = st.n_rev = st.n_clamp = 0; st.failed = false;
-          ArgusFrame* stkp = sm.cstack[cs];
           bool ok = true;
           for (int e = 0; e < tn && ok; ++e) {
             const uint4 pe = evb[e];
-            ok = argus_seq_step(a, stkp, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w);
+            ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w);
           }
           tot_ctx += st.n_ctx; tot_rev += st.n_rev; tot_clamp += st.n_clamp;
           sm.ch = st.h;
@@ -384,6 +403,14 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
         ch = sm.ch;
         n_int = sm.n_int;
         if (sm.failed) stream_failed = true;
+        if (tid < ch) {
+          const ArgusFrame f = sm.fstk[tid];
+          car_next[tid] = make_uint4((u32)f.ts, (u32)(f.ts >> 32), f.region << 1, f.ctx);
+          accb[nbase + tid] = f.child;
+          sm.cidx[b ^ 1][tid] = f.idx;
+          sm.cchild[b ^ 1][tid] = f.child;
+        }
+        __syncthreads();
       }
       if (stream_failed) {
         if (ti + 1 < ntiles) {  // drain the prefetched tile before the buffer is reused
@@ -397,11 +424,13 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
 
     __syncthreads();
     if (sm.dead) {
-      if (tid == 0) { argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, 0); tma_wait_all0(); }
+      if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, 0);
       return;
     }
     if (!a.redo) {
-      if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cstack[cs][tid].idx, ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
+      // frames still open at the end of the stream (they sit in the block the next tile would read)
+      const int bl = (int)(ntiles & 1u);
+      if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[bl][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
       if (tid == 0) a.counts[s] = n_int;
     }
     __syncthreads();
@@ -417,9 +446,7 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
       if (tot_clamp) atomicAdd((u64*)&a.status->n_child_clamped, (u64)tot_clamp);
     }
   }
-  if (tid == 0) tma_wait_all0();  // shared memory must outlive the last bulk store
 }
-
 template <int NT, int E>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   static int grid_cache = 0;
@@ -439,8 +466,25 @@ int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   return ARGUS_OK;
 }
 
+int g_variant = 0;
+
 }  // namespace
 
 bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0; }
 
-int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) { return launch_tiled<256, 5>(a, stream); }
+// Tile shape used by the tiled kernel: 0 = default. Other values select alternative shapes (tuning aid).
+extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
+
+int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
+  switch (g_variant) {
+    case 1: return launch_tiled<128, 7>(a, stream);
+    case 2: return launch_tiled<128, 9>(a, stream);
+    case 3: return launch_tiled<256, 7>(a, stream);
+    case 4: return launch_tiled<128, 5>(a, stream);
+    case 5: return launch_tiled<128, 11>(a, stream);
+    case 6: return launch_tiled<256, 9>(a, stream);
+    case 7: return launch_tiled<128, 15>(a, stream);
+    case 8: return launch_tiled<64, 9>(a, stream);
+    default: return launch_tiled<256, 5>(a, stream);
+  }
+}
