@@ -55,6 +55,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
   return false;
 }
 
+#ifdef ARGUS_TILE_TIMING
+__device__ unsigned long long g_tile_timing[8];
+#define TT_MARK(i) do { if (tid == 0) { const long long c__ = clock64(); tt[i] += (unsigned long long)(c__ - tlast); tlast = c__; } } while (0)
+#else
+#define TT_MARK(i) do { } while (0)
+#endif
+
 constexpr int kLevelWindow = 32;  // levels [lbase, lbase + 32) may hold open begins of a tile
 constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 1 sink for "no parent", padding
 constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
@@ -80,6 +87,7 @@ struct TileSmem {
   int hend[NT];                    // per thread: stack height after its last event
   u32 mask[kLevelWindow][NW];      // per level: threads that leave a begin open at that level
   u32 wmask[kLevelWindow];         // per level: warps with a non-zero mask word
+  short prev[kLevelWindow][NW + 1];  // per level and warp w: latest open begin in warps < w (tile index or -1); [NW] = all warps
   u32 warp_tot[32];
   u64 bar[2];
   u64 cur_stream;
@@ -88,28 +96,8 @@ struct TileSmem {
   int bad, dead, failed;
 };
 
-template <int NT, int E>
-__device__ __forceinline__ int tile_lookup(const TileSmem<NT, E>& sm, int L, int lbase, int warp, int lane) {
-  // latest begin left open at level L by a thread before (warp, lane); -1 if none in this tile
-  const int l = L - lbase;
-  if (l < 0 || l >= kLevelWindow) return -1;
-  u32 m = warp < TileSmem<NT, E>::NW ? (sm.mask[l][warp] & ((1u << lane) - 1u)) : 0u;
-  int w = warp;
-  if (!m) {
-    const u32 ww = sm.wmask[l] & ((1u << warp) - 1u);
-    if (!ww) return -1;
-    w = 31 - __clz(ww);
-    m = sm.mask[l][w];
-    if (!m) return -1;
-  }
-  const int tau = w * 32 + 31 - __clz(m);
-  const int sh = 4 * (sm.hend[tau] - 1 - L);
-  const int j = (int)((sm.opens[tau] >> (sh & 63)) & 15ull);
-  return tau * E + j;
-}
-
-template <int NT, int E>
-__global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
+template <int NT, int E, int MINB>
+__global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   using SM = TileSmem<NT, E>;
   constexpr int T = SM::T, NW = SM::NW, MAXI = SM::MAXI, NI = SM::NI;
   constexpr int kBad = 0x3fff;  // reference that marks a tile as not well nested
@@ -129,6 +117,10 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
   u32 ph0 = 0, ph1 = 0;  // mbarrier phase parities
   const u64 off0 = a.stream_offsets[0];
   u32 tot_ctx = 0, tot_rev = 0, tot_clamp = 0;
+#ifdef ARGUS_TILE_TIMING
+  unsigned long long tt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  long long tlast = clock64();
+#endif
 
   for (;;) {
     if (tid == 0) sm.cur_stream = atomicAdd(a.redo ? &a.ctl->ticket2 : &a.ctl->ticket, 1ull);
@@ -176,11 +168,13 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
         mbar_expect_tx(&sm.bar[b ^ 1], bytes);
         tma_load_1d(b ? ev0 : ev1, src + nstart, bytes, &sm.bar[b ^ 1]);
       }
+      TT_MARK(0);
       {
         const bool ok = mbar_wait_bounded(&sm.bar[b], b ? ph1 : ph0);
         if (b) ph1 ^= 1; else ph0 ^= 1;
         if (!ok) sm.dead = 1;
       }
+      TT_MARK(1);
 
       // ---------------- phase A: local shape, prefix sums, open-level masks ----------------
       u32 tags[E];
@@ -240,13 +234,14 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
       const int olo = lsp > 0 ? hend - lsp - lbase : 1000;  // levels of the begins this thread leaves open
       const int ohi = lsp > 0 ? hend - lbase : -1000;       // (relative to lbase, half-open)
       if (lsp > 0 && (olo < 0 || ohi > kLevelWindow)) bad = true;
+      const u64 opens_reg = stk;
       sm.opens[tid] = stk;
       sm.hend[tid] = hend;
+      u32 mine = 0;  // lane l: threads of this warp that leave a begin open at level lbase + l
       {
         int wlo = __reduce_min_sync(0xffffffffu, olo), whi = __reduce_max_sync(0xffffffffu, ohi);
         wlo = wlo < 0 ? 0 : wlo;
         whi = whi > kLevelWindow ? kLevelWindow : whi;
-        u32 mine = 0;
         for (int l = wlo; l < whi; ++l) {
           const u32 bal = __ballot_sync(0xffffffffu, l >= olo && l < ohi);
           if (lane == l) mine = bal;
@@ -258,25 +253,59 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
       }
       if (bad) sm.bad = 1;
       __syncthreads();
+      {  // per (level, warp): the latest open begin among the warps before it
+        const int l = tid / NW, w = tid % NW;
+        const u32 wm = sm.wmask[l];
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+          const int wq = pass ? NW : w;
+          if (pass && w != NW - 1) break;
+          const u32 ww = wm & ((1u << wq) - 1u);
+          int e = -1;
+          if (ww) {
+            const int wp = 31 - __clz(ww);
+            const u32 m = sm.mask[l][wp];
+            if (m) {
+              const int tau = wp * 32 + 31 - __clz(m);
+              const int sh = 4 * (sm.hend[tau] - 1 - (lbase + l));
+              e = tau * E + (int)((sm.opens[tau] >> (sh & 63)) & 15ull);
+            }
+          }
+          sm.prev[l][wq] = (short)e;
+        }
+      }
+      __syncthreads();
+      TT_MARK(2);
 
       // ---------------- phase B1: one descriptor per end marker (who is my begin, who is my parent) -------------
-      const int nmax = __reduce_max_sync(0xffffffffu, npend);  // warp-wide, outside any divergent branch
-      if (!bad) {
-        // frames below this thread's floor, outermost needed first: level h0-1-j for j = 0..npend, 15 bits each
-        u64 outer_lo = 0, outer_hi = 0;
+      const int nmax = __reduce_max_sync(0xffffffffu, npend);  // warp-wide: the loop below shuffles, so every lane runs it
+      // frames below this thread's floor, outermost needed first: level h0-1-j for j = 0..npend, 15 bits each
+      u64 outer_lo = 0, outer_hi = 0;
+      {
         for (int j = 0; j <= nmax; ++j) {
           const int L = h0 - 1 - j;
+          const int l = L - lbase;
+          const bool want = j <= npend && L >= 0 && l >= 0 && l < kLevelWindow;
+          // the mask word of my warp for level l sits in lane l's register
+          const u32 mword = __shfl_sync(0xffffffffu, mine, want ? l : 0);
+          const u32 m = want ? (mword & ((1u << lane) - 1u)) : 0u;
+          const int srcl = m ? 31 - __clz(m) : lane;
+          const int hend_s = __shfl_sync(0xffffffffu, hend, srcl);
+          const u64 opens_s = __shfl_sync(0xffffffffu, opens_reg, srcl);
           int ref;
           if (j > npend) ref = 0;
           else if (L < 0) ref = cbase + kSink;
           else {
-            ref = tile_lookup<NT, E>(sm, L, lbase, warp, lane);
+            if (m) ref = (warp * 32 + srcl) * E + (int)((opens_s >> ((4 * (hend_s - 1 - L)) & 63)) & 15ull);
+            else ref = want ? (int)sm.prev[l][warp] : -1;
             if (ref < 0) ref = L < ch ? cbase + L : kBad;
           }
           const u64 v = (u64)((u32)ref & 0x7fffu);
           if (j < 4) outer_lo |= v << (15 * j); else outer_hi |= v << (15 * ((j - 4) & 3));
           if (j >= 8 && j <= npend) bad = true;  // more than 8 frames closed from outside: leave it to the redo path
         }
+      }
+      if (!bad) {
         int h = h0, rank = rank0, pi = 0;
         stk = 0; lsp = 0;
         auto outer_at = [&](int j) -> int {
@@ -309,6 +338,7 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
         if (bad) sm.bad = 1;
       }
       __syncthreads();
+      TT_MARK(3);
 
       // ---------------- phase B2a: one thread per end marker: inclusive time feeds the parent frame -------------
       if (!sm.bad) {
@@ -321,11 +351,19 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
             const uint4 pe = evb[(int)(short)(d.x >> 16)];
             if ((pe.z >> 1) != (ee.z >> 1) || (pe.z & 1u)) sm.bad = 1;
             const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
-            if (ts > bts) atomicAdd(&accb[(int)(short)(d.y & 0xffffu)], ts - bts);
+            if (ts > bts) {  // 64-bit add as two native 32-bit shared atomics; each carry is propagated exactly once
+              const u64 dlt = ts - bts;
+              u32* p = reinterpret_cast<u32*>(&accb[(int)(short)(d.y & 0xffffu)]);
+              const u32 lo32 = (u32)dlt, hi32 = (u32)(dlt >> 32);
+              const u32 old = atomicAdd(p, lo32);
+              if (hi32) atomicAdd(p + 1, hi32);
+              if (old + lo32 < old) atomicAdd(p + 1, 1u);
+            }
           }
         }
       }
       __syncthreads();
+      TT_MARK(4);
       const bool tile_bad = sm.bad != 0;
       if (sm.dead) {  // a bulk copy never arrived: report and leave (uniform decision)
         if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
@@ -366,7 +404,8 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
         }
         const int new_ch = ch + tile_nb - tile_ne;
         if (tid < new_ch) {  // the stack this tile leaves behind, in the next tile's index space
-          const int e = tile_lookup<NT, E>(sm, tid, lbase, NW, 0);
+          const int l = tid - lbase;
+          const int e = (l >= 0 && l < kLevelWindow) ? (int)sm.prev[l][NW] : -1;
           const int from = e >= 0 ? e : cbase + tid;
           car_next[tid] = evb[from];
           accb[nbase + tid] = accb[from];
@@ -376,6 +415,7 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
         ch = new_ch;
         n_int += (u64)tile_ne;
         __syncthreads();
+        TT_MARK(5);
       } else {
         // ---------------- redo this tile with the sequential stack machine ----------------
         if (tid < ch) {
@@ -436,6 +476,9 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
     __syncthreads();
   }  // streams
 
+#ifdef ARGUS_TILE_TIMING
+  if (tid == 0 && !a.redo) for (int i = 0; i < 8; ++i) atomicAdd(&g_tile_timing[i], tt[i]);
+#endif
   if (!a.redo) {
     tot_ctx = __reduce_add_sync(0xffffffffu, tot_ctx);
     tot_rev = __reduce_add_sync(0xffffffffu, tot_rev);
@@ -447,21 +490,21 @@ __global__ void __launch_bounds__(NT) k_pair_tiled(ArgusPairArgs a) {
     }
   }
 }
-template <int NT, int E>
+template <int NT, int E, int MINB>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   static int grid_cache = 0;
   const size_t smem = sizeof(TileSmem<NT, E>) + 128;
   if (!grid_cache) {
-    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int dev = 0, sms = 0, per_sm = 0;
     ARGUS_CUDA_TRY(cudaGetDevice(&dev));
     ARGUS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E>, NT, smem));
+    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB>, NT, smem));
     if (per_sm < 1) return ARGUS_ERR_CUDA;
     grid_cache = sms * per_sm;
   }
   const u32 grid = a.num_streams < (u32)grid_cache ? a.num_streams : (u32)grid_cache;
-  k_pair_tiled<NT, E><<<grid, NT, smem, stream>>>(a);
+  k_pair_tiled<NT, E, MINB><<<grid, NT, smem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   return ARGUS_OK;
 }
@@ -472,19 +515,29 @@ int g_variant = 0;
 
 bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0; }
 
+#ifdef ARGUS_TILE_TIMING
+// Debug build only: cycles thread 0 of every CTA spent per phase (other, wait, A, B1, B2a, B2b), summed; resets them.
+extern "C" int argus_debug_tile_timing(unsigned long long* out8) {
+  if (cudaMemcpyFromSymbol(out8, g_tile_timing, 64) != cudaSuccess) return ARGUS_ERR_CUDA;
+  unsigned long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (cudaMemcpyToSymbol(g_tile_timing, z, 64) != cudaSuccess) return ARGUS_ERR_CUDA;
+  return ARGUS_OK;
+}
+#endif
+
 // Tile shape used by the tiled kernel: 0 = default. Other values select alternative shapes (tuning aid).
 extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   switch (g_variant) {
-    case 1: return launch_tiled<128, 7>(a, stream);
-    case 2: return launch_tiled<128, 9>(a, stream);
-    case 3: return launch_tiled<256, 7>(a, stream);
-    case 4: return launch_tiled<128, 5>(a, stream);
-    case 5: return launch_tiled<128, 11>(a, stream);
-    case 6: return launch_tiled<256, 9>(a, stream);
-    case 7: return launch_tiled<128, 15>(a, stream);
-    case 8: return launch_tiled<64, 9>(a, stream);
-    default: return launch_tiled<256, 5>(a, stream);
+    case 1: return launch_tiled<128, 7, 4>(a, stream);
+    case 2: return launch_tiled<128, 9, 4>(a, stream);
+    case 3: return launch_tiled<256, 7, 2>(a, stream);
+    case 4: return launch_tiled<128, 5, 6>(a, stream);
+    case 5: return launch_tiled<128, 11, 3>(a, stream);
+    case 6: return launch_tiled<256, 9, 2>(a, stream);
+    case 7: return launch_tiled<128, 5, 5>(a, stream);
+    case 8: return launch_tiled<64, 9, 8>(a, stream);
+    default: return launch_tiled<256, 5, 3>(a, stream);
   }
 }
