@@ -5,14 +5,12 @@
 // coalesced 16-byte stores, one thread per record. The per-stream region stack is carried from tile
 // to tile in shared memory, so CTAs never wait on one another.
 //
-// Inside a tile every thread owns E consecutive events (E odd: conflict-free 16-byte shared loads)
-// and the stack height before each event comes from a block-wide prefix sum of +1/-1. With heights
-// known, a frame is identified by its level (stack position):
-//   - begin/end pairs that fall inside one thread are matched by that thread with a 4-bit-per-entry
-//     register stack;
-//   - an end whose begin lies in an earlier thread finds it through per-level bitmasks of the
-//     threads that leave a begin open at that level (latest such thread before it); if there is
-//     none, the begin is in the stack carried from earlier tiles;
+// Inside a tile the stack height before each event comes from a block-wide prefix sum of +1/-1, so
+// every marker knows its level (stack position) without walking the stack:
+//   - every begin sets its bit in a per-level bitmap over the tile's event positions;
+//   - every end (one thread per end marker) finds its begin as the latest set bit of its own level
+//     before it, and its parent as the latest set bit one level down before that begin; when there
+//     is none in the tile, the frame is in the stack carried from earlier tiles;
 //   - every finished interval adds its inclusive time to its parent frame's accumulator (shared
 //     atomics), which gives exclusive time without ordering the threads.
 // This is exact when the tile is well nested (every end meets the frame on top with the same region
@@ -62,9 +60,10 @@ __device__ unsigned long long g_tile_timing[8];
 #define TT_MARK(i) do { } while (0)
 #endif
 
-constexpr int kLevelWindow = 32;  // levels [lbase, lbase + 32) may hold open begins of a tile
+constexpr int kLevelWindow = 32;  // begins of a tile may sit at levels [lbase, lbase + 32)
 constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 1 sink for "no parent", padding
 constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
+constexpr int kBadRef = 0x3fff;   // reference that marks a tile as not well nested
 
 // Shared memory of one CTA. Events of the two tile buffers and the frames carried from earlier tiles
 // share one index space, so that "the frame an end closes" and "its parent" are plain indices:
@@ -75,19 +74,17 @@ template <int NT, int E>
 struct TileSmem {
   static constexpr int T = NT * E;
   static constexpr int NW = NT / 32;
+  static constexpr int NWORDS = T / 32;                 // bitmap words per level
   static constexpr int MAXI = T / 2 + ARGUS_MAX_DEPTH;  // intervals a well-nested tile can emit
   static constexpr int NI = (MAXI + NT - 1) / NT;       // intervals per thread in the emission phases
   uint4 evall[2 * T + 2 * kCar];
   u64 accall[T + 2 * kCar];        // child time per frame, same index space shifted by kCar
-  uint2 desc[MAXI];                // per end, in end order: {end idx | partner << 16, parent | depth << 16}
+  u32 desc[MAXI];                  // per end, in end order: event index | level << 16
+  u32 bm[kLevelWindow][NWORDS];    // per level: bit e set = event e of the tile is a begin at that level
+  u64 summ[kLevelWindow];          // per level: bit w set = bm[level][w] != 0
   u32 cidx[2][ARGUS_MAX_DEPTH];    // begin index (within the stream) of each carried frame
   u64 cchild[2][ARGUS_MAX_DEPTH];  // child time of each carried frame as the tile found it (for the redo path)
   ArgusFrame fstk[ARGUS_MAX_DEPTH];  // stack in the layout the sequential redo path uses
-  u64 opens[NT];                   // per thread: local indices of begins left open (top = low nibble)
-  int hend[NT];                    // per thread: stack height after its last event
-  u32 mask[kLevelWindow][NW];      // per level: threads that leave a begin open at that level
-  u32 wmask[kLevelWindow];         // per level: warps with a non-zero mask word
-  short prev[kLevelWindow][NW + 1];  // per level and warp w: latest open begin in warps < w (tile index or -1); [NW] = all warps
   u32 warp_tot[32];
   u64 bar[2];
   u64 cur_stream;
@@ -96,13 +93,29 @@ struct TileSmem {
   int bad, dead, failed;
 };
 
+// Latest begin of the tile at level L and position < pos; -1 if there is none.
+template <int NT, int E>
+__device__ __forceinline__ int tile_latest_begin(const TileSmem<NT, E>& sm, int L, int lbase, int pos) {
+  constexpr int NWORDS = TileSmem<NT, E>::NWORDS;
+  const int l = L - lbase;
+  if (l < 0 || l >= kLevelWindow) return -1;
+  const int w = pos >> 5;
+  if (w < NWORDS) {
+    const u32 m = sm.bm[l][w] & ((1u << (pos & 31)) - 1u);
+    if (m) return w * 32 + 31 - __clz(m);
+  }
+  const u64 s = sm.summ[l] & ((w >= 64) ? ~0ull : ((1ull << w) - 1ull));
+  if (!s) return -1;
+  const int w2 = 63 - __clzll((long long)s);
+  const u32 m2 = sm.bm[l][w2];
+  return m2 ? w2 * 32 + 31 - __clz(m2) : -1;
+}
+
 template <int NT, int E, int MINB>
 __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   using SM = TileSmem<NT, E>;
-  constexpr int T = SM::T, NW = SM::NW, MAXI = SM::MAXI, NI = SM::NI;
-  constexpr int kBad = 0x3fff;  // reference that marks a tile as not well nested
-  static_assert(E % 2 == 1 && E <= 15, "E must be odd and fit 4-bit indices");
-  static_assert(NW <= 16 && NT % 32 == 0 && NT >= ARGUS_MAX_DEPTH && T + kCar < kBad, "block shape");
+  constexpr int T = SM::T, NW = SM::NW, NWORDS = SM::NWORDS, MAXI = SM::MAXI, NI = SM::NI;
+  static_assert(NW <= 32 && NT % 32 == 0 && NT >= ARGUS_MAX_DEPTH && NWORDS <= 64 && T + kCar < kBadRef, "block shape");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   SM& sm = *reinterpret_cast<SM*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -176,36 +189,23 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       }
       TT_MARK(1);
 
-      // ---------------- phase A: local shape, prefix sums, open-level masks ----------------
+      // ---------------- phase A: heights by prefix sum; begins into per-level bitmaps; ends into `desc` ------------
       u32 tags[E];
-      u32 valid = 0;
-#pragma unroll
-      for (int k = 0; k < E; ++k) {
-        const int e = tid * E + k;
-        tags[k] = reinterpret_cast<const u32*>(evb + e)[2];
-        if (e < tn) valid |= 1u << k;
-        accb[e] = 0;
-      }
-      u64 stk = 0;
-      int lsp = 0, npend = 0, nb = 0, ne = 0, rel = 0, maxrel = 0;
+      int nb = 0, ne = 0, rel = 0, minrel = 0, maxrel = 0;
       bool bad = false;
 #pragma unroll
       for (int k = 0; k < E; ++k) {
-        if (valid & (1u << k)) {
+        const int e = tid * E + k;
+        tags[k] = e < tn ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;  // all ones = no event
+        accb[e] = 0;
+        (&sm.bm[0][0])[e] = 0;  // kLevelWindow * NWORDS == T words
+        if (tags[k] != 0xffffffffu) {
           if ((tags[k] >> 1) >= a.num_regions) bad = true;
-          if (tags[k] & 1u) {
-            ++ne; --rel;
-            if (lsp > 0) { stk >>= 4; --lsp; } else { ++npend; }
-          } else {
-            ++nb; ++rel;
-            stk = (stk << 4) | (u64)k; ++lsp;
-            maxrel = rel > maxrel ? rel : maxrel;
-          }
+          if (tags[k] & 1u) { ++ne; --rel; minrel = rel < minrel ? rel : minrel; }
+          else { ++nb; ++rel; maxrel = rel > maxrel ? rel : maxrel; }
         }
       }
-      // zero the per-tile tables before the scan's barrier
-      sm.mask[tid / NW][tid % NW] = 0;
-      if (tid < kLevelWindow) sm.wmask[tid] = 0;
+      if (tid < kLevelWindow) sm.summ[tid] = 0;
       if (tid == 0) { sm.bad = 0; sm.failed = 0; accb[cbase + kSink] = 0; }
       // block prefix sum of (begins, ends), 16 bits each: one barrier
       const u32 mine_cnt = (u32)nb | ((u32)ne << 16);
@@ -227,143 +227,71 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       const u32 ex = before + incl_cnt - mine_cnt;
       const int tile_nb = (int)(tot & 0xffffu), tile_ne = (int)(tot >> 16);
       const int h0 = ch + (int)(ex & 0xffffu) - (int)(ex >> 16);
-      const int rank0 = (int)(ex >> 16);
-      const int hend = h0 + nb - ne;
       const int lbase = ch > 16 ? ch - 16 : 0;
-      if (h0 - npend < 0 || h0 + maxrel > ARGUS_MAX_DEPTH || tile_ne > MAXI) bad = true;
-      const int olo = lsp > 0 ? hend - lsp - lbase : 1000;  // levels of the begins this thread leaves open
-      const int ohi = lsp > 0 ? hend - lbase : -1000;       // (relative to lbase, half-open)
-      if (lsp > 0 && (olo < 0 || ohi > kLevelWindow)) bad = true;
-      const u64 opens_reg = stk;
-      sm.opens[tid] = stk;
-      sm.hend[tid] = hend;
-      u32 mine = 0;  // lane l: threads of this warp that leave a begin open at level lbase + l
-      {
-        int wlo = __reduce_min_sync(0xffffffffu, olo), whi = __reduce_max_sync(0xffffffffu, ohi);
-        wlo = wlo < 0 ? 0 : wlo;
-        whi = whi > kLevelWindow ? kLevelWindow : whi;
-        for (int l = wlo; l < whi; ++l) {
-          const u32 bal = __ballot_sync(0xffffffffu, l >= olo && l < ohi);
-          if (lane == l) mine = bal;
-        }
-        if (mine) {
-          sm.mask[lane][warp] = mine;
-          atomicOr(&sm.wmask[lane], 1u << warp);
-        }
-      }
+      // well nested so far: height never negative, never above the limit, begins inside the level window
+      if (h0 + minrel < 0 || h0 + maxrel > ARGUS_MAX_DEPTH || tile_ne > MAXI) bad = true;
+      if (nb > 0 && (h0 + minrel < lbase || h0 + maxrel > lbase + kLevelWindow)) bad = true;
       if (bad) sm.bad = 1;
-      __syncthreads();
-      {  // per (level, warp): the latest open begin among the warps before it
-        const int l = tid / NW, w = tid % NW;
-        const u32 wm = sm.wmask[l];
+      else {
+        int h = h0, rank = (int)(ex >> 16);
 #pragma unroll
-        for (int pass = 0; pass < 2; ++pass) {
-          const int wq = pass ? NW : w;
-          if (pass && w != NW - 1) break;
-          const u32 ww = wm & ((1u << wq) - 1u);
-          int e = -1;
-          if (ww) {
-            const int wp = 31 - __clz(ww);
-            const u32 m = sm.mask[l][wp];
-            if (m) {
-              const int tau = wp * 32 + 31 - __clz(m);
-              const int sh = 4 * (sm.hend[tau] - 1 - (lbase + l));
-              e = tau * E + (int)((sm.opens[tau] >> (sh & 63)) & 15ull);
-            }
+        for (int k = 0; k < E; ++k) {
+          if (tags[k] == 0xffffffffu) continue;
+          const int e = tid * E + k;
+          if (tags[k] & 1u) {
+            --h;
+            sm.desc[rank++] = (u32)e | ((u32)h << 16);
+          } else {
+            const int l = h - lbase;
+            atomicOr(&sm.bm[l][e >> 5], 1u << (e & 31));
+            atomicOr(reinterpret_cast<u32*>(&sm.summ[l]) + (e >> 10), 1u << ((e >> 5) & 31));
+            ++h;
           }
-          sm.prev[l][wq] = (short)e;
         }
       }
       __syncthreads();
       TT_MARK(2);
 
-      // ---------------- phase B1: one descriptor per end marker (who is my begin, who is my parent) -------------
-      const int nmax = __reduce_max_sync(0xffffffffu, npend);  // warp-wide: the loop below shuffles, so every lane runs it
-      // frames below this thread's floor, outermost needed first: level h0-1-j for j = 0..npend, 15 bits each
-      u64 outer_lo = 0, outer_hi = 0;
-      {
-        for (int j = 0; j <= nmax; ++j) {
-          const int L = h0 - 1 - j;
-          const int l = L - lbase;
-          const bool want = j <= npend && L >= 0 && l >= 0 && l < kLevelWindow;
-          // the mask word of my warp for level l sits in lane l's register
-          const u32 mword = __shfl_sync(0xffffffffu, mine, want ? l : 0);
-          const u32 m = want ? (mword & ((1u << lane) - 1u)) : 0u;
-          const int srcl = m ? 31 - __clz(m) : lane;
-          const int hend_s = __shfl_sync(0xffffffffu, hend, srcl);
-          const u64 opens_s = __shfl_sync(0xffffffffu, opens_reg, srcl);
-          int ref;
-          if (j > npend) ref = 0;
-          else if (L < 0) ref = cbase + kSink;
-          else {
-            if (m) ref = (warp * 32 + srcl) * E + (int)((opens_s >> ((4 * (hend_s - 1 - L)) & 63)) & 15ull);
-            else ref = want ? (int)sm.prev[l][warp] : -1;
-            if (ref < 0) ref = L < ch ? cbase + L : kBad;
-          }
-          const u64 v = (u64)((u32)ref & 0x7fffu);
-          if (j < 4) outer_lo |= v << (15 * j); else outer_hi |= v << (15 * ((j - 4) & 3));
-          if (j >= 8 && j <= npend) bad = true;  // more than 8 frames closed from outside: leave it to the redo path
-        }
-      }
-      if (!bad) {
-        int h = h0, rank = rank0, pi = 0;
-        stk = 0; lsp = 0;
-        auto outer_at = [&](int j) -> int {
-          const u64 w = j < 4 ? outer_lo : outer_hi;
-          int r = (int)((w >> (15 * (j & 3))) & 0x7fffull);
-          return (r & 0x4000) ? r - 0x8000 : r;  // sign-extend 15 bits (carried references of buffer 1 are negative)
-        };
-#pragma unroll
-        for (int k = 0; k < E; ++k) {
-          if (!(valid & (1u << k))) continue;
-          if (!(tags[k] & 1u)) {
-            stk = (stk << 4) | (u64)k; ++lsp; ++h;
-            continue;
-          }
-          --h;  // level of the frame this end closes
-          int partner, parent;
-          if (lsp > 0) {
-            partner = tid * E + (int)(stk & 15ull);
-            stk >>= 4; --lsp;
-            parent = lsp > 0 ? tid * E + (int)(stk & 15ull) : outer_at(pi);
-          } else {
-            partner = outer_at(pi);
-            ++pi;
-            parent = outer_at(pi);
-            if (h < 0) bad = true;
-          }
-          if (partner == kBad || parent == kBad) bad = true;
-          sm.desc[rank++] = make_uint2((u32)(tid * E + k) | ((u32)partner << 16), ((u32)parent & 0xffffu) | ((u32)h << 16));
-        }
-        if (bad) sm.bad = 1;
-      }
-      __syncthreads();
-      TT_MARK(3);
-
-      // ---------------- phase B2a: one thread per end marker: inclusive time feeds the parent frame -------------
+      // ---------------- phase B: one thread per end marker: find begin and parent, feed the parent's child time -----
+      u32 refs[NI];
       if (!sm.bad) {
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
           const int rk = tid + i * NT;
+          refs[i] = 0;
           if (rk < tile_ne) {
-            const uint2 d = sm.desc[rk];
-            const uint4 ee = evb[d.x & 0xffffu];
-            const uint4 pe = evb[(int)(short)(d.x >> 16)];
-            if ((pe.z >> 1) != (ee.z >> 1) || (pe.z & 1u)) sm.bad = 1;
+            const u32 d = sm.desc[rk];
+            const int e = (int)(d & 0xffffu), L = (int)(d >> 16);
+            int partner = tile_latest_begin<NT, E>(sm, L, lbase, e);
+            int parent;
+            if (partner < 0) {  // opened in an earlier tile: so was its parent
+              partner = L < ch ? cbase + L : kBadRef;
+              parent = L == 0 ? cbase + kSink : cbase + L - 1;
+            } else if (L == 0) {
+              parent = cbase + kSink;
+            } else {
+              parent = tile_latest_begin<NT, E>(sm, L - 1, lbase, partner);
+              if (parent < 0) parent = L - 1 < ch ? cbase + L - 1 : kBadRef;
+            }
+            if (partner == kBadRef || parent == kBadRef) { sm.bad = 1; continue; }
+            const uint4 ee = evb[e];
+            const uint4 pe = evb[partner];
+            if ((pe.z >> 1) != (ee.z >> 1)) sm.bad = 1;
             const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
             if (ts > bts) {  // 64-bit add as two native 32-bit shared atomics; each carry is propagated exactly once
               const u64 dlt = ts - bts;
-              u32* p = reinterpret_cast<u32*>(&accb[(int)(short)(d.y & 0xffffu)]);
+              u32* p = reinterpret_cast<u32*>(&accb[parent]);
               const u32 lo32 = (u32)dlt, hi32 = (u32)(dlt >> 32);
               const u32 old = atomicAdd(p, lo32);
               if (hi32) atomicAdd(p + 1, hi32);
               if (old + lo32 < old) atomicAdd(p + 1, 1u);
             }
+            refs[i] = ((u32)partner & 0xffffu) | ((u32)parent << 16);
           }
         }
       }
       __syncthreads();
-      TT_MARK(4);
+      TT_MARK(3);
       const bool tile_bad = sm.bad != 0;
       if (sm.dead) {  // a bulk copy never arrived: report and leave (uniform decision)
         if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
@@ -371,15 +299,15 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       }
 
       if (!tile_bad) {
-        // ---------------- phase B2b: exclusive time, parent region, interval records; carried stack -------------
+        // ---------------- phase C: exclusive time, parent region, interval records; carried stack -------------
         const u64 pos0 = out_base + n_int;
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
           const int rk = tid + i * NT;
           if (rk < tile_ne) {
-            const uint2 d = sm.desc[rk];
-            const int partner = (int)(short)(d.x >> 16), parent = (int)(short)(d.y & 0xffffu);
-            const uint4 ee = evb[d.x & 0xffffu];
+            const u32 d = sm.desc[rk];
+            const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
+            const uint4 ee = evb[d & 0xffffu];
             const uint4 pe = evb[partner];
             const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
             const u64 child = accb[partner];
@@ -396,7 +324,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               uint4* q = reinterpret_cast<uint4*>(a.intervals + pos);
               q[0] = make_uint4(pe.x, pe.y, (u32)incl, (u32)(incl >> 32));
               q[1] = make_uint4((u32)excl, (u32)(excl >> 32), pe.z >> 1, pe.w);
-              q[2] = make_uint4(s, preg, bidx, (d.y >> 16) | (flags << 16));
+              q[2] = make_uint4(s, preg, bidx, (d >> 16) | (flags << 16));
             } else if (!a.redo) {
               a.ctl->spec_overflow = 1;
             }
@@ -404,8 +332,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         }
         const int new_ch = ch + tile_nb - tile_ne;
         if (tid < new_ch) {  // the stack this tile leaves behind, in the next tile's index space
-          const int l = tid - lbase;
-          const int e = (l >= 0 && l < kLevelWindow) ? (int)sm.prev[l][NW] : -1;
+          const int e = tile_latest_begin<NT, E>(sm, tid, lbase, T);
           const int from = e >= 0 ? e : cbase + tid;
           car_next[tid] = evb[from];
           accb[nbase + tid] = accb[from];
@@ -415,7 +342,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         ch = new_ch;
         n_int += (u64)tile_ne;
         __syncthreads();
-        TT_MARK(5);
+        TT_MARK(4);
       } else {
         // ---------------- redo this tile with the sequential stack machine ----------------
         if (tid < ch) {
@@ -490,6 +417,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     }
   }
 }
+
 template <int NT, int E, int MINB>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   static int grid_cache = 0;
@@ -516,7 +444,7 @@ int g_variant = 0;
 bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0; }
 
 #ifdef ARGUS_TILE_TIMING
-// Debug build only: cycles thread 0 of every CTA spent per phase (other, wait, A, B1, B2a, B2b), summed; resets them.
+// Debug build only: cycles thread 0 of every CTA spent per phase (other, wait, A, B, C), summed; resets them.
 extern "C" int argus_debug_tile_timing(unsigned long long* out8) {
   if (cudaMemcpyFromSymbol(out8, g_tile_timing, 64) != cudaSuccess) return ARGUS_ERR_CUDA;
   unsigned long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -530,14 +458,14 @@ extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   switch (g_variant) {
-    case 1: return launch_tiled<128, 7, 4>(a, stream);
-    case 2: return launch_tiled<128, 9, 4>(a, stream);
-    case 3: return launch_tiled<256, 7, 2>(a, stream);
-    case 4: return launch_tiled<128, 5, 6>(a, stream);
-    case 5: return launch_tiled<128, 11, 3>(a, stream);
-    case 6: return launch_tiled<256, 9, 2>(a, stream);
-    case 7: return launch_tiled<128, 5, 5>(a, stream);
-    case 8: return launch_tiled<64, 9, 8>(a, stream);
+    case 1: return launch_tiled<128, 8, 4>(a, stream);
+    case 2: return launch_tiled<256, 8, 2>(a, stream);
+    case 3: return launch_tiled<256, 6, 2>(a, stream);
+    case 4: return launch_tiled<128, 4, 6>(a, stream);
+    case 5: return launch_tiled<128, 6, 5>(a, stream);
+    case 6: return launch_tiled<256, 4, 3>(a, stream);
+    case 7: return launch_tiled<512, 4, 1>(a, stream);
+    case 8: return launch_tiled<64, 8, 8>(a, stream);
     default: return launch_tiled<256, 5, 3>(a, stream);
   }
 }
