@@ -243,6 +243,38 @@ int argus_overlap(const argus_interval_t* intervals /*device*/, uint64_t max_int
                   argus_status_t* status /*device*/, void* workspace /*device*/,
                   size_t workspace_bytes, void* cuda_stream);
 
+/* ---------------------------------------------------------------------------------------
+ * argus_synthesize — the three operations above in one call, with identical results
+ * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
+ *
+ * Arguments have the meaning they have in argus_pair_intervals, argus_aggregate and
+ * argus_overlap. When num_regions <= 256 the pairing kernel aggregates every interval and
+ * selects the overlap spans while the interval is still in registers, so the interval array
+ * is written once and never read back; otherwise the three operations run one after the
+ * other. Any of the four tables may be NULL; num_pairs may be 0. max_overlap_spans bounds
+ * the spans selected for overlap over all pairs (an interval counts once per pair and role
+ * its region appears in); more than that -> ARGUS_ERR_CAPACITY with the count in
+ * status->intervals_required. One status block reports the first error of any stage.
+ * ------------------------------------------------------------------------------------- */
+size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t num_streams,
+                                        uint32_t num_regions, uint64_t ambig_capacity,
+                                        uint32_t num_pairs, uint32_t num_sms,
+                                        uint64_t max_overlap_spans);
+
+int argus_synthesize(const argus_event_t* events /*device*/, uint64_t num_events,
+                     const uint64_t* stream_offsets /*device [S+1]*/, uint32_t num_streams,
+                     uint32_t num_regions, argus_interval_t* intervals /*device*/,
+                     uint64_t interval_capacity, uint64_t* interval_offsets /*device [S+1] out*/,
+                     argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
+                     uint64_t* ambig_offsets /*device [S+1] out*/, uint32_t warps_per_cta,
+                     const uint32_t* cta_sm /*device [C]*/, uint32_t num_sms,
+                     argus_agg_t* warp_tab /*device, nullable*/, argus_agg_t* cta_tab /*device, nullable*/,
+                     argus_agg_t* sm_tab /*device, nullable*/, argus_agg_t* kernel_tab /*device, nullable*/,
+                     const uint32_t* pairs /*device [K][2]*/, uint32_t num_pairs,
+                     argus_overlap_t* overlap_out /*device [K][M]*/, uint64_t max_overlap_spans,
+                     argus_status_t* status /*device*/, void* workspace /*device*/,
+                     size_t workspace_bytes, void* cuda_stream);
+
 /* Copies the device status block to host memory and synchronises `cuda_stream`.
  * Returns ARGUS_OK or ARGUS_ERR_CUDA; the device-side code is in host_copy->code. */
 int argus_status_fetch(const argus_status_t* dev_status, argus_status_t* host_copy,

@@ -8,12 +8,14 @@ from .binding import (AGG_DTYPE, AMBIG_DTYPE, EVENT_DTYPE, INTERVAL_DTYPE, OVERL
                       AggregateResult, PairResult, argus_aggregate, argus_aggregate_workspace_bytes, argus_overlap,
                       argus_overlap_workspace_bytes, argus_pair_intervals, argus_pair_workspace_bytes,
                       argus_launch_count, argus_profile_enable, argus_profile_read, argus_status_fetch, argus_strerror,
-                      argus_version, library_path, load_library, pair_aggregate_host)
+                      argus_version, library_path, load_library, pair_aggregate_host, argus_synthesize,
+                      argus_synthesize_workspace_bytes, SynthesizeResult)
 
 __all__ = [
     "AGG_DTYPE", "AMBIG_DTYPE", "EVENT_DTYPE", "INTERVAL_DTYPE", "OVERLAP_DTYPE", "STATUS_DTYPE", "ArgusError",
     "AggregateResult", "PairResult", "argus_aggregate", "argus_aggregate_workspace_bytes", "argus_overlap",
     "argus_overlap_workspace_bytes", "argus_pair_intervals", "argus_pair_workspace_bytes", "argus_status_fetch",
     "argus_strerror", "argus_version", "library_path", "load_library", "pair_aggregate_host", "argus_launch_count",
-    "argus_profile_enable", "argus_profile_read",
+    "argus_profile_enable", "argus_profile_read", "argus_synthesize", "argus_synthesize_workspace_bytes",
+    "SynthesizeResult",
 ]

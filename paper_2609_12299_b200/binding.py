@@ -259,6 +259,72 @@ def argus_overlap(intervals: torch.Tensor, max_intervals: int, interval_offsets:
     return out, status
 
 
+@dataclass
+class SynthesizeResult:
+    pair: PairResult
+    agg: AggregateResult
+    overlap: torch.Tensor | None   # uint8 [K * M * 32]
+    status: torch.Tensor
+    workspace: torch.Tensor
+    max_overlap_spans: int
+
+    def fetch_status(self):
+        return argus_status_fetch(self.status)
+
+    def overlap_numpy(self, num_sms: int) -> np.ndarray:
+        return self.overlap.cpu().numpy().view(OVERLAP_DTYPE).reshape(-1, num_sms)
+
+
+def argus_synthesize_workspace_bytes(num_events: int, num_streams: int, num_regions: int, ambig_capacity: int,
+                                     num_pairs: int, num_sms: int, max_overlap_spans: int) -> int:
+    lib = load_library()
+    lib.argus_synthesize_workspace_bytes.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64,
+                                                     ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64]
+    lib.argus_synthesize_workspace_bytes.restype = ctypes.c_size_t
+    return lib.argus_synthesize_workspace_bytes(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms,
+                                                max_overlap_spans)
+
+
+def argus_synthesize(events: torch.Tensor, stream_offsets: torch.Tensor, num_regions: int, warps_per_cta: int,
+                     cta_sm: torch.Tensor, num_sms: int, pairs: torch.Tensor | None = None,
+                     interval_capacity: int | None = None, ambig_capacity: int | None = None,
+                     max_overlap_spans: int | None = None, levels=("warp", "cta", "sm", "kernel"),
+                     out: SynthesizeResult | None = None) -> SynthesizeResult:
+    """Whole hot path in one call (pair -> aggregate -> overlap); enqueues on the current stream."""
+    lib = load_library()
+    vp, u32, u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
+    lib.argus_synthesize.argtypes = [vp, u64, vp, u32, u32, vp, u64, vp, vp, u64, vp, u32, vp, u32, vp, vp, vp, vp, vp, u32,
+                                     vp, u64, vp, vp, ctypes.c_size_t, vp]
+    lib.argus_synthesize.restype = ctypes.c_int
+    dev = events.device
+    n = events.numel() * events.element_size() // 16
+    S = stream_offsets.numel() - 1
+    K = 0 if pairs is None else pairs.numel() // 2
+    if out is None:
+        icap = n // 2 if interval_capacity is None else int(interval_capacity)
+        acap = n if ambig_capacity is None else int(ambig_capacity)
+        mos = (2 * K * icap if max_overlap_spans is None else int(max_overlap_spans)) if K else 0
+        C = S // warps_per_cta if warps_per_cta else 0
+        keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1}
+        tabs = {lv: (_bytes(keys[lv] * num_regions * 576, dev) if lv in levels else None) for lv in keys}
+        status = _bytes(64, dev)
+        pr = PairResult(_bytes(icap * 48, dev), torch.empty(S + 1, dtype=torch.int64, device=dev), _bytes(acap * 32, dev),
+                        torch.empty(S + 1, dtype=torch.int64, device=dev), status, icap, acap, _bytes(1, dev))
+        ag = AggregateResult(tabs["warp"], tabs["cta"], tabs["sm"], tabs["kernel"], status, _bytes(1, dev),
+                             {lv: (keys[lv], num_regions) for lv in keys})
+        ws = _bytes(argus_synthesize_workspace_bytes(n, S, num_regions, acap, K, num_sms, mos), dev)
+        out = SynthesizeResult(pr, ag, _bytes(K * num_sms * 32, dev) if K else None, status, ws, mos)
+    p, a = out.pair, out.agg
+    rc = lib.argus_synthesize(_ptr(events), n, _ptr(stream_offsets), S, num_regions, _ptr(p.intervals), p.interval_capacity,
+                              _ptr(p.interval_offsets), _ptr(p.ambig), p.ambig_capacity, _ptr(p.ambig_offsets), warps_per_cta,
+                              _ptr(cta_sm), num_sms, _ptr(a.warp), _ptr(a.cta), _ptr(a.sm), _ptr(a.kernel), _ptr(pairs), K,
+                              _ptr(out.overlap), out.max_overlap_spans, _ptr(out.status), _ptr(out.workspace),
+                              out.workspace.numel(), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_synthesize")
+    return out
+
+
 def pair_aggregate_host(events: np.ndarray, stream_offsets: np.ndarray, num_regions: int, warps_per_cta: int,
                         cta_sm: np.ndarray, num_sms: int, device="cuda:0", state: dict | None = None):
     """End-to-end call with HOST buffers: copies the events (and offsets) to the device, runs

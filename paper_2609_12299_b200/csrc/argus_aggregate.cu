@@ -126,6 +126,19 @@ __global__ void __launch_bounds__(256) k_agg_scatter(AggArgs a) {
   }
 }
 
+// ambiguity counters into the warp-scope table (used when the intervals were aggregated by the pairing kernel)
+__global__ void __launch_bounds__(256) k_agg_ambig(AggArgs a) {
+  for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
+    const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
+    u64* row = a.warp_tab + (size_t)s * a.num_regions * kCell;
+    for (u64 i = alo + threadIdx.x; i < ahi && ahi >= alo; i += blockDim.x) {
+      const u32 region = a.ambig[i].tag >> 1;
+      if (region >= a.num_regions) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
+      atomicAdd(row + (size_t)region * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
+    }
+  }
+}
+
 struct AggLayout { size_t warp, cta, total; };
 
 AggLayout agg_layout(uint32_t num_streams, uint32_t num_regions) {
@@ -139,15 +152,52 @@ AggLayout agg_layout(uint32_t num_streams, uint32_t num_regions) {
 
 }  // namespace
 
+// Roll-up of a filled warp-scope table into the CTA, SM and kernel scopes.
+static int agg_rollup(AggArgs& a, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab, cudaStream_t stream) {
+  if (cta_tab || sm_tab || kernel_tab) {
+    k_agg_cta<<<1184, 256, 0, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  if (sm_tab || kernel_tab) {
+    if (sm_tab) { k_agg_init<<<296, 256, 0, stream>>>(a.sm_tab, (u64)a.num_sms * a.num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
+    if (kernel_tab) { k_agg_init<<<16, 256, 0, stream>>>(a.kernel_tab, (u64)a.num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
+    k_agg_scatter<<<1184, 256, 0, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  return ARGUS_OK;
+}
+
+// Second half of aggregation when the pairing kernel already filled the interval statistics of
+// warp_tab: ambiguity counters, then the roll-up. warp_tab and cta_work must be non-null.
+int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                              argus_agg_t* warp_tab, argus_agg_t* cta_work, bool want_cta, argus_agg_t* sm_tab,
+                              argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream) {
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (num_streams == 0) return ARGUS_OK;
+  AggArgs a;
+  a.intervals = nullptr; a.interval_offsets = nullptr; a.ambig = ambig; a.ambig_offsets = (const u64*)ambig_offsets;
+  a.num_streams = num_streams; a.warps_per_cta = warps_per_cta; a.num_ctas = num_streams / warps_per_cta;
+  a.num_sms = num_sms; a.num_regions = num_regions; a.cta_sm = cta_sm;
+  a.warp_tab = (u64*)warp_tab; a.cta_tab = (u64*)cta_work; a.sm_tab = (u64*)sm_tab; a.kernel_tab = (u64*)kernel_tab;
+  a.status = status; a.use_smem = 0;
+  if (ambig && ambig_offsets) {
+    k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  return agg_rollup(a, want_cta || sm_tab || kernel_tab ? cta_work : nullptr, sm_tab, kernel_tab, stream);
+}
+
 extern "C" size_t argus_aggregate_workspace_bytes(uint64_t /*num_intervals*/, uint32_t num_streams, uint32_t num_regions) {
   return agg_layout(num_streams, num_regions).total + 256;
 }
 
-extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
-                               const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                               uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                               argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
-                               argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                             const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                             uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                             argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
+                             argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                             bool reset_status) {
   if (!interval_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
@@ -158,7 +208,7 @@ extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t
   const AggLayout L = agg_layout(num_streams, num_regions);
   if (workspace_bytes < L.total) return ARGUS_ERR_WORKSPACE;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
+  if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
   if (num_streams == 0) {
     if (kernel_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)kernel_tab, (u64)num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
     if (sm_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)sm_tab, (u64)num_sms * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
@@ -179,15 +229,15 @@ extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t
   k_agg_streams<<<num_streams, kAggThreads, a.use_smem ? smem : 0, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 1);
-  if (cta_tab || sm_tab || kernel_tab) {
-    k_agg_cta<<<1184, 256, 0, stream>>>(a);
-    ARGUS_CHECK_LAUNCH();
-  }
-  if (sm_tab || kernel_tab) {
-    if (sm_tab) { k_agg_init<<<296, 256, 0, stream>>>(a.sm_tab, (u64)num_sms * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
-    if (kernel_tab) { k_agg_init<<<16, 256, 0, stream>>>(a.kernel_tab, (u64)num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
-    k_agg_scatter<<<1184, 256, 0, stream>>>(a);
-    ARGUS_CHECK_LAUNCH();
-  }
-  return ARGUS_OK;
+  return agg_rollup(a, cta_tab, sm_tab, kernel_tab, stream);
+}
+
+extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                               const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                               uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                               argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
+                               argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return argus_internal_aggregate(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
+                                  num_sms, num_regions, warp_tab, cta_tab, sm_tab, kernel_tab, status, workspace,
+                                  workspace_bytes, cuda_stream, true);
 }

@@ -1,0 +1,132 @@
+// argus_fuse.cuh — per-interval hooks that let the pairing kernel feed aggregation and overlap
+// selection while the interval is still in registers (no second read of the interval array).
+//
+// Aggregation: the CTA that walks a stream keeps that stream's row of the warp-scope table in
+// shared memory in a compact form (per region: sums, min, max, counts and a 16-bin window of the
+// 64-bin log2 histogram; bins outside the window go straight to the global row) and writes it to
+// the global row when the stream ends. All updates are integer atomics, so thread order is irrelevant.
+// Overlap: spans of intervals whose region appears in a (producer, consumer) pair are appended to a
+// global list tagged with their (pair, SM, role) segment; the overlap kernels take it from there.
+#ifndef ARGUS_FUSE_CUH_
+#define ARGUS_FUSE_CUH_
+
+#include "argus_common.cuh"
+
+constexpr u32 kAggWindow = 16;          // histogram bins kept in shared memory per region
+constexpr u32 kAggUnset = 0xffffffffu;  // window base not chosen yet
+constexpr u32 kFuseMaxRegions = 256;    // fused aggregation keeps num_regions * 112 bytes in shared memory
+constexpr u32 kAggCellWords = 72;       // u64 words of one argus_agg_t
+
+struct ArgusAggCell {  // 112 bytes
+  u64 sum_incl, sum_excl, min_incl, max_incl;
+  u32 count, nflag, hbase, pad;
+  u32 h[kAggWindow];
+};
+
+struct ArgusFuseArgs {
+  u64* warp_tab;          // [S][R][72], zeroed before the kernel; null = no fused aggregation
+  const u32* cta_sm;      // [C]
+  u32 warps_per_cta, num_sms;
+  const u32* pairs;       // [K][2]
+  u32 num_pairs;
+  ulonglong2* ov_spans;   // appended (start, end); null = no fused overlap selection
+  u32* ov_seg;            // segment of each appended span: (pair * num_sms + sm) * 2 + role
+  u64 ov_capacity;
+  u64* ov_count;          // spans appended so far (may exceed the capacity)
+};
+
+struct ArgusFuseCtx {     // per CTA, for the stream it is walking
+  ArgusAggCell* tab;      // shared memory [R]; null = aggregation off
+  const u32* pairbits;    // shared memory bitmap over regions: region appears in some pair; null = overlap off
+  u64* row;               // global row of this stream in the warp-scope table
+  u32 sm_index;           // SM of this stream's CTA
+};
+
+__device__ __forceinline__ u32 argus_log2_bin(u64 d) { return d ? 63u - (u32)__clzll((long long)d) : 0u; }
+
+// 64-bit add as native 32-bit atomics; each carry is propagated exactly once
+__device__ __forceinline__ void argus_atomic_add64_split(u64* p64, u64 v) {
+  u32* p = reinterpret_cast<u32*>(p64);
+  const u32 lo = (u32)v, hi = (u32)(v >> 32);
+  if (lo) {
+    const u32 old = atomicAdd(p, lo);
+    if (old + lo < old) atomicAdd(p + 1, 1u);
+  }
+  if (hi) atomicAdd(p + 1, hi);
+}
+
+__device__ __forceinline__ void argus_fuse_init(ArgusAggCell* tab, u32 num_regions, u32 tid, u32 nthreads) {
+  u32* w = reinterpret_cast<u32*>(tab);
+  constexpr u32 kWords = sizeof(ArgusAggCell) / 4;
+  for (u32 i = tid; i < num_regions * kWords; i += nthreads) {
+    const u32 f = i % kWords;
+    w[i] = (f == 4 || f == 5 || f == 10) ? 0xffffffffu : 0u;  // min_incl = all ones, hbase = unset
+  }
+}
+
+__device__ __forceinline__ void argus_fuse_aggregate(const ArgusFuseCtx& fx, u32 region, u64 incl, u64 excl, u32 flags) {
+  ArgusAggCell& c = fx.tab[region];
+  atomicAdd(&c.count, 1u);
+  argus_atomic_add64_split(&c.sum_incl, incl);
+  argus_atomic_add64_split(&c.sum_excl, excl);
+  if (incl < *reinterpret_cast<volatile u64*>(&c.min_incl)) atomicMin(&c.min_incl, incl);
+  if (incl > *reinterpret_cast<volatile u64*>(&c.max_incl)) atomicMax(&c.max_incl, incl);
+  if (flags) atomicAdd(&c.nflag, 1u);
+  const u32 bin = argus_log2_bin(incl);
+  u32 hb = *reinterpret_cast<volatile u32*>(&c.hbase);
+  if (hb == kAggUnset) {
+    const u32 want = bin > 6u ? (bin - 6u > 64u - kAggWindow ? 64u - kAggWindow : bin - 6u) : 0u;
+    const u32 old = atomicCAS(&c.hbase, kAggUnset, want);
+    hb = old == kAggUnset ? want : old;
+  }
+  const u32 rel = bin - hb;
+  if (rel < kAggWindow) atomicAdd(&c.h[rel], 1u);
+  else atomicAdd(fx.row + (size_t)region * kAggCellWords + 8 + bin, 1ull);
+}
+
+__device__ __forceinline__ void argus_fuse_flush(const ArgusFuseCtx& fx, u32 num_regions, u32 tid, u32 nthreads) {
+  constexpr u32 kItems = 8 + kAggWindow;
+  for (u32 i = tid; i < num_regions * kItems; i += nthreads) {
+    const u32 r = i / kItems, f = i % kItems;
+    const ArgusAggCell& c = fx.tab[r];
+    u64* cell = fx.row + (size_t)r * kAggCellWords;
+    switch (f) {
+      case 0: cell[0] = c.count; break;
+      case 1: cell[1] = c.sum_incl; break;
+      case 2: cell[2] = c.min_incl; break;
+      case 3: cell[3] = c.max_incl; break;
+      case 4: cell[4] = c.sum_excl; break;
+      case 5: case 6: break;  // ambiguity counters are added later from the ambiguity records
+      case 7: cell[7] = c.nflag; break;
+      default: {
+        const u32 j = f - 8;
+        if (c.h[j]) atomicAdd(cell + 8 + c.hbase + j, (u64)c.h[j]);
+      }
+    }
+  }
+}
+
+// Appends the span of a selected interval once per (pair, role) it takes part in.
+__device__ __forceinline__ void argus_fuse_overlap(const ArgusFuseArgs& f, const ArgusFuseCtx& fx, u32 region, u64 t_begin,
+                                                   u64 incl) {
+  if (!incl || !((fx.pairbits[region >> 5] >> (region & 31)) & 1u)) return;
+  for (u32 k = 0; k < f.num_pairs; ++k) {
+#pragma unroll
+    for (u32 role = 0; role < 2; ++role) {
+      if (f.pairs[2 * k + role] != region) continue;
+      const u64 slot = atomicAdd(f.ov_count, 1ull);
+      if (slot < f.ov_capacity) {
+        f.ov_spans[slot] = make_ulonglong2(t_begin, t_begin + incl);
+        f.ov_seg[slot] = (k * f.num_sms + fx.sm_index) * 2 + role;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void argus_fuse_emit(const ArgusFuseArgs& f, const ArgusFuseCtx& fx, u32 region, u64 t_begin,
+                                                u64 incl, u64 excl, u32 flags) {
+  if (fx.tab) argus_fuse_aggregate(fx, region, incl, excl, flags);
+  if (fx.pairbits) argus_fuse_overlap(f, fx, region, t_begin, incl);
+}
+
+#endif  // ARGUS_FUSE_CUH_

@@ -73,6 +73,35 @@ __global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatt
   }
 }
 
+// Same two roles for spans that the pairing kernel already selected: list entries carry their segment;
+// entries of reserved but unused slots have segment 0xffffffff.
+struct OvList {
+  const ulonglong2* spans;
+  const u32* seg;
+  const u64* count;  // slots reserved (may exceed capacity)
+  u64 capacity;
+};
+
+__global__ void __launch_bounds__(256) k_ov_list_count_or_scatter(OvArgs a, OvList l, int scatter) {
+  if (scatter && a.status->code != 0) return;
+  const u64 reserved = *l.count;
+  if (reserved > l.capacity && blockIdx.x == 0 && threadIdx.x == 0) {
+    argus_set_error(a.status, ARGUS_ERR_CAPACITY, 0, reserved);
+    a.status->intervals_required = reserved;
+  }
+  const u64 n = reserved < l.capacity ? reserved : l.capacity;
+  for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (u64)gridDim.x * blockDim.x) {
+    const u32 seg = l.seg[i];
+    if (seg >= a.nseg) continue;
+    if (!scatter) {
+      atomicAdd(&a.seg_count[seg], 1ull);
+    } else {
+      const u64 slot = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], 1ull);
+      if (slot < a.capacity) a.spans[slot] = l.spans[i];
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kOvThreads) k_ov_scan(OvArgs a) {
   __shared__ u64 sh[33];
   u64 carry = 0;
@@ -250,25 +279,40 @@ extern "C" size_t argus_overlap_workspace_bytes(uint64_t max_intervals, uint32_t
   return L.total_fixed + argus_align_up((size_t)max_intervals * 2 * num_pairs * 24 + 256, 256);
 }
 
-extern "C" int argus_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
-                             uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
-                             const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
-                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  if (!interval_offsets || !cta_sm || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
-  if (warps_per_cta == 0 || num_streams % warps_per_cta != 0 || num_sms == 0) return ARGUS_ERR_INVALID_ARG;
-  if (num_pairs > kMaxPairs || (num_pairs && (!pairs || !out))) return ARGUS_ERR_INVALID_ARG;
-  if ((max_intervals && !intervals) || ((uintptr_t)intervals & 15) || ((uintptr_t)workspace & 255) || ((uintptr_t)out & 7))
-    return ARGUS_ERR_INVALID_ARG;
-  if ((uint64_t)num_pairs * num_sms * 2 > 0x7fffffffull) return ARGUS_ERR_INVALID_ARG;
-  cudaStream_t stream = (cudaStream_t)cuda_stream;
-  ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
-  if (num_pairs == 0) return ARGUS_OK;
+// Shared tail of both entry paths. `list` null: spans are selected from the interval array;
+// otherwise they come from the list the pairing kernel appended.
+static int ov_run(OvArgs& a, const OvList* list, cudaStream_t stream) {
+  const unsigned sel_grid = a.num_streams < 2368 ? (a.num_streams ? a.num_streams : 1) : 2368;
+  for (int pass = 0; pass < 2; ++pass) {
+    if (list) {
+      k_ov_list_count_or_scatter<<<592, 256, 0, stream>>>(a, *list, pass);
+      ARGUS_CHECK_LAUNCH();
+    } else if (a.num_streams) {
+      k_ov_count_or_scatter<<<sel_grid, 256, 0, stream>>>(a, pass);
+      ARGUS_CHECK_LAUNCH();
+    }
+    if (pass == 0) {
+      k_ov_scan<<<1, kOvThreads, 0, stream>>>(a);
+      ARGUS_CHECK_LAUNCH();
+    }
+  }
+  argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 0);
+  k_ov_sort<<<a.nseg, kOvThreads, 0, stream>>>(a);
+  ARGUS_CHECK_LAUNCH();
+  argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 1);
+  k_ov_measure<<<a.nseg / 2, 256, 0, stream>>>(a);
+  ARGUS_CHECK_LAUNCH();
+  return ARGUS_OK;
+}
+
+static int ov_setup(OvArgs& a, uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                    const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status, void* workspace,
+                    size_t workspace_bytes, cudaStream_t stream) {
   const u32 nseg = num_pairs * num_sms * 2;
   const OvLayout L = ov_layout(nseg);
   if (workspace_bytes < L.total_fixed + 256) return ARGUS_ERR_WORKSPACE;
   char* ws = (char*)workspace;
-  OvArgs a;
-  a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets; a.num_streams = num_streams;
+  a.intervals = nullptr; a.interval_offsets = nullptr; a.num_streams = num_streams;
   a.warps_per_cta = warps_per_cta; a.num_sms = num_sms; a.num_pairs = num_pairs; a.cta_sm = cta_sm; a.pairs = pairs;
   a.out = out; a.status = status;
   a.seg_count = (u64*)(ws + L.seg_count); a.seg_cursor = (u64*)(ws + L.seg_cursor); a.seg_base = (u64*)(ws + L.seg_base);
@@ -278,22 +322,48 @@ extern "C" int argus_overlap(const argus_interval_t* intervals, uint64_t max_int
   a.nseg = nseg;
   ARGUS_CUDA_TRY(cudaMemsetAsync(ws, 0, L.seg_base, stream));
   ARGUS_CUDA_TRY(cudaMemsetAsync(out, 0, (size_t)num_pairs * num_sms * sizeof(argus_overlap_t), stream));
-  if (num_streams) {
-    k_ov_count_or_scatter<<<num_streams < 2368 ? num_streams : 2368, 256, 0, stream>>>(a, 0);
-    ARGUS_CHECK_LAUNCH();
-  }
-  k_ov_scan<<<1, kOvThreads, 0, stream>>>(a);
-  ARGUS_CHECK_LAUNCH();
-  if (num_streams) {
-    k_ov_count_or_scatter<<<num_streams < 2368 ? num_streams : 2368, 256, 0, stream>>>(a, 1);
-    ARGUS_CHECK_LAUNCH();
-  }
-  argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 0);
-  k_ov_sort<<<nseg, kOvThreads, 0, stream>>>(a);
-  ARGUS_CHECK_LAUNCH();
-  argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 1);
-  k_ov_measure<<<nseg / 2, 256, 0, stream>>>(a);
-  ARGUS_CHECK_LAUNCH();
-  (void)max_intervals;
   return ARGUS_OK;
+}
+
+// Overlap from a span list appended by the pairing kernel (see argus_fuse.cuh).
+int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* list_seg, const uint64_t* list_count,
+                                     uint64_t list_capacity, uint32_t num_sms, uint32_t num_pairs, argus_overlap_t* out,
+                                     argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (num_pairs == 0) return ARGUS_OK;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  OvArgs a;
+  const int rc = ov_setup(a, 0, 1, nullptr, num_sms, nullptr, num_pairs, out, status, workspace, workspace_bytes, stream);
+  if (rc != ARGUS_OK) return rc;
+  OvList l;
+  l.spans = (const ulonglong2*)list_spans; l.seg = list_seg; l.count = (const u64*)list_count; l.capacity = list_capacity;
+  return ov_run(a, &l, stream);
+}
+
+int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                           const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status) {
+  if (!interval_offsets || !cta_sm || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
+  if (warps_per_cta == 0 || num_streams % warps_per_cta != 0 || num_sms == 0) return ARGUS_ERR_INVALID_ARG;
+  if (num_pairs > kMaxPairs || (num_pairs && (!pairs || !out))) return ARGUS_ERR_INVALID_ARG;
+  if ((max_intervals && !intervals) || ((uintptr_t)intervals & 15) || ((uintptr_t)workspace & 255) || ((uintptr_t)out & 7))
+    return ARGUS_ERR_INVALID_ARG;
+  if ((uint64_t)num_pairs * num_sms * 2 > 0x7fffffffull) return ARGUS_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
+  if (num_pairs == 0) return ARGUS_OK;
+  OvArgs a;
+  const int rc = ov_setup(a, num_streams, warps_per_cta, cta_sm, num_sms, pairs, num_pairs, out, status, workspace,
+                          workspace_bytes, stream);
+  if (rc != ARGUS_OK) return rc;
+  a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets;
+  return ov_run(a, nullptr, stream);
+}
+
+extern "C" int argus_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                             uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                             const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return argus_internal_overlap(intervals, max_intervals, interval_offsets, num_streams, warps_per_cta, cta_sm, num_sms,
+                                pairs, num_pairs, out, status, workspace, workspace_bytes, cuda_stream, true);
 }

@@ -10,6 +10,8 @@
 //   ambiguity     : popcount prefix over the bitmap -> rank of every note -> ordered records, offsets
 #include "argus_pair_common.cuh"
 
+#include <string.h>
+
 namespace {
 
 constexpr int kScanThreads = 1024;
@@ -198,17 +200,21 @@ Layout make_layout(uint64_t num_events, uint32_t num_streams, uint64_t ambig_cap
 // implemented in argus_pair_tiled.cu
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream);
 bool argus_pair_tiled_usable(const ArgusPairArgs& a);
+bool argus_pair_tiled_can_fuse(uint32_t num_regions);
 
 extern "C" size_t argus_pair_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint64_t ambig_capacity) {
   return make_layout(num_events, num_streams, ambig_capacity).total;
 }
 
-// kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled
-extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
-                                       uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
-                                       uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
-                                       uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status,
-                                       void* workspace, size_t workspace_bytes, void* cuda_stream, int kernel_choice) {
+// Whole pairing pipeline. kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled.
+// `fuse` (nullable) asks the tiled kernel to feed aggregation / overlap selection; *fused_out tells the
+// caller whether it did (only the tiled kernel can).
+int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                        uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                        uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                        uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
+                        bool reset_status, bool* fused_out) {
   if (!stream_offsets || !interval_offsets || !ambig_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if ((num_events && !events) || (interval_capacity && !intervals) || (ambig_capacity && !ambig)) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
@@ -232,12 +238,16 @@ extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num
   a.ctl = (ArgusPairCtl*)(ws + L.ctl);
   a.status = status;
   a.redo = 0;
+  memset(&a.fuse, 0, sizeof(a.fuse));
 
-  ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
+  if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
   // control block, counts and bitmap are contiguous at the start of the workspace
   ARGUS_CUDA_TRY(cudaMemsetAsync(ws, 0, L.word_prefix, stream));
 
   const bool tiled = kernel_choice != 1 && argus_pair_tiled_usable(a);
+  const bool fused = tiled && fuse && argus_pair_tiled_can_fuse(num_regions);
+  if (fused) a.fuse = *fuse;
+  if (fused_out) *fused_out = fused;
   for (int pass = 0; pass < 2; ++pass) {
     a.redo = pass;
     if (num_streams) {
@@ -274,6 +284,16 @@ extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num
   k_ambig_offsets<<<(num_streams + 1 + 255) / 256, 256, 0, stream>>>(g);
   ARGUS_CHECK_LAUNCH();
   return ARGUS_OK;
+}
+
+extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                                       uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                                       uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                                       uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status,
+                                       void* workspace, size_t workspace_bytes, void* cuda_stream, int kernel_choice) {
+  return argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
+                             interval_offsets, ambig, ambig_capacity, ambig_offsets, status, workspace, workspace_bytes,
+                             cuda_stream, kernel_choice, nullptr, true, nullptr);
 }
 
 extern "C" int argus_pair_intervals(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,

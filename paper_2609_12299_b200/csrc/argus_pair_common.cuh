@@ -11,6 +11,7 @@
 #define ARGUS_PAIR_COMMON_CUH_
 
 #include "argus_common.cuh"
+#include "argus_fuse.cuh"
 
 struct ArgusFrame {  // one open region occurrence, 32 bytes
   u64 ts;
@@ -48,6 +49,7 @@ struct ArgusPairArgs {
   ArgusPairCtl* ctl;
   argus_status_t* status;
   int redo;               // 0 = first pass with provisional bases, 1 = second pass with final bases
+  ArgusFuseArgs fuse;     // optional aggregation / overlap selection fed from the pairing kernel (first pass only)
 };
 
 #define ARGUS_NOTE_POS_BITS 48
@@ -77,7 +79,8 @@ struct ArgusSeqState {
 // Processes one event exactly as the definition states. `stk` holds ARGUS_MAX_DEPTH frames.
 // `out_base` is the position of this stream's first interval. Returns false on a device error.
 __device__ __forceinline__ bool argus_seq_step(const ArgusPairArgs& a, ArgusFrame* stk, ArgusSeqState& s, u32 stream,
-                                               u64 stream_gpos0, u64 out_base, u32 i, u64 ts, u32 tag, u32 ctx) {
+                                               u64 stream_gpos0, u64 out_base, u32 i, u64 ts, u32 tag, u32 ctx,
+                                               const ArgusFuseCtx* fx = nullptr) {
   const u32 region = tag >> 1;
   if (region >= a.num_regions) {
     argus_set_error(a.status, ARGUS_ERR_BAD_REGION, stream, i);
@@ -119,6 +122,7 @@ __device__ __forceinline__ bool argus_seq_step(const ArgusPairArgs& a, ArgusFram
     a.ctl->spec_overflow = 1;
   }
   s.n_int++;
+  if (fx && !a.redo) argus_fuse_emit(a.fuse, *fx, f.region, f.ts, incl, excl, flags);
   if (s.h > 0) stk[s.h - 1].child += incl;
   return true;
 }

@@ -111,7 +111,9 @@ __device__ __forceinline__ int tile_latest_begin(const TileSmem<NT, E>& sm, int 
   return m2 ? w2 * 32 + 31 - __clz(m2) : -1;
 }
 
-template <int NT, int E, int MINB>
+constexpr u32 kOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
+
+template <int NT, int E, int MINB, bool FUSE>
 __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   using SM = TileSmem<NT, E>;
   constexpr int T = SM::T, NW = SM::NW, NWORDS = SM::NWORDS, MAXI = SM::MAXI, NI = SM::NI;
@@ -130,6 +132,26 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   u32 ph0 = 0, ph1 = 0;  // mbarrier phase parities
   const u64 off0 = a.stream_offsets[0];
   u32 tot_ctx = 0, tot_rev = 0, tot_clamp = 0;
+  // fused aggregation / overlap selection (first pass only): compact table and pair bitmap follow TileSmem
+  ArgusFuseCtx fx;
+  fx.tab = nullptr; fx.pairbits = nullptr; fx.row = nullptr; fx.sm_index = 0;
+  u64 ovc_base = 0;        // warp-uniform: current chunk of the global overlap span list
+  u32 ovc_used = kOvChunk;
+  if (FUSE && !a.redo) {
+    ArgusAggCell* tab = reinterpret_cast<ArgusAggCell*>(smem_raw + ((sizeof(SM) + 15) & ~(size_t)15));
+    u32* pairbits = reinterpret_cast<u32*>(tab + a.num_regions);
+    if (a.fuse.warp_tab) fx.tab = tab;
+    if (a.fuse.ov_spans && a.fuse.num_pairs) {
+      for (u32 i = tid; i < (a.num_regions + 31) / 32; i += NT) pairbits[i] = 0;
+      __syncthreads();
+      for (u32 i = tid; i < 2 * a.fuse.num_pairs; i += NT) {
+        const u32 r = a.fuse.pairs[i];
+        if (r < a.num_regions) atomicOr(&pairbits[r >> 5], 1u << (r & 31));
+      }
+      fx.pairbits = pairbits;
+      __syncthreads();
+    }
+  }
 #ifdef ARGUS_TILE_TIMING
   unsigned long long tt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   long long tlast = clock64();
@@ -158,6 +180,18 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     int ch = 0;          // carried stack height (uniform)
     u64 n_int = 0;       // intervals of this stream so far (uniform)
     bool stream_failed = false;
+    if (FUSE && !a.redo) {
+      if (fx.tab) {
+        argus_fuse_init(fx.tab, a.num_regions, tid, NT);
+        fx.row = a.fuse.warp_tab + (size_t)s * a.num_regions * kAggCellWords;
+      }
+      if (fx.pairbits) {
+        const u32 m = a.fuse.cta_sm[s / a.fuse.warps_per_cta];
+        if (m >= a.fuse.num_sms && tid == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
+        fx.sm_index = m < a.fuse.num_sms ? m : 0;
+      }
+      __syncthreads();
+    }
     if (tid == 0 && ntiles > 0) {
       const u32 bytes = (n < (u32)T ? n : (u32)T) * 16u;
       mbar_expect_tx(&sm.bar[0], bytes);
@@ -304,6 +338,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
           const int rk = tid + i * NT;
+          u32 f_region = 0xffffffffu;  // region / begin / inclusive time of this thread's interval, for the fused hooks
+          u64 f_begin = 0, f_incl = 0;
           if (rk < tile_ne) {
             const u32 d = sm.desc[rk];
             const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
@@ -327,6 +363,35 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               q[2] = make_uint4(s, preg, bidx, (d >> 16) | (flags << 16));
             } else if (!a.redo) {
               a.ctl->spec_overflow = 1;
+            }
+            if (FUSE && !a.redo) {
+              f_region = pe.z >> 1; f_begin = bts; f_incl = incl;
+              if (fx.tab) argus_fuse_aggregate(fx, f_region, incl, excl, flags);
+            }
+          }
+          if (FUSE && !a.redo && fx.pairbits) {  // every lane takes part: spans are appended a warp at a time
+            const bool cand = f_region != 0xffffffffu && f_incl && ((fx.pairbits[f_region >> 5] >> (f_region & 31)) & 1u);
+            if (__ballot_sync(0xffffffffu, cand)) {
+              for (u32 k = 0; k < 2 * a.fuse.num_pairs; ++k) {
+                const bool sel = cand && a.fuse.pairs[k] == f_region;
+                const u32 bal = __ballot_sync(0xffffffffu, sel);
+                if (!bal) continue;
+                const u32 c = __popc(bal);
+                if (ovc_used + c > kOvChunk) {
+                  u64 nbase = 0;
+                  if (lane == 0) nbase = atomicAdd(a.fuse.ov_count, (u64)kOvChunk);
+                  ovc_base = __shfl_sync(0xffffffffu, nbase, 0);
+                  ovc_used = 0;
+                }
+                if (sel) {
+                  const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
+                  if (slot < a.fuse.ov_capacity) {
+                    a.fuse.ov_spans[slot] = make_ulonglong2(f_begin, f_begin + f_incl);
+                    a.fuse.ov_seg[slot] = ((k >> 1) * a.fuse.num_sms + fx.sm_index) * 2 + (k & 1u);
+                  }
+                }
+                ovc_used += c;
+              }
             }
           }
         }
@@ -358,7 +423,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           bool ok = true;
           for (int e = 0; e < tn && ok; ++e) {
             const uint4 pe = evb[e];
-            ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w);
+            ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w,
+                                (FUSE && !a.redo) ? &fx : nullptr);
           }
           tot_ctx += st.n_ctx; tot_rev += st.n_rev; tot_clamp += st.n_clamp;
           sm.ch = st.h;
@@ -400,6 +466,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[bl][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
       if (tid == 0) a.counts[s] = n_int;
     }
+    if (FUSE && !a.redo && fx.tab) argus_fuse_flush(fx, a.num_regions, tid, NT);
     __syncthreads();
   }  // streams
 
@@ -418,23 +485,33 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   }
 }
 
-template <int NT, int E, int MINB>
+template <int NT, int E, int MINB, bool FUSE>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   static int grid_cache = 0;
-  const size_t smem = sizeof(TileSmem<NT, E>) + 128;
-  if (!grid_cache) {
-    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  static size_t smem_cache = 0;
+  size_t smem = ((sizeof(TileSmem<NT, E>) + 15) & ~(size_t)15) + 128;
+  if (FUSE) smem += (size_t)a.num_regions * sizeof(ArgusAggCell) + ((a.num_regions + 31) / 32) * 4 + 16;
+  if (!grid_cache || smem_cache != smem) {
+    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int dev = 0, sms = 0, per_sm = 0;
     ARGUS_CUDA_TRY(cudaGetDevice(&dev));
     ARGUS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB>, NT, smem));
+    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB, FUSE>, NT, smem));
     if (per_sm < 1) return ARGUS_ERR_CUDA;
+    if (per_sm > MINB) per_sm = MINB;
     grid_cache = sms * per_sm;
+    smem_cache = smem;
   }
   const u32 grid = a.num_streams < (u32)grid_cache ? a.num_streams : (u32)grid_cache;
-  k_pair_tiled<NT, E, MINB><<<grid, NT, smem, stream>>>(a);
+  k_pair_tiled<NT, E, MINB, FUSE><<<grid, NT, smem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   return ARGUS_OK;
+}
+
+template <int NT, int E, int MINB>
+int launch_tiled_any(const ArgusPairArgs& a, cudaStream_t stream) {
+  const bool fuse = !a.redo && (a.fuse.warp_tab || a.fuse.ov_spans);
+  return fuse ? launch_tiled<NT, E, MINB, true>(a, stream) : launch_tiled<NT, E, MINB, false>(a, stream);
 }
 
 int g_variant = 0;
@@ -442,6 +519,8 @@ int g_variant = 0;
 }  // namespace
 
 bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0; }
+
+bool argus_pair_tiled_can_fuse(uint32_t num_regions) { return num_regions <= kFuseMaxRegions; }
 
 #ifdef ARGUS_TILE_TIMING
 // Debug build only: cycles thread 0 of every CTA spent per phase (other, wait, A, B, C), summed; resets them.
@@ -458,14 +537,15 @@ extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   switch (g_variant) {
-    case 1: return launch_tiled<128, 8, 4>(a, stream);
-    case 2: return launch_tiled<256, 8, 2>(a, stream);
-    case 3: return launch_tiled<256, 6, 2>(a, stream);
-    case 4: return launch_tiled<128, 4, 6>(a, stream);
-    case 5: return launch_tiled<128, 6, 5>(a, stream);
-    case 6: return launch_tiled<256, 4, 3>(a, stream);
-    case 7: return launch_tiled<512, 4, 1>(a, stream);
-    case 8: return launch_tiled<64, 8, 8>(a, stream);
-    default: return launch_tiled<256, 5, 3>(a, stream);
+    case 1: return launch_tiled_any<128, 5, 4>(a, stream);
+    case 2: return launch_tiled_any<128, 7, 4>(a, stream);
+    case 3: return launch_tiled_any<256, 7, 2>(a, stream);
+    case 4: return launch_tiled_any<128, 9, 3>(a, stream);
+    case 5: return launch_tiled_any<256, 5, 2>(a, stream);
+    case 6: return launch_tiled_any<64, 5, 8>(a, stream);
+    case 7: return launch_tiled_any<64, 7, 8>(a, stream);
+    case 8: return launch_tiled_any<192, 5, 4>(a, stream);
+    case 9: return launch_tiled_any<256, 3, 4>(a, stream);
+    default: return launch_tiled_any<256, 5, 3>(a, stream);
   }
 }

@@ -1,0 +1,130 @@
+// argus_synthesize.cu — the whole hot path in one call: pair -> aggregate -> overlap.
+//
+// When the tiled pairing kernel can host the aggregation table (num_regions <= 256) the intervals
+// are aggregated and the overlap spans selected while they are still in registers, so the interval
+// array is written once and never read back. Otherwise this is the three plain calls in sequence.
+// Results are identical either way.
+#include "argus_fuse.cuh"
+
+int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                        uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                        uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                        uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
+                        bool reset_status, bool* fused_out);
+int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                             const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                             uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                             argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
+                             argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                             bool reset_status);
+int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                              argus_agg_t* warp_tab, argus_agg_t* cta_work, bool want_cta, argus_agg_t* sm_tab,
+                              argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream);
+int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                           const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status);
+int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* list_seg, const uint64_t* list_count,
+                                     uint64_t list_capacity, uint32_t num_sms, uint32_t num_pairs, argus_overlap_t* out,
+                                     argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+bool argus_pair_tiled_can_fuse(uint32_t num_regions);
+
+namespace {
+
+struct SynLayout {
+  size_t pair, pair_bytes, agg, agg_bytes, list_count, list_seg, list_spans, ov, ov_bytes, total;
+};
+
+SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_regions, uint64_t ambig_capacity,
+                     uint32_t num_pairs, uint32_t num_sms, uint64_t max_overlap_spans) {
+  SynLayout L;
+  size_t o = 0;
+  L.pair = o; L.pair_bytes = argus_pair_workspace_bytes(num_events, num_streams, ambig_capacity); o += argus_align_up(L.pair_bytes, 256);
+  L.agg = o; L.agg_bytes = argus_aggregate_workspace_bytes(num_events / 2, num_streams, num_regions); o += argus_align_up(L.agg_bytes, 256);
+  L.list_count = o; o += 256;
+  L.list_seg = o; o += argus_align_up((size_t)max_overlap_spans * 4 + 4, 256);
+  L.list_spans = o; o += argus_align_up((size_t)max_overlap_spans * 16 + 16, 256);
+  L.ov = o;
+  L.ov_bytes = argus_align_up((size_t)num_pairs * num_sms * 2 * 8 * 3 + 1024 + (size_t)max_overlap_spans * 24 + 256, 256);
+  o += L.ov_bytes;
+  L.total = o;
+  return L;
+}
+
+}  // namespace
+
+extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint32_t num_regions,
+                                                   uint64_t ambig_capacity, uint32_t num_pairs, uint32_t num_sms,
+                                                   uint64_t max_overlap_spans) {
+  return syn_layout(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms, max_overlap_spans).total;
+}
+
+extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                                uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                                uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                                uint64_t ambig_capacity, uint64_t* ambig_offsets, uint32_t warps_per_cta,
+                                const uint32_t* cta_sm, uint32_t num_sms, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                                argus_agg_t* sm_tab, argus_agg_t* kernel_tab, const uint32_t* pairs, uint32_t num_pairs,
+                                argus_overlap_t* overlap_out, uint64_t max_overlap_spans, argus_status_t* status,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!status || !workspace || ((uintptr_t)workspace & 255)) return ARGUS_ERR_INVALID_ARG;
+  if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
+  if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
+  if ((sm_tab || num_pairs) && (!cta_sm || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
+  if (num_pairs && (!pairs || !overlap_out)) return ARGUS_ERR_INVALID_ARG;
+  const SynLayout L = syn_layout(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms, max_overlap_spans);
+  if (workspace_bytes < L.total) return ARGUS_ERR_WORKSPACE;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  char* ws = (char*)workspace;
+  const size_t row_bytes = (size_t)num_regions * sizeof(argus_agg_t);
+  argus_agg_t* warp_work = warp_tab ? warp_tab : (argus_agg_t*)(ws + L.agg);
+  argus_agg_t* cta_work = cta_tab ? cta_tab : (argus_agg_t*)(ws + L.agg + argus_align_up((size_t)num_streams * row_bytes, 256));
+  const bool want_agg = warp_tab || cta_tab || sm_tab || kernel_tab;
+
+  ArgusFuseArgs f;
+  f.warp_tab = nullptr; f.cta_sm = cta_sm; f.warps_per_cta = warps_per_cta; f.num_sms = num_sms;
+  f.pairs = pairs; f.num_pairs = num_pairs; f.ov_spans = nullptr; f.ov_seg = nullptr; f.ov_capacity = 0; f.ov_count = nullptr;
+  const bool can_fuse = num_streams > 0 && argus_pair_tiled_can_fuse(num_regions);
+  if (can_fuse && want_agg) {
+    f.warp_tab = (u64*)warp_work;
+    ARGUS_CUDA_TRY(cudaMemsetAsync(warp_work, 0, (size_t)num_streams * row_bytes, stream));
+  }
+  if (can_fuse && num_pairs) {
+    f.ov_spans = (ulonglong2*)(ws + L.list_spans);
+    f.ov_seg = (u32*)(ws + L.list_seg);
+    f.ov_capacity = max_overlap_spans;
+    f.ov_count = (u64*)(ws + L.list_count);
+    ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_count, 0, 256, stream));
+    ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)max_overlap_spans * 4 + 4, stream));
+  }
+  bool fused = false;
+  int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
+                               interval_offsets, ambig, ambig_capacity, ambig_offsets, status, ws + L.pair, L.pair_bytes,
+                               cuda_stream, 0, (f.warp_tab || f.ov_spans) ? &f : nullptr, true, &fused);
+  if (rc != ARGUS_OK) return rc;
+
+  if (want_agg) {
+    if (fused && f.warp_tab) {
+      rc = argus_internal_agg_finish(ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm, num_sms, num_regions, warp_work,
+                                     cta_work, cta_tab != nullptr, sm_tab, kernel_tab, status, cuda_stream);
+    } else {
+      rc = argus_internal_aggregate(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
+                                    num_sms, num_regions, warp_tab, cta_tab, sm_tab, kernel_tab, status, ws + L.agg,
+                                    L.agg_bytes, cuda_stream, false);
+    }
+    if (rc != ARGUS_OK) return rc;
+  }
+  if (num_pairs) {
+    if (fused && f.ov_spans) {
+      rc = argus_internal_overlap_from_list(f.ov_spans, f.ov_seg, (const uint64_t*)f.ov_count, f.ov_capacity, num_sms, num_pairs, overlap_out,
+                                            status, ws + L.ov, L.ov_bytes, cuda_stream);
+    } else {
+      rc = argus_internal_overlap(intervals, interval_capacity, interval_offsets, num_streams, warps_per_cta, cta_sm, num_sms,
+                                  pairs, num_pairs, overlap_out, status, ws + L.ov, L.ov_bytes, cuda_stream, false);
+    }
+    if (rc != ARGUS_OK) return rc;
+  }
+  return ARGUS_OK;
+}

@@ -249,3 +249,93 @@ def test_overlap_random_spans_and_capacity():
     # a workspace too small for the selected spans is reported, not overrun
     ov, st = argus.argus_overlap(d_iv, len(iv), d_off, W, cta_sm, M, pairs, workspace_bytes=64 * 1024)
     assert int(argus.argus_status_fetch(st)["code"]) == 4
+
+
+def _synthesize_matches(spec, ev, offs, **kw):
+    d_ev, d_off = to_dev(ev, offs)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs_np = np.concatenate([spec.overlap_pairs, spec.overlap_pairs[:, ::-1], [[0, 0]]]).astype(np.uint32)
+    pairs = torch.from_numpy(pairs_np.view(np.int32)).to(DEV)
+    res = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, pairs, **kw)
+    st = res.fetch_status()
+    assert int(st["code"]) == 0, st
+    rc, o_iv, o_ioffs, o_am, o_aoffs, o_st = oracle.pair(ev, offs, spec.num_regions)
+    assert res.pair.intervals_numpy().tobytes() == o_iv.tobytes()
+    assert res.pair.ambig_numpy().tobytes() == o_am.tobytes()
+    assert np.array_equal(res.pair.interval_offsets.cpu().numpy().view(np.uint64), o_ioffs)
+    assert np.array_equal(res.pair.ambig_offsets.cpu().numpy().view(np.uint64), o_aoffs)
+    _, o_tabs, _ = oracle.aggregate(o_iv, o_ioffs, o_am, o_aoffs, spec.warps_per_cta, spec.cta_sm, spec.num_sms,
+                                    spec.num_regions)
+    for lv in ("warp", "cta", "sm", "kernel"):
+        got, want = res.agg.table_numpy(lv), o_tabs[lv]
+        if got.tobytes() != want.tobytes():
+            bad = np.argwhere(got != want)
+            raise AssertionError(f"{lv}: {len(bad)} cells differ; first {bad[0]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}")
+    _, o_ov, _ = oracle.overlap(o_iv, o_ioffs, spec.warps_per_cta, spec.cta_sm, spec.num_sms, pairs_np)
+    assert res.overlap_numpy(spec.num_sms).tobytes() == o_ov.tobytes()
+    return res, st
+
+
+@pytest.mark.parametrize("idx,ctas,iters", [(0, 4, 626), (1, 7, 300), (2, 3, 3), (3, 3, 9), (4, 9, 400)])
+def test_synthesize_fused_matches_oracle(idx, ctas, iters):
+    """One-call pipeline (aggregation and overlap selection fused into the pairing kernel)."""
+    spec = tg.config(idx).scaled(ctas, iters)
+    ev, offs = tg.generate_host(spec)
+    res, st = _synthesize_matches(spec, ev, offs)
+    if spec.well_formed:
+        assert int(st["n_sequential_tiles"]) == 0
+
+
+def test_synthesize_wide_histogram_and_flags():
+    """Durations spread over many log2 bins (outside the 16-bin shared-memory window), flagged intervals,
+    min/max extremes and a region that never occurs."""
+    rng = np.random.default_rng(21)
+    spec = tg.TraceSpec(tg.GEMM, 2, 1)  # only for warps_per_cta / cta_sm / pairs
+    S = spec.num_streams
+    evs, offs = [], [0]
+    for s in range(S):
+        rows, t = [], 1 << 40
+        for i in range(int(rng.integers(200, 3000))):
+            r = int(rng.integers(0, 4))
+            d = int(2 ** rng.uniform(0, 50)) if rng.random() < 0.9 else 0
+            rows.append((t, "B", r, i))
+            inner = int(rng.integers(0, d + 1))
+            if rng.random() < 0.5:
+                rows.append((t + 1, "B", (r + 1) % 4, i))
+                rows.append((t + 1 + inner, "E", (r + 1) % 4, i + (1 if rng.random() < 0.05 else 0)))
+            t_end = t + d - (2 * d if rng.random() < 0.02 else 0)
+            rows.append((t_end, "E", r, i))
+            t += d + int(rng.integers(0, 100))
+        ev = make_events(rows)
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    _synthesize_matches(spec, np.concatenate(evs), np.array(offs, np.uint64))
+
+
+def test_synthesize_many_regions_falls_back_to_plain_calls():
+    rng = np.random.default_rng(5)
+    R = 300  # more than the fused table holds
+    spec = tg.TraceSpec(tg.TINY, 2, 1)
+    evs, offs = [], [0]
+    for s in range(spec.num_streams):
+        ev = random_wellformed(rng, 400, R, max_height=5)
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    ev, offs = np.concatenate(evs), np.array(offs, np.uint64)
+
+    class Spec:  # same fields _synthesize_matches reads
+        num_regions, warps_per_cta, cta_sm, num_sms = R, 4, spec.cta_sm, spec.num_sms
+        overlap_pairs = np.array([(1, 2), (7, 299)], np.uint32)
+    _synthesize_matches(Spec, ev, offs)
+
+
+def test_synthesize_overlap_span_capacity():
+    spec = tg.config(2).scaled(2, 2)
+    ev, offs = tg.generate_host(spec)
+    d_ev, d_off = to_dev(ev, offs)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(DEV)
+    res = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, pairs,
+                                 max_overlap_spans=512)
+    st = res.fetch_status()
+    assert int(st["code"]) == 4 and int(st["intervals_required"]) > 512
