@@ -160,6 +160,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-ctas", type=int, default=6, help="CTAs of the workload the CPU baseline is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--three-calls", action="store_true",
+                    help="time argus_pair_intervals + argus_aggregate + argus_overlap instead of the one-call argus_synthesize")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -207,15 +209,24 @@ def main():
     acap = max(n_events // 64, 4096)
     ov_ws = torch.empty(min(argus.argus_overlap_workspace_bytes(icap, S, len(spec.overlap_pairs), spec.num_sms),
                             2 << 30), dtype=torch.uint8, device=dev)
-    state = {"pair": None, "agg": None}
+    state = {"pair": None, "agg": None, "syn": None}
+    mos = max(n_events // 8, 1 << 16)  # overlap spans the one-call pipeline may select
 
-    def step():
+    def step_three_calls():
         state["pair"] = p = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions, interval_capacity=icap,
                                                        ambig_capacity=acap, out=state["pair"])
         state["agg"] = argus.argus_aggregate(p.intervals, p.interval_offsets, p.ambig, p.ambig_offsets,
                                              spec.warps_per_cta, cta_sm, spec.num_sms, spec.num_regions, out=state["agg"])
         state["ov"] = argus.argus_overlap(p.intervals, icap, p.interval_offsets, spec.warps_per_cta, cta_sm, spec.num_sms,
                                           pairs, workspace=ov_ws)
+
+    def step_one_call():
+        state["syn"] = r = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms,
+                                                  pairs, interval_capacity=icap, ambig_capacity=acap,
+                                                  max_overlap_spans=mos, out=state["syn"])
+        state["pair"], state["agg"], state["ov"] = r.pair, r.agg, (r.overlap, r.status)
+
+    step = step_three_calls if args.three_calls else step_one_call
 
     def barrier():
         if world > 1:
@@ -264,7 +275,7 @@ def main():
     peak, peak_src = load_peaks()
     pair_ms = prof_ms["pair"] / max(prof_n["pair"], 1)
     achieved = ALG_BYTES_PER_EVENT * n_events / (pair_ms * 1e-3) / 1e9 if pair_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "pairing kernel of argus_pair_intervals", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "tiled pairing kernel (k_pair_tiled)" + ("" if args.three_calls else " with fused aggregation and overlap selection"), "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "peak_source": peak_src,
                 "traffic": None, "ms_per_launch": pair_ms, "algorithmic_bytes_per_event": ALG_BYTES_PER_EVENT,
                 "pipeline_frac": ALG_BYTES_PER_EVENT * n_events / (ms_per_step * 1e-3) / 1e9 / peak}
@@ -328,7 +339,8 @@ def main():
             "data": "synthetic",
             "config": {"workload": spec.name, "events_per_gpu": n_events, "streams": S, "regions": spec.num_regions,
                        "input_bytes_per_gpu": n_events * 16, "l2": "inputs (>= 1 GB) are larger than the 126 MB L2",
-                       "step": "argus_pair_intervals + argus_aggregate + argus_overlap on one trace per GPU"},
+                       "step": ("argus_pair_intervals + argus_aggregate + argus_overlap" if args.three_calls else
+                                "argus_synthesize (pair + aggregate + overlap in one call)") + " on one trace per GPU"},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline, "kernel_ms": kernel_ms,
         }

@@ -64,11 +64,15 @@ __device__ __forceinline__ void argus_fuse_init(ArgusAggCell* tab, u32 num_regio
   }
 }
 
-__device__ __forceinline__ void argus_fuse_aggregate(const ArgusFuseCtx& fx, u32 region, u64 incl, u64 excl, u32 flags) {
-  ArgusAggCell& c = fx.tab[region];
-  atomicAdd(&c.count, 1u);
-  argus_atomic_add64_split(&c.sum_incl, incl);
-  argus_atomic_add64_split(&c.sum_excl, excl);
+// count and sums of one cell (the part a thread may instead keep in registers for hot regions)
+__device__ __forceinline__ void argus_fuse_agg_sums(ArgusAggCell& c, u32 count, u64 sum_incl, u64 sum_excl) {
+  atomicAdd(&c.count, count);
+  argus_atomic_add64_split(&c.sum_incl, sum_incl);
+  argus_atomic_add64_split(&c.sum_excl, sum_excl);
+}
+
+// min, max, flag count and histogram bin of one interval
+__device__ __forceinline__ void argus_fuse_agg_rest(const ArgusFuseCtx& fx, ArgusAggCell& c, u32 region, u64 incl, u32 flags) {
   if (incl < *reinterpret_cast<volatile u64*>(&c.min_incl)) atomicMin(&c.min_incl, incl);
   if (incl > *reinterpret_cast<volatile u64*>(&c.max_incl)) atomicMax(&c.max_incl, incl);
   if (flags) atomicAdd(&c.nflag, 1u);
@@ -80,8 +84,19 @@ __device__ __forceinline__ void argus_fuse_aggregate(const ArgusFuseCtx& fx, u32
     hb = old == kAggUnset ? want : old;
   }
   const u32 rel = bin - hb;
-  if (rel < kAggWindow) atomicAdd(&c.h[rel], 1u);
-  else atomicAdd(fx.row + (size_t)region * kAggCellWords + 8 + bin, 1ull);
+  // lanes of this warp that hit the same (region, bin) add once, through their lowest lane
+  const u32 peers = __match_any_sync(__activemask(), (region << 6) | bin);
+  if ((threadIdx.x & 31u) == (u32)(__ffs(peers) - 1)) {
+    const u32 n = __popc(peers);
+    if (rel < kAggWindow) atomicAdd(&c.h[rel], n);
+    else atomicAdd(fx.row + (size_t)region * kAggCellWords + 8 + bin, (u64)n);
+  }
+}
+
+__device__ __forceinline__ void argus_fuse_aggregate(const ArgusFuseCtx& fx, u32 region, u64 incl, u64 excl, u32 flags) {
+  ArgusAggCell& c = fx.tab[region];
+  argus_fuse_agg_sums(c, 1u, incl, excl);
+  argus_fuse_agg_rest(fx, c, region, incl, flags);
 }
 
 __device__ __forceinline__ void argus_fuse_flush(const ArgusFuseCtx& fx, u32 num_regions, u32 tid, u32 nthreads) {

@@ -34,41 +34,50 @@ struct OvArgs {
 };
 
 __global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatter) {
+  // One stream per block iteration: all of its spans belong to one SM, so the block counts per
+  // (pair, role) in shared memory and touches each global counter once.
   __shared__ u32 sh_pairs[2 * kMaxPairs];
+  __shared__ u32 sh_cnt[2 * kMaxPairs];
+  __shared__ u64 sh_base[2 * kMaxPairs];
   for (u32 i = threadIdx.x; i < 2 * a.num_pairs; i += blockDim.x) sh_pairs[i] = a.pairs[i];
   __syncthreads();
   if (scatter && a.status->code != 0) return;
   for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
     const u32 m = a.cta_sm[s / a.warps_per_cta];
-    if (m >= a.num_sms) {
-      if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
-      continue;
-    }
     const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
-    if (hi < lo) {
-      if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
+    if (m >= a.num_sms || hi < lo) {
+      if (threadIdx.x == 0) argus_set_error(a.status, m >= a.num_sms ? ARGUS_ERR_INVALID_ARG : ARGUS_ERR_BAD_OFFSETS, s, m);
       continue;
     }
-    for (u64 i = lo + threadIdx.x; i < hi; i += blockDim.x) {
-      const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
-      const uint4 q0 = __ldg(p), q1 = __ldg(p + 1);
-      const u64 t0 = (u64)q0.x | ((u64)q0.y << 32);
-      const u64 incl = (u64)q0.z | ((u64)q0.w << 32);
-      const u32 region = q1.z;
-      if (incl == 0) continue;
-      for (u32 k = 0; k < a.num_pairs; ++k) {
-#pragma unroll
-        for (u32 role = 0; role < 2; ++role) {
-          if (sh_pairs[2 * k + role] != region) continue;
-          const u32 seg = (k * a.num_sms + m) * 2 + role;
-          if (!scatter) {
-            atomicAdd(&a.seg_count[seg], 1ull);
-          } else {
-            const u64 slot = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], 1ull);
+    for (u32 i = threadIdx.x; i < 2 * a.num_pairs; i += blockDim.x) sh_cnt[i] = 0;
+    __syncthreads();
+    for (int pass = 0; pass < (scatter ? 2 : 1); ++pass) {
+      for (u64 i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+        const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
+        const uint4 q0 = __ldg(p);
+        const u64 incl = (u64)q0.z | ((u64)q0.w << 32);
+        if (incl == 0) continue;
+        const u32 region = __ldg(reinterpret_cast<const u32*>(p + 1) + 2);
+        const u64 t0 = (u64)q0.x | ((u64)q0.y << 32);
+        for (u32 k = 0; k < 2 * a.num_pairs; ++k) {
+          if (sh_pairs[k] != region) continue;
+          const u32 local = atomicAdd(&sh_cnt[k], 1u);
+          if (pass == 1) {
+            const u64 slot = sh_base[k] + local;
             if (slot < a.capacity) a.spans[slot] = make_ulonglong2(t0, t0 + incl);
           }
         }
       }
+      __syncthreads();
+      for (u32 k = threadIdx.x; k < 2 * a.num_pairs; k += blockDim.x) {
+        const u32 seg = ((k >> 1) * a.num_sms + m) * 2 + (k & 1u);
+        if (pass == 0 && sh_cnt[k]) {
+          if (!scatter) atomicAdd(&a.seg_count[seg], (u64)sh_cnt[k]);
+          else sh_base[k] = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], (u64)sh_cnt[k]);
+        }
+        sh_cnt[k] = 0;
+      }
+      __syncthreads();
     }
   }
 }
@@ -82,7 +91,12 @@ struct OvList {
   u64 capacity;
 };
 
+constexpr u32 kOvListSegs = 2048;   // segments a block can count in shared memory
+constexpr u32 kOvListChunk = 8192;  // list entries a block handles per iteration
+
 __global__ void __launch_bounds__(256) k_ov_list_count_or_scatter(OvArgs a, OvList l, int scatter) {
+  __shared__ u32 sh_cnt[kOvListSegs];
+  __shared__ u64 sh_base[kOvListSegs];
   if (scatter && a.status->code != 0) return;
   const u64 reserved = *l.count;
   if (reserved > l.capacity && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -90,14 +104,42 @@ __global__ void __launch_bounds__(256) k_ov_list_count_or_scatter(OvArgs a, OvLi
     a.status->intervals_required = reserved;
   }
   const u64 n = reserved < l.capacity ? reserved : l.capacity;
-  for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (u64)gridDim.x * blockDim.x) {
-    const u32 seg = l.seg[i];
-    if (seg >= a.nseg) continue;
-    if (!scatter) {
-      atomicAdd(&a.seg_count[seg], 1ull);
-    } else {
-      const u64 slot = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], 1ull);
-      if (slot < a.capacity) a.spans[slot] = l.spans[i];
+  const bool local = a.nseg <= kOvListSegs;
+  for (u64 c0 = (u64)blockIdx.x * kOvListChunk; c0 < n; c0 += (u64)gridDim.x * kOvListChunk) {
+    const u64 c1 = c0 + kOvListChunk < n ? c0 + kOvListChunk : n;
+    if (!local) {  // too many segments for shared counters: global atomics per entry
+      for (u64 i = c0 + threadIdx.x; i < c1; i += blockDim.x) {
+        const u32 seg = l.seg[i];
+        if (seg >= a.nseg) continue;
+        if (!scatter) atomicAdd(&a.seg_count[seg], 1ull);
+        else {
+          const u64 slot = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], 1ull);
+          if (slot < a.capacity) a.spans[slot] = l.spans[i];
+        }
+      }
+      continue;
+    }
+    for (u32 g = threadIdx.x; g < a.nseg; g += blockDim.x) sh_cnt[g] = 0;
+    __syncthreads();
+    for (int pass = 0; pass < (scatter ? 2 : 1); ++pass) {
+      for (u64 i = c0 + threadIdx.x; i < c1; i += blockDim.x) {
+        const u32 seg = l.seg[i];
+        if (seg >= a.nseg) continue;
+        const u32 pos = atomicAdd(&sh_cnt[seg], 1u);
+        if (pass == 1) {
+          const u64 slot = sh_base[seg] + pos;
+          if (slot < a.capacity) a.spans[slot] = l.spans[i];
+        }
+      }
+      __syncthreads();
+      for (u32 g = threadIdx.x; g < a.nseg; g += blockDim.x) {
+        if (pass == 0 && sh_cnt[g]) {
+          if (!scatter) atomicAdd(&a.seg_count[g], (u64)sh_cnt[g]);
+          else sh_base[g] = a.seg_base[g] + atomicAdd(&a.seg_cursor[g], (u64)sh_cnt[g]);
+        }
+        sh_cnt[g] = 0;
+      }
+      __syncthreads();
     }
   }
 }

@@ -91,6 +91,7 @@ struct TileSmem {
   u64 n_int;                       // written by the sequential redo path
   int ch;
   int bad, dead, failed;
+  u32 hot[2];                      // fused aggregation: the two regions whose count and sums threads keep in registers
 };
 
 // Latest begin of the tile at level L and position < pos; -1 if there is none.
@@ -137,6 +138,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   fx.tab = nullptr; fx.pairbits = nullptr; fx.row = nullptr; fx.sm_index = 0;
   u64 ovc_base = 0;        // warp-uniform: current chunk of the global overlap span list
   u32 ovc_used = kOvChunk;
+  u32 hot0 = 0xffffffffu, hot1 = 0xffffffffu, hc0 = 0, hc1 = 0;  // hot regions of the current stream, private partial sums
+  u64 hsi0 = 0, hsi1 = 0, hse0 = 0, hse1 = 0;
   if (FUSE && !a.redo) {
     ArgusAggCell* tab = reinterpret_cast<ArgusAggCell*>(smem_raw + ((sizeof(SM) + 15) & ~(size_t)15));
     u32* pairbits = reinterpret_cast<u32*>(tab + a.num_regions);
@@ -184,6 +187,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       if (fx.tab) {
         argus_fuse_init(fx.tab, a.num_regions, tid, NT);
         fx.row = a.fuse.warp_tab + (size_t)s * a.num_regions * kAggCellWords;
+        hot0 = hot1 = 0xffffffffu; hc0 = hc1 = 0; hsi0 = hsi1 = hse0 = hse1 = 0;
+        if (tid < 2) sm.hot[tid] = 0xffffffffu;
       }
       if (fx.pairbits) {
         const u32 m = a.fuse.cta_sm[s / a.fuse.warps_per_cta];
@@ -366,7 +371,13 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             }
             if (FUSE && !a.redo) {
               f_region = pe.z >> 1; f_begin = bts; f_incl = incl;
-              if (fx.tab) argus_fuse_aggregate(fx, f_region, incl, excl, flags);
+              if (fx.tab) {
+                ArgusAggCell& cell = fx.tab[f_region];
+                if (f_region == hot0) { ++hc0; hsi0 += incl; hse0 += excl; }
+                else if (f_region == hot1) { ++hc1; hsi1 += incl; hse1 += excl; }
+                else argus_fuse_agg_sums(cell, 1u, incl, excl);
+                argus_fuse_agg_rest(fx, cell, f_region, incl, flags);
+              }
             }
           }
           if (FUSE && !a.redo && fx.pairbits) {  // every lane takes part: spans are appended a warp at a time
@@ -404,9 +415,25 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           sm.cidx[b ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[b][tid];
           sm.cchild[b ^ 1][tid] = accb[from];
         }
+        if (FUSE && !a.redo && fx.tab && hot0 == 0xffffffffu) {
+          if (ti == 0) {
+            if (warp == 0) {  // top two regions by count so far (counts may still be moving: only a heuristic)
+              u32 best = 0, second = 0;
+              for (u32 r = lane; r < a.num_regions; r += 32) {
+                const u32 key = (*reinterpret_cast<volatile u32*>(&fx.tab[r].count) << 16) | r;
+                if (key > best) { second = best; best = key; } else if (key > second) { second = key; }
+              }
+              const u32 top = __reduce_max_sync(0xffffffffu, best);
+              const u32 cand = best == top ? second : best;
+              const u32 next = __reduce_max_sync(0xffffffffu, cand);
+              if (lane == 0) { sm.hot[0] = (top >> 16) ? (top & 0xffffu) : 0xffffffffu; sm.hot[1] = (next >> 16) ? (next & 0xffffu) : 0xffffffffu; }
+            }
+          }
+        }
         ch = new_ch;
         n_int += (u64)tile_ne;
         __syncthreads();
+        if (FUSE && !a.redo && fx.tab && ti == 0) { hot0 = sm.hot[0]; hot1 = sm.hot[1]; }
         TT_MARK(4);
       } else {
         // ---------------- redo this tile with the sequential stack machine ----------------
@@ -466,7 +493,12 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[bl][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
       if (tid == 0) a.counts[s] = n_int;
     }
-    if (FUSE && !a.redo && fx.tab) argus_fuse_flush(fx, a.num_regions, tid, NT);
+    if (FUSE && !a.redo && fx.tab) {
+      if (hc0) argus_fuse_agg_sums(fx.tab[hot0], hc0, hsi0, hse0);
+      if (hc1) argus_fuse_agg_sums(fx.tab[hot1], hc1, hsi1, hse1);
+      __syncthreads();
+      argus_fuse_flush(fx, a.num_regions, tid, NT);
+    }
     __syncthreads();
   }  // streams
 
@@ -546,6 +578,17 @@ int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
     case 7: return launch_tiled_any<64, 7, 8>(a, stream);
     case 8: return launch_tiled_any<192, 5, 4>(a, stream);
     case 9: return launch_tiled_any<256, 3, 4>(a, stream);
-    default: return launch_tiled_any<256, 5, 3>(a, stream);
+    case 10: return launch_tiled_any<320, 5, 2>(a, stream);
+    case 11: return launch_tiled_any<352, 5, 2>(a, stream);
+    case 12: return launch_tiled_any<288, 5, 2>(a, stream);
+    case 13: return launch_tiled_any<512, 3, 1>(a, stream);
+    case 14: return launch_tiled_any<224, 7, 2>(a, stream);
+    case 15: return launch_tiled_any<256, 5, 3>(a, stream);
+    default: {
+      // automatic: four CTAs of 192 threads per SM, unless the fused aggregation table is large enough
+      // to cost a CTA slot; then two CTAs of 320 threads (streams per CTA stay balanced either way)
+      const bool big_table = !a.redo && a.fuse.warp_tab && (size_t)a.num_regions * sizeof(ArgusAggCell) > 6 * 1024;
+      return big_table ? launch_tiled_any<320, 5, 2>(a, stream) : launch_tiled_any<192, 5, 4>(a, stream);
+    }
   }
 }
