@@ -84,13 +84,8 @@ __device__ __forceinline__ void argus_fuse_agg_rest(const ArgusFuseCtx& fx, Argu
     hb = old == kAggUnset ? want : old;
   }
   const u32 rel = bin - hb;
-  // lanes of this warp that hit the same (region, bin) add once, through their lowest lane
-  const u32 peers = __match_any_sync(__activemask(), (region << 6) | bin);
-  if ((threadIdx.x & 31u) == (u32)(__ffs(peers) - 1)) {
-    const u32 n = __popc(peers);
-    if (rel < kAggWindow) atomicAdd(&c.h[rel], n);
-    else atomicAdd(fx.row + (size_t)region * kAggCellWords + 8 + bin, (u64)n);
-  }
+  if (rel < kAggWindow) atomicAdd(&c.h[rel], 1u);
+  else atomicAdd(fx.row + (size_t)region * kAggCellWords + 8 + bin, 1ull);
 }
 
 __device__ __forceinline__ void argus_fuse_aggregate(const ArgusFuseCtx& fx, u32 region, u64 incl, u64 excl, u32 flags) {

@@ -375,8 +375,12 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
                 ArgusAggCell& cell = fx.tab[f_region];
                 if (f_region == hot0) { ++hc0; hsi0 += incl; hse0 += excl; }
                 else if (f_region == hot1) { ++hc1; hsi1 += incl; hse1 += excl; }
+#ifndef AGG_SKIP_NONHOT
                 else argus_fuse_agg_sums(cell, 1u, incl, excl);
+#endif
+#ifndef AGG_SKIP_REST
                 argus_fuse_agg_rest(fx, cell, f_region, incl, flags);
+#endif
               }
             }
           }
