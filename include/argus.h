@@ -55,7 +55,8 @@ enum {
   ARGUS_ERR_DEPTH = 5,       /* device: a stream would hold more than ARGUS_MAX_DEPTH open frames */
   ARGUS_ERR_BAD_REGION = 6,  /* device: tag>>1 >= num_regions                             */
   ARGUS_ERR_BAD_OFFSETS = 7, /* device: stream_offsets / interval_offsets not non-decreasing */
-  ARGUS_ERR_TIMEOUT = 8      /* device: a bounded wait expired (reserved)                 */
+  ARGUS_ERR_TIMEOUT = 8,     /* device: a bounded wait expired                            */
+  ARGUS_ERR_STATIC_LIMIT = 9 /* host: input larger than the built-in scratch of a *_static call */
 };
 
 /* One marker event, 16 bytes. tag = region_id << 1 | is_end. ts = globaltimer ns.
@@ -192,6 +193,41 @@ int argus_pair_intervals_ex(const argus_event_t* events /*device*/, uint64_t num
                             uint64_t* ambig_offsets /*device [S+1] out*/,
                             argus_status_t* status /*device*/, void* workspace /*device*/,
                             size_t workspace_bytes, void* cuda_stream, int kernel_choice);
+
+/* ---------------------------------------------------------------------------------------
+ * argus_pair_intervals_static — no counterpart in the paper: a convenience variant of
+ * argus_pair_intervals for callers that cannot allocate device memory.
+ *
+ * Some callers run where cudaMalloc is off limits: inside a profiler or tool callback, in a
+ * process whose memory pool is owned by another component, or on a path that must not touch
+ * the allocator because an allocation could synchronise the device or fail late. This entry
+ * point needs no workspace argument: its scratch (control block, per-stream counters, event
+ * bitmap and its prefix tables, ambiguity notes) lives in a fixed array inside the library's
+ * device image, about 0.9 MB per GPU that loads the library, held until the process exits.
+ * Inputs and outputs are still the caller's buffers. The call makes no cudaMalloc, cudaFree
+ * or other allocating call.
+ *
+ * Limits (larger requests return ARGUS_ERR_STATIC_LIMIT and do nothing):
+ *   num_events <= ARGUS_STATIC_MAX_EVENTS, num_streams <= ARGUS_STATIC_MAX_STREAMS,
+ *   ambig_capacity <= ARGUS_STATIC_MAX_AMBIG.
+ * The first call on each device looks up the scratch array's device address (with that
+ * device current); make that first call before starting any stream capture. All calls on a
+ * device share the one scratch array: the parts that must start at zero are cleared at the
+ * start of every call, but two calls that overlap on the GPU (different streams, no ordering
+ * between them) race on it; callers must order them. Results equal argus_pair_intervals'.
+ * ------------------------------------------------------------------------------------- */
+#define ARGUS_STATIC_MAX_EVENTS  (1u << 20)
+#define ARGUS_STATIC_MAX_STREAMS 4096u
+#define ARGUS_STATIC_MAX_AMBIG   (1u << 16)
+
+int argus_pair_intervals_static(const argus_event_t* events /*device*/, uint64_t num_events,
+                                const uint64_t* stream_offsets /*device [S+1]*/,
+                                uint32_t num_streams, uint32_t num_regions,
+                                argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
+                                uint64_t* interval_offsets /*device [S+1] out*/,
+                                argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
+                                uint64_t* ambig_offsets /*device [S+1] out*/,
+                                argus_status_t* status /*device*/, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------
  * argus_aggregate — Section 3.2 "Region and scope" + the `duration` signal (Section 3.1).

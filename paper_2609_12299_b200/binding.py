@@ -78,6 +78,13 @@ def load_library():
     lib.argus_profile_enable.restype = None
     lib.argus_profile_read.argtypes = [vp, vp]
     lib.argus_profile_read.restype = ci
+    lib.argus_pair_intervals_static.argtypes = [vp, u64, vp, u32, u32, vp, u64, vp, vp, u64, vp, vp, vp]
+    lib.argus_pair_intervals_static.restype = ci
+    lib.argus_synthesize_workspace_bytes.argtypes = [u64, u32, u32, u64, u32, u32, u64]
+    lib.argus_synthesize_workspace_bytes.restype = sz
+    lib.argus_synthesize.argtypes = [vp, u64, vp, u32, u32, vp, u64, vp, vp, u64, vp, u32, vp, u32, vp, vp, vp, vp, vp, u32,
+                                     vp, u64, vp, vp, sz, vp]
+    lib.argus_synthesize.restype = ci
     _lib = lib
     return lib
 
@@ -200,6 +207,28 @@ def argus_pair_intervals(events: torch.Tensor, stream_offsets: torch.Tensor, num
     return out
 
 
+def argus_pair_intervals_static(events: torch.Tensor, stream_offsets: torch.Tensor, num_regions: int,
+                                interval_capacity: int | None = None, ambig_capacity: int | None = None) -> PairResult:
+    """Pairing through the entry point that needs no workspace: for callers that cannot allocate device
+    memory, its scratch is a fixed array inside the library (inputs up to 2^20 events, 4096 streams,
+    2^16 ambiguity records). This wrapper still allocates the OUTPUT tensors with torch; a caller that
+    cannot allocate passes its own buffers to the C function directly."""
+    lib = load_library()
+    dev = events.device
+    n = events.numel() * events.element_size() // 16
+    S = stream_offsets.numel() - 1
+    icap = n // 2 if interval_capacity is None else int(interval_capacity)
+    acap = min(n, 1 << 16) if ambig_capacity is None else int(ambig_capacity)
+    out = PairResult(_bytes(icap * 48, dev), torch.empty(S + 1, dtype=torch.int64, device=dev), _bytes(acap * 32, dev),
+                     torch.empty(S + 1, dtype=torch.int64, device=dev), _bytes(64, dev), icap, acap, _bytes(1, dev))
+    rc = lib.argus_pair_intervals_static(_ptr(events), n, _ptr(stream_offsets), S, num_regions, _ptr(out.intervals), icap,
+                                         _ptr(out.interval_offsets), _ptr(out.ambig), acap, _ptr(out.ambig_offsets),
+                                         _ptr(out.status), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_pair_intervals_static")
+    return out
+
+
 @dataclass
 class AggregateResult:
     warp: torch.Tensor | None    # uint8 [S * R * 576]
@@ -278,9 +307,6 @@ class SynthesizeResult:
 def argus_synthesize_workspace_bytes(num_events: int, num_streams: int, num_regions: int, ambig_capacity: int,
                                      num_pairs: int, num_sms: int, max_overlap_spans: int) -> int:
     lib = load_library()
-    lib.argus_synthesize_workspace_bytes.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64,
-                                                     ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64]
-    lib.argus_synthesize_workspace_bytes.restype = ctypes.c_size_t
     return lib.argus_synthesize_workspace_bytes(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms,
                                                 max_overlap_spans)
 
@@ -292,10 +318,6 @@ def argus_synthesize(events: torch.Tensor, stream_offsets: torch.Tensor, num_reg
                      out: SynthesizeResult | None = None) -> SynthesizeResult:
     """Whole hot path in one call (pair -> aggregate -> overlap); enqueues on the current stream."""
     lib = load_library()
-    vp, u32, u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
-    lib.argus_synthesize.argtypes = [vp, u64, vp, u32, u32, vp, u64, vp, vp, u64, vp, u32, vp, u32, vp, vp, vp, vp, vp, u32,
-                                     vp, u64, vp, vp, ctypes.c_size_t, vp]
-    lib.argus_synthesize.restype = ctypes.c_int
     dev = events.device
     n = events.numel() * events.element_size() // 16
     S = stream_offsets.numel() - 1

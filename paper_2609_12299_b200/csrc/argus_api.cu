@@ -8,6 +8,7 @@
 namespace {
 std::atomic<unsigned long long> g_launches{0};
 std::atomic<int> g_prof_on{0};
+std::atomic<int> g_prof_suppress{0};
 std::mutex g_prof_mu;
 struct ProfPair { cudaEvent_t a, b; };
 std::vector<ProfPair> g_prof[ARGUS_PROF_SLOTS];
@@ -16,7 +17,9 @@ std::vector<ProfPair> g_prof[ARGUS_PROF_SLOTS];
 void argus_count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 void argus_prof_mark(int slot, cudaStream_t stream, int end) {
-  if (!g_prof_on.load(std::memory_order_relaxed) || slot < 0 || slot >= ARGUS_PROF_SLOTS) return;
+  if (!g_prof_on.load(std::memory_order_relaxed) || g_prof_suppress.load(std::memory_order_relaxed) > 0 || slot < 0 ||
+      slot >= ARGUS_PROF_SLOTS)
+    return;
   std::lock_guard<std::mutex> lk(g_prof_mu);
   if (!end) {
     ProfPair p;
@@ -28,6 +31,8 @@ void argus_prof_mark(int slot, cudaStream_t stream, int end) {
     cudaEventRecord(g_prof[slot].back().b, stream);
   }
 }
+
+void argus_prof_suppress(int delta) { g_prof_suppress.fetch_add(delta); }
 
 extern "C" unsigned long long argus_launch_count(void) { return g_launches.load(); }
 
@@ -71,6 +76,7 @@ extern "C" const char* argus_strerror(int code) {
     case ARGUS_ERR_BAD_REGION: return "region id out of range";
     case ARGUS_ERR_BAD_OFFSETS: return "offsets are not non-decreasing or exceed the buffer";
     case ARGUS_ERR_TIMEOUT: return "bounded device wait expired";
+    case ARGUS_ERR_STATIC_LIMIT: return "input exceeds the built-in scratch of the allocation-free entry point (see ARGUS_STATIC_MAX_*)";
     default: return "unknown error code";
   }
 }

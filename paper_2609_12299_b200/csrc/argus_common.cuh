@@ -26,6 +26,7 @@ static_assert(sizeof(argus_status_t) == 64, "status layout");
 // host-side bookkeeping implemented in argus_api.cu
 void argus_count_launch();                                      // one more kernel launched by this library
 void argus_prof_mark(int slot, cudaStream_t stream, int end);   // CUDA events around a dominant kernel (if enabled)
+void argus_prof_suppress(int delta);                            // +1 / -1: event recording off while > 0 (it creates events)
 enum { ARGUS_PROF_PAIR = 0, ARGUS_PROF_AGGREGATE = 1, ARGUS_PROF_OVERLAP = 2, ARGUS_PROF_SLOTS = 4 };
 
 #define ARGUS_CHECK_LAUNCH()                                      \
