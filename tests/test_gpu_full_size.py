@@ -1,0 +1,143 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times (argus_synthesize on
+a trace generated in GPU memory): sampled CTAs are regenerated on the host (the generator is
+bit-identical on host and device), run through the CPU oracle one by one and compared bit for bit;
+properties that hold at any size are checked on the whole output."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_12299_b200 as argus
+from paper_2609_12299_b200 import tracegen as tg
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _run_full(spec):
+    d_ev, d_off = tg.generate_cuda(spec, DEV)
+    n = d_ev.numel() // 16
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(DEV)
+    res = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, pairs,
+                                 interval_capacity=n // 2, ambig_capacity=max(n // 64, 4096),
+                                 max_overlap_spans=max(n // 8, 1 << 16))
+    st = res.fetch_status()
+    assert int(st["code"]) == 0, st
+    return res, st, n, d_off.cpu().numpy().view(np.uint64)
+
+
+def _check_cta(spec, res, offs, c):
+    """Everything the path produced for CTA `c` against the oracle run on that CTA alone."""
+    W, R = spec.warps_per_cta, spec.num_regions
+    s0, s1 = c * W, (c + 1) * W
+    ev = tg.host_streams(spec, offs, s0, s1)
+    sub = (offs[s0:s1 + 1] - offs[s0]).astype(np.uint64)
+    rc, o_iv, o_ioffs, o_am, o_aoffs, o_st = oracle.pair(ev, sub, R, ambig_cap=max(len(ev) // 16, 4096))
+    assert rc == 0 and int(o_st["code"]) == 0
+    ioffs = res.pair.interval_offsets.cpu().numpy().view(np.uint64)
+    aoffs = res.pair.ambig_offsets.cpu().numpy().view(np.uint64)
+    assert np.array_equal(ioffs[s0:s1 + 1] - ioffs[s0], o_ioffs)
+    assert np.array_equal(aoffs[s0:s1 + 1] - aoffs[s0], o_aoffs)
+    g_iv = res.pair.intervals[int(ioffs[s0]) * 48:int(ioffs[s1]) * 48].cpu().numpy().view(argus.INTERVAL_DTYPE)
+    want = o_iv.copy()
+    want["stream"] += s0
+    assert g_iv.tobytes() == want.tobytes(), f"intervals of CTA {c} differ"
+    g_am = res.pair.ambig[int(aoffs[s0]) * 32:int(aoffs[s1]) * 32].cpu().numpy().view(argus.AMBIG_DTYPE)
+    want_am = o_am.copy()
+    want_am["stream"] += s0
+    assert g_am.tobytes() == want_am.tobytes(), f"ambiguity records of CTA {c} differ"
+    _, o_tabs, _ = oracle.aggregate(o_iv, o_ioffs, o_am, o_aoffs, W, np.zeros(1, np.uint32), 1, R)
+    row = R * 576
+    g_warp = res.agg.warp[s0 * row:s1 * row].cpu().numpy().view(argus.AGG_DTYPE).reshape(W, R)
+    assert g_warp.tobytes() == o_tabs["warp"].tobytes(), f"warp rows of CTA {c} differ"
+    g_cta = res.agg.cta[c * row:(c + 1) * row].cpu().numpy().view(argus.AGG_DTYPE).reshape(1, R)
+    assert g_cta.tobytes() == o_tabs["cta"].tobytes(), f"CTA row {c} differs"
+    if np.array_equal(spec.cta_sm, np.arange(spec.num_ctas)):  # one CTA per SM: SM row and overlap are this CTA's
+        g_sm = res.agg.sm[c * row:(c + 1) * row].cpu().numpy().view(argus.AGG_DTYPE).reshape(1, R)
+        assert g_sm.tobytes() == o_tabs["sm"].tobytes(), f"SM row {c} differs"
+        _, o_ov, _ = oracle.overlap(o_iv, o_ioffs, W, np.zeros(1, np.uint32), 1, spec.overlap_pairs)
+        g_ov = res.overlap_numpy(spec.num_sms)[:, c]
+        assert g_ov.tobytes() == o_ov[:, 0].tobytes(), f"overlap of SM {c} differs"
+    return len(o_iv), len(o_am)
+
+
+def _check_global(spec, res, st, n, well_formed):
+    """Size-independent properties of the whole output."""
+    S, R = spec.num_streams, spec.num_regions
+    ioffs = res.pair.interval_offsets.cpu().numpy().view(np.uint64)
+    total = int(ioffs[-1])
+    assert int(st["intervals_required"]) == total
+    if well_formed:
+        assert total * 2 == n and int(st["ambig_required"]) == 0 and int(st["n_sequential_tiles"]) == 0
+    warp = res.agg.table_numpy("warp")
+    cta, sm, ker = res.agg.table_numpy("cta"), res.agg.table_numpy("sm"), res.agg.table_numpy("kernel")
+    assert int(ker["count"].sum()) == total
+    assert np.array_equal(warp["count"].sum(1), np.diff(ioffs))       # per-stream counts = CSR offsets
+    for f in ("count", "sum_incl", "sum_excl", "n_flagged", "n_unmatched_begin", "n_unmatched_end", "hist"):
+        for tab in (warp, cta, sm):
+            assert np.array_equal(tab[f].sum(0, dtype=np.uint64), ker[f][0]), f
+    for tab in (warp, cta, sm):
+        assert np.array_equal(tab["min_incl"].min(0), ker["min_incl"][0])
+        assert np.array_equal(tab["max_incl"].max(0), ker["max_incl"][0])
+    assert np.array_equal(ker["hist"].sum(-1), ker["count"])
+    assert int((ker["n_unmatched_begin"] + ker["n_unmatched_end"]).sum()) == int(st["ambig_required"])
+    ov = res.overlap_numpy(spec.num_sms)
+    assert np.all(ov["overlap_ns"] <= np.minimum(ov["producer_ns"], ov["consumer_ns"]))
+    assert np.array_equal(ov["either_ns"], ov["producer_ns"] + ov["consumer_ns"] - ov["overlap_ns"])
+    del warp
+
+
+def test_decode_megakernel_full_size_sampled():
+    """The bench workload: 1.23 G events (19.65 GB), 202 regions."""
+    spec = tg.config(3)
+    res, st, n, offs = _run_full(spec)
+    assert n == 1_228_177_408
+    _check_global(spec, res, st, n, well_formed=True)
+    for c in (0, 73, 147):
+        ni, na = _check_cta(spec, res, offs, c)
+        assert ni == spec.warps_per_cta * 259_328 and na == 0
+    del res
+    torch.cuda.empty_cache()
+
+
+def test_attention_full_size_sampled():
+    spec = tg.config(2)
+    res, st, n, offs = _run_full(spec)
+    assert n == 153_513_888
+    _check_global(spec, res, st, n, well_formed=True)
+    for c in (0, 101, 147):
+        _check_cta(spec, res, offs, c)
+    ov = res.overlap_numpy(spec.num_sms)
+    assert np.all(ov["overlap_ns"] > 0)  # producer and consumer spans do overlap on every SM in this trace
+    del res
+    torch.cuda.empty_cache()
+
+
+def test_persistent_gemm_full_size_sampled():
+    spec = tg.config(1)
+    res, st, n, offs = _run_full(spec)
+    assert n == 68_672_000
+    _check_global(spec, res, st, n, well_formed=True)
+    for c in (0, 64, 147):
+        _check_cta(spec, res, offs, c)
+    del res
+    torch.cuda.empty_cache()
+
+
+def test_malformed_full_size_sampled():
+    """Dropped ends, duplicated begins and truncated streams at full size: ambiguity records, the
+    second (re-basing) pass and the sequential redo of tiles that are not well nested."""
+    spec = tg.config(4)
+    res, st, n, offs = _run_full(spec)
+    assert int(st["ambig_required"]) > 0 and int(st["n_sequential_tiles"]) > 0
+    _check_global(spec, res, st, n, well_formed=False)
+    lens = np.diff(offs)
+    truncated = np.nonzero(lens < np.where(np.arange(spec.num_streams) % 12 < 2, 72000, 32000) * 0.99)[0]
+    ctas = sorted({0, 147} | {int(s) // spec.warps_per_cta for s in truncated[:3]})
+    amb = 0
+    for c in ctas:
+        amb += _check_cta(spec, res, offs, c)[1]
+    assert amb > 0
+    del res
+    torch.cuda.empty_cache()
