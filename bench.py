@@ -166,9 +166,8 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2609_12299_b200.multirank import max_over_ranks, rank_env, rank_spec, whole_job_rate
+    rank, world, local_rank = rank_env()
 
     from paper_2609_12299_b200 import tracegen as tg
     spec = tg.config(args.workload)
@@ -198,8 +197,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # every rank its own trace of the same shape (weak scaling)
-    from dataclasses import replace
-    spec = replace(spec, seed=spec.seed + 1000 * rank)
+    spec = rank_spec(spec, rank)
     d_ev, d_off = tg.generate_cuda(spec, dev)
     n_events = d_ev.numel() // 16
     S = spec.num_streams
@@ -264,12 +262,9 @@ def main():
     if int(argus.argus_status_fetch(state["ov"][1])["code"]) != 0:
         raise RuntimeError("device status in overlap after the timed region")
 
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
-    value = n_events * world / (ms_per_step * 1e-3)
+    value = whole_job_rate(n_events, world, ms_per_step)
 
     # roofline of the dominant kernel (the pairing kernel): algorithmic bytes / its own launch time
     peak, peak_src = load_peaks()
@@ -309,12 +304,9 @@ def main():
         b.record()
         barrier()
         ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(ms, world, dev)
         assert int(pin_out[-1].numpy().view(argus.STATUS_DTYPE)[0]["code"]) == 0
-        e2e = {"value": n_events * world / (ms / args.e2e_steps * 1e-3), "unit": UNIT,
+        e2e = {"value": whole_job_rate(n_events, world, ms / args.e2e_steps), "unit": UNIT,
                "h2d_bytes_per_step": int(pin_ev.numel() + pin_off.numel() * 8),
                "d2h_bytes_per_step": int(sum(p.numel() * p.element_size() for p in pin_out)),
                "steps": args.e2e_steps, "ms_per_step": ms / args.e2e_steps}
