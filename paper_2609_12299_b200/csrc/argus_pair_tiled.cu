@@ -63,13 +63,14 @@ __device__ unsigned long long g_tile_timing[8];
 constexpr int kLevelWindow = 32;  // begins of a tile may sit at levels [lbase, lbase + 32)
 constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 1 sink for "no parent", padding
 constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
-constexpr int kBadRef = 0x3fff;   // reference that marks a tile as not well nested
+constexpr int kBadRef = 0x3fff;   // reference that marks a window as not well nested
+constexpr int kSeqChunk = 128;    // markers handed to the sequential machine at once when cuts come densely
 
 // Shared memory of one CTA. Events of the two tile buffers and the frames carried from earlier tiles
 // share one index space, so that "the frame an end closes" and "its parent" are plain indices:
 //   ev0[0..T) | car0[0..80) | car1[0..80) | ev1[0..T)
-// A tile in buffer 0 addresses carried level L as T + L (car0); a tile in buffer 1 as L - 80 (car1).
-// The tile in buffer b reads car_b and writes the stack it leaves behind into car_{b^1}.
+// Seen from buffer 0, carried block c holds level L at T + 80 c + L; seen from buffer 1 at 80 c + L - 160.
+// A window reads the current block and writes the stack it leaves behind into the other one.
 template <int NT, int E>
 struct TileSmem {
   static constexpr int T = NT * E;
@@ -78,19 +79,20 @@ struct TileSmem {
   static constexpr int MAXI = T / 2 + ARGUS_MAX_DEPTH;  // intervals a well-nested tile can emit
   static constexpr int NI = (MAXI + NT - 1) / NT;       // intervals per thread in the emission phases
   uint4 evall[2 * T + 2 * kCar];
-  u64 accall[T + 2 * kCar];        // child time per frame, same index space shifted by kCar
+  u64 accall[T + 4 * kCar];        // child time per frame, same index space shifted by 2 kCar
   u32 desc[MAXI];                  // per end, in end order: event index | level << 16
   u32 bm[kLevelWindow][NWORDS];    // per level: bit e set = event e of the tile is a begin at that level
   u64 summ[kLevelWindow];          // per level: bit w set = bm[level][w] != 0
   u32 cidx[2][ARGUS_MAX_DEPTH];    // begin index (within the stream) of each carried frame
-  u64 cchild[2][ARGUS_MAX_DEPTH];  // child time of each carried frame as the tile found it (for the redo path)
+  u64 cchild[2][ARGUS_MAX_DEPTH];  // child time of each carried frame as the window found it
   ArgusFrame fstk[ARGUS_MAX_DEPTH];  // stack in the layout the sequential redo path uses
   u32 warp_tot[32];
   u64 bar[2];
   u64 cur_stream;
   u64 n_int;                       // written by the sequential redo path
   int ch;
-  int bad, dead, failed;
+  int badpos;                      // first position of the window where the parallel rules fail (INT_MAX = none)
+  int dead, failed;
   u32 hot[2];                      // fused aggregation: the two regions whose count and sums threads keep in registers
 };
 
@@ -203,6 +205,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       tma_load_1d(sm.evall, src, bytes, &sm.bar[0]);
     }
 
+    int cpar = 0;        // which carried-frame block holds the current stack
     for (u32 ti = 0; ti < ntiles; ++ti) {
       const int b = ti & 1;
       const u32 tile_start = ti * (u32)T;
@@ -210,10 +213,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       uint4* const ev0 = sm.evall;
       uint4* const ev1 = sm.evall + T + 2 * kCar;
       const uint4* evb = b ? ev1 : ev0;                  // evb[ref] for every reference of this tile
-      u64* accb = sm.accall + kCar;                      // accb[ref]
-      const int cbase = b ? -kCar : T;                   // carried level L of this tile -> reference cbase + L
-      const int nbase = b ? T : -kCar;                   // same for the next tile (other buffer)
-      uint4* const car_next = sm.evall + T + (b ? 0 : kCar);
+      u64* accb = sm.accall + 2 * kCar;                  // accb[ref], ref in [-2 kCar, T + 2 kCar)
+      const int carlo = b ? -2 * kCar : T;               // reference of slot 0 of carried block 0, seen from this buffer
       if (tid == 0 && ti + 1 < ntiles) {  // prefetch the next tile into the other buffer
         const u32 nstart = tile_start + T;
         const u32 bytes = ((n - nstart) < (u32)T ? (n - nstart) : (u32)T) * 16u;
@@ -228,254 +229,271 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       }
       TT_MARK(1);
 
-      // ---------------- phase A: heights by prefix sum; begins into per-level bitmaps; ends into `desc` ------------
-      u32 tags[E];
-      int nb = 0, ne = 0, rel = 0, minrel = 0, maxrel = 0;
-      bool bad = false;
-#pragma unroll
-      for (int k = 0; k < E; ++k) {
-        const int e = tid * E + k;
-        tags[k] = e < tn ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;  // all ones = no event
-        accb[e] = 0;
-        (&sm.bm[0][0])[e] = 0;  // kLevelWindow * NWORDS == T words
-        if (tags[k] != 0xffffffffu) {
-          if ((tags[k] >> 1) >= a.num_regions) bad = true;
-          if (tags[k] & 1u) { ++ne; --rel; minrel = rel < minrel ? rel : minrel; }
-          else { ++nb; ++rel; maxrel = rel > maxrel ? rel : maxrel; }
-        }
-      }
-      if (tid < kLevelWindow) sm.summ[tid] = 0;
-      if (tid == 0) { sm.bad = 0; sm.failed = 0; accb[cbase + kSink] = 0; }
-      // block prefix sum of (begins, ends), 16 bits each: one barrier
-      const u32 mine_cnt = (u32)nb | ((u32)ne << 16);
-      u32 incl_cnt = mine_cnt;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const u32 o = __shfl_up_sync(0xffffffffu, incl_cnt, d);
-        if (lane >= d) incl_cnt += o;
-      }
-      if (lane == 31) sm.warp_tot[warp] = incl_cnt;
-      __syncthreads();
-      u32 before = 0, tot = 0;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        const u32 t = sm.warp_tot[w];
-        if (w < warp) before += t;
-        tot += t;
-      }
-      const u32 ex = before + incl_cnt - mine_cnt;
-      const int tile_nb = (int)(tot & 0xffffu), tile_ne = (int)(tot >> 16);
-      const int h0 = ch + (int)(ex & 0xffffu) - (int)(ex >> 16);
-      const int lbase = ch > 16 ? ch - 16 : 0;
-      // well nested so far: height never negative, never above the limit, begins inside the level window
-      if (h0 + minrel < 0 || h0 + maxrel > ARGUS_MAX_DEPTH || tile_ne > MAXI) bad = true;
-      if (nb > 0 && (h0 + minrel < lbase || h0 + maxrel > lbase + kLevelWindow)) bad = true;
-      if (bad) sm.bad = 1;
-      else {
-        int h = h0, rank = (int)(ex >> 16);
+      // The tile is consumed in windows [w0, wend). A well-nested tile is one window. When the parallel
+      // rules fail first at position p, the window is cut there: [w0, p) is redone in parallel (it is well
+      // nested), the marker at p goes through the sequential stack machine, and a new window starts after it.
+      int w0 = 0, wend = tn, small_streak = 0;
+      while (w0 < tn) {
+        const int cbase = carlo + cpar * kCar;           // carried level L -> reference cbase + L
+        uint4* const car_next = sm.evall + T + (cpar ^ 1) * kCar;
+
+        // ---------------- phase A: heights by prefix sum; begins into per-level bitmaps; ends into `desc` ----------
+        u32 tags[E];
+        int nb = 0, ne = 0;
 #pragma unroll
         for (int k = 0; k < E; ++k) {
-          if (tags[k] == 0xffffffffu) continue;
-          const int e = tid * E + k;
-          if (tags[k] & 1u) {
-            --h;
-            sm.desc[rank++] = (u32)e | ((u32)h << 16);
-          } else {
-            const int l = h - lbase;
-            atomicOr(&sm.bm[l][e >> 5], 1u << (e & 31));
-            atomicOr(reinterpret_cast<u32*>(&sm.summ[l]) + (e >> 10), 1u << ((e >> 5) & 31));
-            ++h;
-          }
+          const int e = w0 + tid * E + k;
+          tags[k] = e < wend ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;  // all ones = no event
+          if (e < wend) accb[e] = 0;
+          (&sm.bm[0][0])[tid * E + k] = 0;  // kLevelWindow * NWORDS == T words
+          if (tags[k] != 0xffffffffu) { if (tags[k] & 1u) ++ne; else ++nb; }
         }
-      }
-      __syncthreads();
-      TT_MARK(2);
-
-      // ---------------- phase B: one thread per end marker: find begin and parent, feed the parent's child time -----
-      u32 refs[NI];
-      if (!sm.bad) {
+        if (tid < kLevelWindow) sm.summ[tid] = 0;
+        if (tid < ch) accb[cbase + tid] = sm.cchild[cpar][tid];  // a cut window may have added to these: start clean
+        if (tid == 0) { sm.badpos = 0x7fffffff; sm.failed = 0; accb[cbase + kSink] = 0; }
+        // block prefix sum of (begins, ends), 16 bits each: one barrier
+        const u32 mine_cnt = (u32)nb | ((u32)ne << 16);
+        u32 incl_cnt = mine_cnt;
 #pragma unroll
-        for (int i = 0; i < NI; ++i) {
-          const int rk = tid + i * NT;
-          refs[i] = 0;
-          if (rk < tile_ne) {
-            const u32 d = sm.desc[rk];
-            const int e = (int)(d & 0xffffu), L = (int)(d >> 16);
-            int partner = tile_latest_begin<NT, E>(sm, L, lbase, e);
-            int parent;
-            if (partner < 0) {  // opened in an earlier tile: so was its parent
-              partner = L < ch ? cbase + L : kBadRef;
-              parent = L == 0 ? cbase + kSink : cbase + L - 1;
-            } else if (L == 0) {
-              parent = cbase + kSink;
+        for (int d = 1; d < 32; d <<= 1) {
+          const u32 o = __shfl_up_sync(0xffffffffu, incl_cnt, d);
+          if (lane >= d) incl_cnt += o;
+        }
+        if (lane == 31) sm.warp_tot[warp] = incl_cnt;
+        __syncthreads();
+        u32 before = 0, tot = 0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+          const u32 t = sm.warp_tot[w];
+          if (w < warp) before += t;
+          tot += t;
+        }
+        const u32 ex = before + incl_cnt - mine_cnt;
+        const int win_nb = (int)(tot & 0xffffu);
+        const int win_ne = (int)(tot >> 16) < MAXI ? (int)(tot >> 16) : MAXI;  // more ends than that means a violation earlier
+        const int h0 = ch + (int)(ex & 0xffffu) - (int)(ex >> 16);
+        const int lbase = ch > 16 ? ch - 16 : 0;
+        {
+          int h = h0, rank = (int)(ex >> 16);
+          bool seen = false;  // this thread already reported a violation: later markers only keep `desc` complete
+#pragma unroll
+          for (int k = 0; k < E; ++k) {
+            if (tags[k] == 0xffffffffu) continue;
+            const int e = w0 + tid * E + k;
+            // the parallel rules: known region id, height never negative, at most 64 frames, begins inside the level window
+            bool viol = (tags[k] >> 1) >= a.num_regions;
+            if (tags[k] & 1u) {
+              --h;
+              if (h < 0) viol = true;
+              if (rank < MAXI) sm.desc[rank] = (u32)e | ((u32)(h & 0xff) << 16);
+              ++rank;
             } else {
-              parent = tile_latest_begin<NT, E>(sm, L - 1, lbase, partner);
-              if (parent < 0) parent = L - 1 < ch ? cbase + L - 1 : kBadRef;
+              const int l = h - lbase;
+              if (l < 0 || l >= kLevelWindow || h >= ARGUS_MAX_DEPTH) viol = true;
+              if (!viol && !seen) {
+                atomicOr(&sm.bm[l][e >> 5], 1u << (e & 31));
+                atomicOr(reinterpret_cast<u32*>(&sm.summ[l]) + (e >> 10), 1u << ((e >> 5) & 31));
+              }
+              ++h;
             }
-            if (partner == kBadRef || parent == kBadRef) { sm.bad = 1; continue; }
-            const uint4 ee = evb[e];
-            const uint4 pe = evb[partner];
-            if ((pe.z >> 1) != (ee.z >> 1)) sm.bad = 1;
-            const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
-            if (ts > bts) {  // 64-bit add as two native 32-bit shared atomics; each carry is propagated exactly once
-              const u64 dlt = ts - bts;
-              u32* p = reinterpret_cast<u32*>(&accb[parent]);
-              const u32 lo32 = (u32)dlt, hi32 = (u32)(dlt >> 32);
-              const u32 old = atomicAdd(p, lo32);
-              if (hi32) atomicAdd(p + 1, hi32);
-              if (old + lo32 < old) atomicAdd(p + 1, 1u);
-            }
-            refs[i] = ((u32)partner & 0xffffu) | ((u32)parent << 16);
+            if (viol && !seen) { atomicMin(&sm.badpos, e); seen = true; }
           }
         }
-      }
-      __syncthreads();
-      TT_MARK(3);
-      const bool tile_bad = sm.bad != 0;
-      if (sm.dead) {  // a bulk copy never arrived: report and leave (uniform decision)
-        if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
-        return;
-      }
+        __syncthreads();
+        TT_MARK(2);
 
-      if (!tile_bad) {
-        // ---------------- phase C: exclusive time, parent region, interval records; carried stack -------------
-        const u64 pos0 = out_base + n_int;
+        // ---------------- phase B: one thread per end marker: find begin and parent, feed the parent's child time ---
+        u32 refs[NI];
+        {
+          const int first_bad = sm.badpos;  // violations found so far; ends at or after it need no work
 #pragma unroll
-        for (int i = 0; i < NI; ++i) {
-          const int rk = tid + i * NT;
-          u32 f_region = 0xffffffffu;  // region / begin / inclusive time of this thread's interval, for the fused hooks
-          u64 f_begin = 0, f_incl = 0;
-          if (rk < tile_ne) {
-            const u32 d = sm.desc[rk];
-            const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
-            const uint4 ee = evb[d & 0xffffu];
-            const uint4 pe = evb[partner];
-            const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
-            const u64 child = accb[partner];
-            u32 flags = 0;
-            u64 incl = 0, excl = 0;
-            if (ee.w != pe.w) { flags |= ARGUS_FLAG_CTX_MISMATCH; ++tot_ctx; }
-            if (ts < bts) { flags |= ARGUS_FLAG_TIME_REVERSED; ++tot_rev; } else { incl = ts - bts; }
-            if (child > incl) { flags |= ARGUS_FLAG_CHILD_CLAMPED; ++tot_clamp; } else { excl = incl - child; }
-            const bool carried = (u32)partner >= (u32)T;
-            const u32 bidx = carried ? sm.cidx[b][partner - cbase] : tile_start + (u32)partner;
-            const u32 preg = parent == cbase + kSink ? ARGUS_NONE : (reinterpret_cast<const u32*>(evb + parent)[2] >> 1);
-            const u64 pos = pos0 + (u64)rk;
-            if (pos < a.interval_capacity) {
-              uint4* q = reinterpret_cast<uint4*>(a.intervals + pos);
-              q[0] = make_uint4(pe.x, pe.y, (u32)incl, (u32)(incl >> 32));
-              q[1] = make_uint4((u32)excl, (u32)(excl >> 32), pe.z >> 1, pe.w);
-              q[2] = make_uint4(s, preg, bidx, (d >> 16) | (flags << 16));
-            } else if (!a.redo) {
-              a.ctl->spec_overflow = 1;
-            }
-            if (FUSE && !a.redo) {
-              f_region = pe.z >> 1; f_begin = bts; f_incl = incl;
-              if (fx.tab) {
-                ArgusAggCell& cell = fx.tab[f_region];
-                if (f_region == hot0) { ++hc0; hsi0 += incl; hse0 += excl; }
-                else if (f_region == hot1) { ++hc1; hsi1 += incl; hse1 += excl; }
-#ifndef AGG_SKIP_NONHOT
-                else argus_fuse_agg_sums(cell, 1u, incl, excl);
-#endif
-#ifndef AGG_SKIP_REST
-                argus_fuse_agg_rest(fx, cell, f_region, incl, flags);
-#endif
+          for (int i = 0; i < NI; ++i) {
+            const int rk = tid + i * NT;
+            refs[i] = 0;
+            if (rk < win_ne) {
+              const u32 d = sm.desc[rk];
+              const int e = (int)(d & 0xffffu), L = (int)(d >> 16);
+              if (e >= first_bad) continue;
+              int partner = tile_latest_begin<NT, E>(sm, L, lbase, e);
+              int parent;
+              if (partner < 0) {  // opened before this window: so was its parent
+                partner = L < ch ? cbase + L : kBadRef;
+                parent = L == 0 ? cbase + kSink : cbase + L - 1;
+              } else if (L == 0) {
+                parent = cbase + kSink;
+              } else {
+                parent = tile_latest_begin<NT, E>(sm, L - 1, lbase, partner);
+                if (parent < 0) parent = L - 1 < ch ? cbase + L - 1 : kBadRef;
               }
+              if (partner == kBadRef || parent == kBadRef) { atomicMin(&sm.badpos, e); continue; }
+              const uint4 ee = evb[e];
+              const uint4 pe = evb[partner];
+              if ((pe.z >> 1) != (ee.z >> 1)) { atomicMin(&sm.badpos, e); continue; }
+              const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
+              if (ts > bts) {  // 64-bit add as two native 32-bit shared atomics; each carry is propagated exactly once
+                const u64 dlt = ts - bts;
+                u32* p = reinterpret_cast<u32*>(&accb[parent]);
+                const u32 lo32 = (u32)dlt, hi32 = (u32)(dlt >> 32);
+                const u32 old = atomicAdd(p, lo32);
+                if (hi32) atomicAdd(p + 1, hi32);
+                if (old + lo32 < old) atomicAdd(p + 1, 1u);
+              }
+              refs[i] = ((u32)partner & 0xffffu) | ((u32)parent << 16);
             }
           }
-          if (FUSE && !a.redo && fx.pairbits) {  // every lane takes part: spans are appended a warp at a time
-            const bool cand = f_region != 0xffffffffu && f_incl && ((fx.pairbits[f_region >> 5] >> (f_region & 31)) & 1u);
-            if (__ballot_sync(0xffffffffu, cand)) {
-              for (u32 k = 0; k < 2 * a.fuse.num_pairs; ++k) {
-                const bool sel = cand && a.fuse.pairs[k] == f_region;
-                const u32 bal = __ballot_sync(0xffffffffu, sel);
-                if (!bal) continue;
-                const u32 c = __popc(bal);
-                if (ovc_used + c > kOvChunk) {
-                  u64 nbase = 0;
-                  if (lane == 0) nbase = atomicAdd(a.fuse.ov_count, (u64)kOvChunk);
-                  ovc_base = __shfl_sync(0xffffffffu, nbase, 0);
-                  ovc_used = 0;
+        }
+        __syncthreads();
+        TT_MARK(3);
+        if (sm.dead) {  // a bulk copy never arrived: report and leave (uniform decision)
+          if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
+          return;
+        }
+        const int badpos = sm.badpos;
+
+        if (badpos >= wend) {
+          // ---------------- phase C: exclusive time, parent region, interval records; carried stack -------------
+          const u64 pos0 = out_base + n_int;
+#pragma unroll
+          for (int i = 0; i < NI; ++i) {
+            const int rk = tid + i * NT;
+            u32 f_region = 0xffffffffu;  // region / begin / inclusive time of this thread's interval, for the fused hooks
+            u64 f_begin = 0, f_incl = 0;
+            if (rk < win_ne) {
+              const u32 d = sm.desc[rk];
+              const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
+              const uint4 ee = evb[d & 0xffffu];
+              const uint4 pe = evb[partner];
+              const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
+              const u64 child = accb[partner];
+              u32 flags = 0;
+              u64 incl = 0, excl = 0;
+              if (ee.w != pe.w) { flags |= ARGUS_FLAG_CTX_MISMATCH; ++tot_ctx; }
+              if (ts < bts) { flags |= ARGUS_FLAG_TIME_REVERSED; ++tot_rev; } else { incl = ts - bts; }
+              if (child > incl) { flags |= ARGUS_FLAG_CHILD_CLAMPED; ++tot_clamp; } else { excl = incl - child; }
+              const bool carried = (u32)partner >= (u32)T;
+              const u32 bidx = carried ? sm.cidx[cpar][partner - cbase] : tile_start + (u32)partner;
+              const u32 preg = parent == cbase + kSink ? ARGUS_NONE : (reinterpret_cast<const u32*>(evb + parent)[2] >> 1);
+              const u64 pos = pos0 + (u64)rk;
+              if (pos < a.interval_capacity) {
+                uint4* q = reinterpret_cast<uint4*>(a.intervals + pos);
+                q[0] = make_uint4(pe.x, pe.y, (u32)incl, (u32)(incl >> 32));
+                q[1] = make_uint4((u32)excl, (u32)(excl >> 32), pe.z >> 1, pe.w);
+                q[2] = make_uint4(s, preg, bidx, (d >> 16) | (flags << 16));
+              } else if (!a.redo) {
+                a.ctl->spec_overflow = 1;
+              }
+              if (FUSE && !a.redo) {
+                f_region = pe.z >> 1; f_begin = bts; f_incl = incl;
+                if (fx.tab) {
+                  ArgusAggCell& cell = fx.tab[f_region];
+                  if (f_region == hot0) { ++hc0; hsi0 += incl; hse0 += excl; }
+                  else if (f_region == hot1) { ++hc1; hsi1 += incl; hse1 += excl; }
+                  else argus_fuse_agg_sums(cell, 1u, incl, excl);
+                  argus_fuse_agg_rest(fx, cell, f_region, incl, flags);
                 }
-                if (sel) {
-                  const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
-                  if (slot < a.fuse.ov_capacity) {
-                    a.fuse.ov_spans[slot] = make_ulonglong2(f_begin, f_begin + f_incl);
-                    a.fuse.ov_seg[slot] = ((k >> 1) * a.fuse.num_sms + fx.sm_index) * 2 + (k & 1u);
+              }
+            }
+            if (FUSE && !a.redo && fx.pairbits) {  // every lane takes part: spans are appended a warp at a time
+              const bool cand = f_region != 0xffffffffu && f_incl && ((fx.pairbits[f_region >> 5] >> (f_region & 31)) & 1u);
+              if (__ballot_sync(0xffffffffu, cand)) {
+                for (u32 k = 0; k < 2 * a.fuse.num_pairs; ++k) {
+                  const bool sel = cand && a.fuse.pairs[k] == f_region;
+                  const u32 bal = __ballot_sync(0xffffffffu, sel);
+                  if (!bal) continue;
+                  const u32 c = __popc(bal);
+                  if (ovc_used + c > kOvChunk) {
+                    u64 nb64 = 0;
+                    if (lane == 0) nb64 = atomicAdd(a.fuse.ov_count, (u64)kOvChunk);
+                    ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
+                    ovc_used = 0;
                   }
+                  if (sel) {
+                    const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
+                    if (slot < a.fuse.ov_capacity) {
+                      a.fuse.ov_spans[slot] = make_ulonglong2(f_begin, f_begin + f_incl);
+                      a.fuse.ov_seg[slot] = ((k >> 1) * a.fuse.num_sms + fx.sm_index) * 2 + (k & 1u);
+                    }
+                  }
+                  ovc_used += c;
                 }
-                ovc_used += c;
               }
             }
           }
-        }
-        const int new_ch = ch + tile_nb - tile_ne;
-        if (tid < new_ch) {  // the stack this tile leaves behind, in the next tile's index space
-          const int e = tile_latest_begin<NT, E>(sm, tid, lbase, T);
-          const int from = e >= 0 ? e : cbase + tid;
-          car_next[tid] = evb[from];
-          accb[nbase + tid] = accb[from];
-          sm.cidx[b ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[b][tid];
-          sm.cchild[b ^ 1][tid] = accb[from];
-        }
-        if (FUSE && !a.redo && fx.tab && hot0 == 0xffffffffu) {
-          if (ti == 0) {
-            if (warp == 0) {  // top two regions by count so far (counts may still be moving: only a heuristic)
-              u32 best = 0, second = 0;
-              for (u32 r = lane; r < a.num_regions; r += 32) {
-                const u32 key = (*reinterpret_cast<volatile u32*>(&fx.tab[r].count) << 16) | r;
-                if (key > best) { second = best; best = key; } else if (key > second) { second = key; }
-              }
-              const u32 top = __reduce_max_sync(0xffffffffu, best);
-              const u32 cand = best == top ? second : best;
-              const u32 next = __reduce_max_sync(0xffffffffu, cand);
-              if (lane == 0) { sm.hot[0] = (top >> 16) ? (top & 0xffffu) : 0xffffffffu; sm.hot[1] = (next >> 16) ? (next & 0xffffu) : 0xffffffffu; }
+          const int new_ch = ch + win_nb - win_ne;
+          if (tid < new_ch) {  // the stack this window leaves behind, in the next window's index space
+            const int e = tile_latest_begin<NT, E>(sm, tid, lbase, T);
+            const int from = e >= 0 ? e : cbase + tid;
+            car_next[tid] = evb[from];
+            sm.cchild[cpar ^ 1][tid] = accb[from];
+            sm.cidx[cpar ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[cpar][tid];
+          }
+          if (FUSE && !a.redo && fx.tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0 && warp == 0) {
+            // top two regions by count so far (counts may still be moving: only a heuristic)
+            u32 best = 0, second = 0;
+            for (u32 r = lane; r < a.num_regions; r += 32) {
+              const u32 key = (*reinterpret_cast<volatile u32*>(&fx.tab[r].count) << 16) | r;
+              if (key > best) { second = best; best = key; } else if (key > second) { second = key; }
             }
+            const u32 top = __reduce_max_sync(0xffffffffu, best);
+            const u32 cand = best == top ? second : best;
+            const u32 next = __reduce_max_sync(0xffffffffu, cand);
+            if (lane == 0) { sm.hot[0] = (top >> 16) ? (top & 0xffffu) : 0xffffffffu; sm.hot[1] = (next >> 16) ? (next & 0xffffu) : 0xffffffffu; }
           }
-        }
-        ch = new_ch;
-        n_int += (u64)tile_ne;
-        __syncthreads();
-        if (FUSE && !a.redo && fx.tab && ti == 0) { hot0 = sm.hot[0]; hot1 = sm.hot[1]; }
-        TT_MARK(4);
-      } else {
-        // ---------------- redo this tile with the sequential stack machine ----------------
-        if (tid < ch) {
-          const uint4 f = evb[cbase + tid];
-          ArgusFrame& o = sm.fstk[tid];
-          o.ts = (u64)f.x | ((u64)f.y << 32); o.child = sm.cchild[b][tid]; o.region = f.z >> 1; o.ctx = f.w;
-          o.idx = sm.cidx[b][tid]; o.pad = 0;
-        }
-        __syncthreads();
-        if (tid == 0) {
-          ArgusSeqState st;
-          st.h = ch; st.n_int = n_int; st.n_ctx = st.n_rev = st.n_clamp = 0; st.failed = false;
-          bool ok = true;
-          for (int e = 0; e < tn && ok; ++e) {
-            const uint4 pe = evb[e];
-            ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w,
-                                (FUSE && !a.redo) ? &fx : nullptr);
+          const bool pick_hot = FUSE && !a.redo && fx.tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0;
+          small_streak = (wend - w0 < 32) ? small_streak + 1 : 0;
+          ch = new_ch;
+          n_int += (u64)win_ne;
+          cpar ^= 1;
+          w0 = wend;
+          wend = tn;
+          __syncthreads();
+          if (pick_hot) { hot0 = sm.hot[0]; hot1 = sm.hot[1]; }
+          TT_MARK(4);
+        } else if (badpos > w0) {
+          wend = badpos;  // [w0, badpos) is well nested: do it again on its own (nothing was committed yet)
+        } else {
+          // ---------------- the marker(s) at w0 go through the sequential stack machine ----------------
+          const int nseq = small_streak >= 2 ? ((tn - w0) < kSeqChunk ? (tn - w0) : kSeqChunk) : 1;
+          if (tid < ch) {
+            const uint4 f = evb[cbase + tid];
+            ArgusFrame& o = sm.fstk[tid];
+            o.ts = (u64)f.x | ((u64)f.y << 32); o.child = sm.cchild[cpar][tid]; o.region = f.z >> 1; o.ctx = f.w;
+            o.idx = sm.cidx[cpar][tid]; o.pad = 0;
           }
-          tot_ctx += st.n_ctx; tot_rev += st.n_rev; tot_clamp += st.n_clamp;
-          sm.ch = st.h;
-          sm.n_int = st.n_int;
-          sm.failed = ok ? 0 : 1;
-          if (!a.redo) atomicAdd((u64*)&a.status->n_sequential_tiles, 1ull);
+          __syncthreads();
+          if (tid == 0) {
+            ArgusSeqState st;
+            st.h = ch; st.n_int = n_int; st.n_ctx = st.n_rev = st.n_clamp = 0; st.failed = false;
+            bool ok = true;
+            for (int e = w0; e < w0 + nseq && ok; ++e) {
+              const uint4 pe = evb[e];
+              ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w,
+                                  (FUSE && !a.redo) ? &fx : nullptr);
+            }
+            tot_ctx += st.n_ctx; tot_rev += st.n_rev; tot_clamp += st.n_clamp;
+            sm.ch = st.h;
+            sm.n_int = st.n_int;
+            sm.failed = ok ? 0 : 1;
+            if (!a.redo) atomicAdd((u64*)&a.status->n_sequential_tiles, 1ull);
+          }
+          __syncthreads();
+          ch = sm.ch;
+          n_int = sm.n_int;
+          if (sm.failed) stream_failed = true;
+          if (tid < ch) {
+            const ArgusFrame f = sm.fstk[tid];
+            car_next[tid] = make_uint4((u32)f.ts, (u32)(f.ts >> 32), f.region << 1, f.ctx);
+            sm.cchild[cpar ^ 1][tid] = f.child;
+            sm.cidx[cpar ^ 1][tid] = f.idx;
+          }
+          cpar ^= 1;
+          w0 += nseq;
+          wend = tn;
+          ++small_streak;
+          __syncthreads();
+          if (stream_failed) break;
         }
-        __syncthreads();
-        ch = sm.ch;
-        n_int = sm.n_int;
-        if (sm.failed) stream_failed = true;
-        if (tid < ch) {
-          const ArgusFrame f = sm.fstk[tid];
-          car_next[tid] = make_uint4((u32)f.ts, (u32)(f.ts >> 32), f.region << 1, f.ctx);
-          accb[nbase + tid] = f.child;
-          sm.cidx[b ^ 1][tid] = f.idx;
-          sm.cchild[b ^ 1][tid] = f.child;
-        }
-        __syncthreads();
-      }
+      }  // windows
       if (stream_failed) {
         if (ti + 1 < ntiles) {  // drain the prefetched tile before the buffer is reused
           const bool ok = mbar_wait_bounded(&sm.bar[b ^ 1], (b ^ 1) ? ph1 : ph0);
@@ -486,6 +504,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       }
     }  // tiles
 
+
     __syncthreads();
     if (sm.dead) {
       if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, 0);
@@ -493,8 +512,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     }
     if (!a.redo) {
       // frames still open at the end of the stream (they sit in the block the next tile would read)
-      const int bl = (int)(ntiles & 1u);
-      if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[bl][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
+      if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[cpar][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
       if (tid == 0) a.counts[s] = n_int;
     }
     if (FUSE && !a.redo && fx.tab) {
