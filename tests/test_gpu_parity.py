@@ -339,3 +339,40 @@ def test_synthesize_overlap_span_capacity():
                                  max_overlap_spans=512)
     st = res.fetch_status()
     assert int(st["code"]) == 4 and int(st["intervals_required"]) > 512
+
+
+def test_maximum_region_count():
+    """num_regions at its upper bound (65536): pairing, the global-row aggregation path and the one-call
+    pipeline (which cannot host such a table in shared memory and runs the three plain calls)."""
+    R = 65536
+    rng = np.random.default_rng(33)
+    spec = tg.TraceSpec(tg.TINY, 2, 1)
+    evs, offs = [], [0]
+    for s in range(spec.num_streams):
+        ev = random_wellformed(rng, 300, 7, max_height=4)
+        ev = ev.copy()
+        ev["tag"] = ((ev["tag"] >> 1) * 10922 + (R - 1 - 6 * 10922)).astype(np.uint32) << 1 | (ev["tag"] & 1)  # ids up to R-1
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    ev, offs = np.concatenate(evs), np.array(offs, np.uint64)
+    assert int((ev["tag"] >> 1).max()) == R - 1
+
+    class Spec:
+        num_regions, warps_per_cta, cta_sm, num_sms = R, 4, spec.cta_sm, spec.num_sms
+        overlap_pairs = np.array([(R - 1, R - 1 - 10922)], np.uint32)
+    _synthesize_matches(Spec, ev, offs)
+    # one region too many is rejected on the host
+    d_ev, d_off = to_dev(ev, offs)
+    with pytest.raises(argus.ArgusError):
+        argus.argus_pair_intervals(d_ev, d_off, R + 1)
+
+
+def test_single_long_stream_and_many_empty_streams():
+    """One stream of many tiles among empty ones (ragged CSR), and a stream that ends inside a tile."""
+    rng = np.random.default_rng(34)
+    long_ev = random_wellformed(rng, 20000, 5, max_height=9)
+    short_ev = random_wellformed(rng, 3, 5)
+    evs = [make_events([])] * 5 + [long_ev] + [make_events([])] * 3 + [short_ev] + [make_events([])] * 2
+    offs = np.cumsum([0] + [len(e) for e in evs]).astype(np.uint64)
+    for kernel in KERNELS:
+        assert_pair_matches(np.concatenate(evs), offs, 5, kernel)

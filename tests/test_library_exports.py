@@ -50,3 +50,16 @@ def test_host_argument_validation_needs_no_gpu():
     assert rc == 1
     rc = lib.argus_overlap(None, 0, None, 4, 0, None, 1, None, 0, None, None, None, 0, None)
     assert rc == 1
+
+
+def test_header_is_plain_c():
+    """include/argus.h must compile as C (the boundary is a C ABI)."""
+    import subprocess
+    import tempfile
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "t.c")
+        with open(src, "w") as f:
+            f.write('#include "argus.h"\nint main(void) { return sizeof(argus_agg_t) == 576 && sizeof(argus_interval_t) == 48 ? 0 : 1; }\n')
+        exe = os.path.join(d, "t")
+        subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), src, "-o", exe])
+        assert subprocess.call([exe]) == 0
