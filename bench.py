@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 METRIC = "marker events/sec (pair+aggregate+overlap, whole hot path)"
 UNIT = "events/s"
 ALG_BYTES_PER_EVENT = 40.0  # 16 B event read + 48 B interval written per 2 events
+NCU_DRAM_BYTES_PER_EVENT = (668.654080e6 + 922.479616e6) / 38380544  # fused kernel, ncu capture summarised in profiles/
 
 
 def load_peaks():
@@ -272,7 +273,10 @@ def main():
     achieved = ALG_BYTES_PER_EVENT * n_events / (pair_ms * 1e-3) / 1e9 if pair_ms > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "tiled pairing kernel (k_pair_tiled)" + ("" if args.three_calls else " with fused aggregation and overlap selection"), "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "peak_source": peak_src,
-                "traffic": None, "ms_per_launch": pair_ms, "algorithmic_bytes_per_event": ALG_BYTES_PER_EVENT,
+                "traffic": NCU_DRAM_BYTES_PER_EVENT * n_events if args.workload == 3 and not args.three_calls else None,
+                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on a 38.4 M-event "
+                                  "case of the same trace, scaled by events (profiles/)",
+                "ms_per_launch": pair_ms, "algorithmic_bytes_per_event": ALG_BYTES_PER_EVENT,
                 "pipeline_frac": ALG_BYTES_PER_EVENT * n_events / (ms_per_step * 1e-3) / 1e9 / peak}
     kernel_ms = {k: prof_ms[k] / max(prof_n[k], 1) for k in ("pair", "aggregate", "overlap")}
 
@@ -323,6 +327,27 @@ def main():
         cpu_baseline = {"value": len(ev) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "host_cores": os.cpu_count(),
                         "seconds": dt,
                         "sample": f"first {args.cpu_ctas} CTAs = {args.cpu_ctas * spec.warps_per_cta} streams, {len(ev)} events, one pass"}
+        # the same oracle as independent instances, one CTA of the trace each, on all host cores
+        # (the C++ oracle runs outside the interpreter lock; each instance is still single-threaded)
+        from concurrent.futures import ThreadPoolExecutor
+        ncores = len(os.sched_getaffinity(0))
+        offs_all = tg.host_offsets(spec)
+        W = spec.warps_per_cta
+
+        def one_cta(c):
+            e = tg.host_streams(spec, offs_all, c * W, (c + 1) * W, nthreads=1)
+            o = (offs_all[c * W:(c + 1) * W + 1] - offs_all[c * W]).astype(np.uint64)
+            t = time.perf_counter()
+            oracle_step(oracle, e, o, spec, np.zeros(1, np.uint32), 1)
+            return len(e), time.perf_counter() - t
+
+        with ThreadPoolExecutor(ncores) as pool:
+            t0 = time.perf_counter()
+            done = list(pool.map(one_cta, range(min(ncores, spec.num_ctas))))
+            wall = time.perf_counter() - t0
+        cpu_baseline["all_cores"] = {"value": sum(d[0] for d in done) / wall, "unit": UNIT, "cores": ncores,
+                                     "seconds": wall, "sample": f"{len(done)} CTAs, one oracle instance per core "
+                                     "(wall time includes generating each CTA's events on the host)"}
 
     if rank == 0:
         line = {
