@@ -15,12 +15,13 @@
 constexpr u32 kAggWindow = 16;          // histogram bins kept in shared memory per region
 constexpr u32 kAggUnset = 0xffffffffu;  // window base not chosen yet
 constexpr u32 kFuseMaxRegions = 256;    // fused aggregation keeps num_regions * 112 bytes in shared memory
+constexpr u32 kFuseMaxPairs = 128;      // fused overlap selection keeps the pair list (8 bytes a pair) in shared memory
 constexpr u32 kAggCellWords = 72;       // u64 words of one argus_agg_t
 
 struct ArgusAggCell {  // 112 bytes
   u64 sum_incl, sum_excl, min_incl, max_incl;
-  u32 count, nflag, hbase, pad;
-  u32 h[kAggWindow];
+  u32 count_out, nflag, hbase, pad;  // count_out: intervals whose bin fell outside the window
+  u32 h[kAggWindow];                 // the interval count of the region is count_out + the sum of these
 };
 
 struct ArgusFuseArgs {
@@ -64,15 +65,14 @@ __device__ __forceinline__ void argus_fuse_init(ArgusAggCell* tab, u32 num_regio
   }
 }
 
-// count and sums of one cell (the part a thread may instead keep in registers for hot regions)
-__device__ __forceinline__ void argus_fuse_agg_sums(ArgusAggCell& c, u32 count, u64 sum_incl, u64 sum_excl) {
-  atomicAdd(&c.count, count);
+// sums of one cell (the part a thread may instead keep in registers for hot regions)
+__device__ __forceinline__ void argus_fuse_agg_sums(ArgusAggCell& c, u64 sum_incl, u64 sum_excl) {
   argus_atomic_add64_split(&c.sum_incl, sum_incl);
   argus_atomic_add64_split(&c.sum_excl, sum_excl);
 }
 
-// min, max, flag count and histogram bin of one interval
-__device__ __forceinline__ void argus_fuse_agg_rest(const ArgusFuseCtx& fx, ArgusAggCell& c, u32 region, u64 incl, u32 flags) {
+// min, max, flag count and histogram bin of one interval; the bin also counts the interval
+__device__ __forceinline__ void argus_fuse_agg_rest(ArgusAggCell& c, u64* row, u32 region, u64 incl, u32 flags) {
   if (incl < *reinterpret_cast<volatile u64*>(&c.min_incl)) atomicMin(&c.min_incl, incl);
   if (incl > *reinterpret_cast<volatile u64*>(&c.max_incl)) atomicMax(&c.max_incl, incl);
   if (flags) atomicAdd(&c.nflag, 1u);
@@ -84,24 +84,34 @@ __device__ __forceinline__ void argus_fuse_agg_rest(const ArgusFuseCtx& fx, Argu
     hb = old == kAggUnset ? want : old;
   }
   const u32 rel = bin - hb;
-  if (rel < kAggWindow) atomicAdd(&c.h[rel], 1u);
-  else atomicAdd(fx.row + (size_t)region * kAggCellWords + 8 + bin, 1ull);
+  if (rel < kAggWindow) {
+    atomicAdd(&c.h[rel], 1u);
+  } else {
+    atomicAdd(&c.count_out, 1u);
+    atomicAdd(row + (size_t)region * kAggCellWords + 8 + bin, 1ull);
+  }
 }
 
 __device__ __forceinline__ void argus_fuse_aggregate(const ArgusFuseCtx& fx, u32 region, u64 incl, u64 excl, u32 flags) {
   ArgusAggCell& c = fx.tab[region];
-  argus_fuse_agg_sums(c, 1u, incl, excl);
-  argus_fuse_agg_rest(fx, c, region, incl, flags);
+  argus_fuse_agg_sums(c, incl, excl);
+  argus_fuse_agg_rest(c, fx.row, region, incl, flags);
 }
 
-__device__ __forceinline__ void argus_fuse_flush(const ArgusFuseCtx& fx, u32 num_regions, u32 tid, u32 nthreads) {
+__device__ __forceinline__ void argus_fuse_flush(const ArgusAggCell* tab, u64* row, u32 num_regions, u32 tid, u32 nthreads) {
   constexpr u32 kItems = 8 + kAggWindow;
   for (u32 i = tid; i < num_regions * kItems; i += nthreads) {
     const u32 r = i / kItems, f = i % kItems;
-    const ArgusAggCell& c = fx.tab[r];
-    u64* cell = fx.row + (size_t)r * kAggCellWords;
+    const ArgusAggCell& c = tab[r];
+    u64* cell = row + (size_t)r * kAggCellWords;
     switch (f) {
-      case 0: cell[0] = c.count; break;
+      case 0: {
+        u64 n = c.count_out;
+#pragma unroll
+        for (u32 j = 0; j < kAggWindow; ++j) n += c.h[j];
+        cell[0] = n;
+        break;
+      }
       case 1: cell[1] = c.sum_incl; break;
       case 2: cell[2] = c.min_incl; break;
       case 3: cell[3] = c.max_incl; break;

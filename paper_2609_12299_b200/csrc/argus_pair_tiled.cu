@@ -136,26 +136,28 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   const u64 off0 = a.stream_offsets[0];
   u32 tot_ctx = 0, tot_rev = 0, tot_clamp = 0;
   // fused aggregation / overlap selection (first pass only): compact table and pair bitmap follow TileSmem
-  ArgusFuseCtx fx;
-  fx.tab = nullptr; fx.pairbits = nullptr; fx.row = nullptr; fx.sm_index = 0;
+  // (pointers into shared memory stay plain locals derived from the shared array, so that the compiler keeps
+  // their address space; a generic pointer would turn every table access into a generic load or atomic)
+  ArgusAggCell* const tabp = reinterpret_cast<ArgusAggCell*>(smem_raw + ((sizeof(SM) + 15) & ~(size_t)15));
+  u32* const pairbitsp = reinterpret_cast<u32*>(tabp + (FUSE ? a.num_regions : 0u));
+  u32* const pairs_sm = pairbitsp + (a.num_regions + 31) / 32;  // copy of the (producer, consumer) list: [2 K]
+  const bool has_tab = FUSE && !a.redo && a.fuse.warp_tab != nullptr;
+  const bool has_pairs = FUSE && !a.redo && a.fuse.ov_spans != nullptr && a.fuse.num_pairs != 0;
+  u64* row = nullptr;      // global row of the current stream in the warp-scope table
+  u32 sm_index = 0;        // SM of the current stream's CTA
   u64 ovc_base = 0;        // warp-uniform: current chunk of the global overlap span list
   u32 ovc_used = kOvChunk;
-  u32 hot0 = 0xffffffffu, hot1 = 0xffffffffu, hc0 = 0, hc1 = 0;  // hot regions of the current stream, private partial sums
+  u32 hot0 = 0xffffffffu, hot1 = 0xffffffffu;  // hot regions of the current stream, private partial sums
   u64 hsi0 = 0, hsi1 = 0, hse0 = 0, hse1 = 0;
-  if (FUSE && !a.redo) {
-    ArgusAggCell* tab = reinterpret_cast<ArgusAggCell*>(smem_raw + ((sizeof(SM) + 15) & ~(size_t)15));
-    u32* pairbits = reinterpret_cast<u32*>(tab + a.num_regions);
-    if (a.fuse.warp_tab) fx.tab = tab;
-    if (a.fuse.ov_spans && a.fuse.num_pairs) {
-      for (u32 i = tid; i < (a.num_regions + 31) / 32; i += NT) pairbits[i] = 0;
-      __syncthreads();
-      for (u32 i = tid; i < 2 * a.fuse.num_pairs; i += NT) {
-        const u32 r = a.fuse.pairs[i];
-        if (r < a.num_regions) atomicOr(&pairbits[r >> 5], 1u << (r & 31));
-      }
-      fx.pairbits = pairbits;
-      __syncthreads();
+  if (has_pairs) {
+    for (u32 i = tid; i < (a.num_regions + 31) / 32; i += NT) pairbitsp[i] = 0;
+    __syncthreads();
+    for (u32 i = tid; i < 2 * a.fuse.num_pairs; i += NT) {
+      const u32 r = a.fuse.pairs[i];
+      pairs_sm[i] = r;
+      if (r < a.num_regions) atomicOr(&pairbitsp[r >> 5], 1u << (r & 31));
     }
+    __syncthreads();
   }
 #ifdef ARGUS_TILE_TIMING
   unsigned long long tt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -186,16 +188,16 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     u64 n_int = 0;       // intervals of this stream so far (uniform)
     bool stream_failed = false;
     if (FUSE && !a.redo) {
-      if (fx.tab) {
-        argus_fuse_init(fx.tab, a.num_regions, tid, NT);
-        fx.row = a.fuse.warp_tab + (size_t)s * a.num_regions * kAggCellWords;
-        hot0 = hot1 = 0xffffffffu; hc0 = hc1 = 0; hsi0 = hsi1 = hse0 = hse1 = 0;
+      if (has_tab) {
+        argus_fuse_init(tabp, a.num_regions, tid, NT);
+        row = a.fuse.warp_tab + (size_t)s * a.num_regions * kAggCellWords;
+        hot0 = hot1 = 0xffffffffu; hsi0 = hsi1 = hse0 = hse1 = 0;
         if (tid < 2) sm.hot[tid] = 0xffffffffu;
       }
-      if (fx.pairbits) {
+      if (has_pairs) {
         const u32 m = a.fuse.cta_sm[s / a.fuse.warps_per_cta];
         if (m >= a.fuse.num_sms && tid == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
-        fx.sm_index = m < a.fuse.num_sms ? m : 0;
+        sm_index = m < a.fuse.num_sms ? m : 0;
       }
       __syncthreads();
     }
@@ -353,11 +355,10 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         if (badpos >= wend) {
           // ---------------- phase C: exclusive time, parent region, interval records; carried stack -------------
           const u64 pos0 = out_base + n_int;
+          u32 ovmask = 0;  // bit i: this thread's i-th interval belongs to a designated overlap region
 #pragma unroll
           for (int i = 0; i < NI; ++i) {
             const int rk = tid + i * NT;
-            u32 f_region = 0xffffffffu;  // region / begin / inclusive time of this thread's interval, for the fused hooks
-            u64 f_begin = 0, f_incl = 0;
             if (rk < win_ne) {
               const u32 d = sm.desc[rk];
               const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
@@ -383,39 +384,54 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
                 a.ctl->spec_overflow = 1;
               }
               if (FUSE && !a.redo) {
-                f_region = pe.z >> 1; f_begin = bts; f_incl = incl;
-                if (fx.tab) {
-                  ArgusAggCell& cell = fx.tab[f_region];
-                  if (f_region == hot0) { ++hc0; hsi0 += incl; hse0 += excl; }
-                  else if (f_region == hot1) { ++hc1; hsi1 += incl; hse1 += excl; }
-                  else argus_fuse_agg_sums(cell, 1u, incl, excl);
-                  argus_fuse_agg_rest(fx, cell, f_region, incl, flags);
+                const u32 f_region = pe.z >> 1;
+                if (has_pairs && incl && ((pairbitsp[f_region >> 5] >> (f_region & 31)) & 1u)) ovmask |= 1u << i;
+                if (has_tab) {
+                  ArgusAggCell& cell = tabp[f_region];
+                  if (f_region == hot0) { hsi0 += incl; hse0 += excl; }
+                  else if (f_region == hot1) { hsi1 += incl; hse1 += excl; }
+                  else argus_fuse_agg_sums(cell, incl, excl);
+                  argus_fuse_agg_rest(cell, row, f_region, incl, flags);
                 }
               }
             }
-            if (FUSE && !a.redo && fx.pairbits) {  // every lane takes part: spans are appended a warp at a time
-              const bool cand = f_region != 0xffffffffu && f_incl && ((fx.pairbits[f_region >> 5] >> (f_region & 31)) & 1u);
-              if (__ballot_sync(0xffffffffu, cand)) {
-                for (u32 k = 0; k < 2 * a.fuse.num_pairs; ++k) {
-                  const bool sel = cand && a.fuse.pairs[k] == f_region;
-                  const u32 bal = __ballot_sync(0xffffffffu, sel);
-                  if (!bal) continue;
-                  const u32 c = __popc(bal);
-                  if (ovc_used + c > kOvChunk) {
-                    u64 nb64 = 0;
-                    if (lane == 0) nb64 = atomicAdd(a.fuse.ov_count, (u64)kOvChunk);
-                    ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
-                    ovc_used = 0;
-                  }
-                  if (sel) {
-                    const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
-                    if (slot < a.fuse.ov_capacity) {
-                      a.fuse.ov_spans[slot] = make_ulonglong2(f_begin, f_begin + f_incl);
-                      a.fuse.ov_seg[slot] = ((k >> 1) * a.fuse.num_sms + fx.sm_index) * 2 + (k & 1u);
-                    }
-                  }
-                  ovc_used += c;
+          }
+          // Overlap selection: intervals of a designated region are rare in most traces, so the loop above only
+          // notes them; when some lane of the warp has one, the warp appends their spans together here.
+          if (has_pairs && __any_sync(0xffffffffu, ovmask != 0)) {
+#pragma unroll
+            for (int i = 0; i < NI; ++i) {
+              const bool cand = (ovmask >> i) & 1u;
+              if (!__ballot_sync(0xffffffffu, cand)) continue;
+              u32 f_region = 0xffffffffu;
+              u64 f_begin = 0, f_end = 0;
+              if (cand) {
+                const u32 d = sm.desc[tid + i * NT];
+                const uint4 ee = evb[d & 0xffffu];
+                const uint4 pe = evb[(int)(short)(refs[i] & 0xffffu)];
+                f_region = pe.z >> 1;
+                f_begin = (u64)pe.x | ((u64)pe.y << 32);
+                f_end = (u64)ee.x | ((u64)ee.y << 32);
+              }
+              for (u32 k = 0; k < 2 * a.fuse.num_pairs; ++k) {
+                const bool sel = cand && pairs_sm[k] == f_region;
+                const u32 bal = __ballot_sync(0xffffffffu, sel);
+                if (!bal) continue;
+                const u32 c = __popc(bal);
+                if (ovc_used + c > kOvChunk) {
+                  u64 nb64 = 0;
+                  if (lane == 0) nb64 = atomicAdd(a.fuse.ov_count, (u64)kOvChunk);
+                  ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
+                  ovc_used = 0;
                 }
+                if (sel) {
+                  const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
+                  if (slot < a.fuse.ov_capacity) {
+                    a.fuse.ov_spans[slot] = make_ulonglong2(f_begin, f_end);
+                    a.fuse.ov_seg[slot] = ((k >> 1) * a.fuse.num_sms + sm_index) * 2 + (k & 1u);
+                  }
+                }
+                ovc_used += c;
               }
             }
           }
@@ -427,11 +443,14 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             sm.cchild[cpar ^ 1][tid] = accb[from];
             sm.cidx[cpar ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[cpar][tid];
           }
-          if (FUSE && !a.redo && fx.tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0 && warp == 0) {
+          if (has_tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0 && warp == 0) {
             // top two regions by count so far (counts may still be moving: only a heuristic)
             u32 best = 0, second = 0;
             for (u32 r = lane; r < a.num_regions; r += 32) {
-              const u32 key = (*reinterpret_cast<volatile u32*>(&fx.tab[r].count) << 16) | r;
+              u32 cnt = *reinterpret_cast<volatile u32*>(&tabp[r].count_out);
+#pragma unroll
+              for (u32 j = 0; j < kAggWindow; ++j) cnt += *reinterpret_cast<volatile u32*>(&tabp[r].h[j]);
+              const u32 key = ((cnt > 0xffffu ? 0xffffu : cnt) << 16) | r;
               if (key > best) { second = best; best = key; } else if (key > second) { second = key; }
             }
             const u32 top = __reduce_max_sync(0xffffffffu, best);
@@ -439,7 +458,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             const u32 next = __reduce_max_sync(0xffffffffu, cand);
             if (lane == 0) { sm.hot[0] = (top >> 16) ? (top & 0xffffu) : 0xffffffffu; sm.hot[1] = (next >> 16) ? (next & 0xffffu) : 0xffffffffu; }
           }
-          const bool pick_hot = FUSE && !a.redo && fx.tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0;
+          const bool pick_hot = has_tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0;
           small_streak = (wend - w0 < 32) ? small_streak + 1 : 0;
           ch = new_ch;
           n_int += (u64)win_ne;
@@ -462,6 +481,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           }
           __syncthreads();
           if (tid == 0) {
+            ArgusFuseCtx fx;  // the sequential machine is shared with the other pairing kernels and takes the context as a struct
+            fx.tab = has_tab ? tabp : nullptr; fx.pairbits = has_pairs ? pairbitsp : nullptr; fx.row = row; fx.sm_index = sm_index;
             ArgusSeqState st;
             st.h = ch; st.n_int = n_int; st.n_ctx = st.n_rev = st.n_clamp = 0; st.failed = false;
             bool ok = true;
@@ -515,11 +536,11 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[cpar][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
       if (tid == 0) a.counts[s] = n_int;
     }
-    if (FUSE && !a.redo && fx.tab) {
-      if (hc0) argus_fuse_agg_sums(fx.tab[hot0], hc0, hsi0, hse0);
-      if (hc1) argus_fuse_agg_sums(fx.tab[hot1], hc1, hsi1, hse1);
+    if (has_tab) {
+      if (hot0 != 0xffffffffu) argus_fuse_agg_sums(tabp[hot0], hsi0, hse0);
+      if (hot1 != 0xffffffffu) argus_fuse_agg_sums(tabp[hot1], hsi1, hse1);
       __syncthreads();
-      argus_fuse_flush(fx, a.num_regions, tid, NT);
+      argus_fuse_flush(tabp, row, a.num_regions, tid, NT);
     }
     __syncthreads();
   }  // streams
@@ -544,7 +565,7 @@ int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   static int grid_cache = 0;
   static size_t smem_cache = 0;
   size_t smem = ((sizeof(TileSmem<NT, E>) + 15) & ~(size_t)15) + 128;
-  if (FUSE) smem += (size_t)a.num_regions * sizeof(ArgusAggCell) + ((a.num_regions + 31) / 32) * 4 + 16;
+  if (FUSE) smem += (size_t)a.num_regions * sizeof(ArgusAggCell) + ((a.num_regions + 31) / 32) * 4 + (size_t)a.fuse.num_pairs * 8 + 16;
   if (!grid_cache || smem_cache != smem) {
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int dev = 0, sms = 0, per_sm = 0;
@@ -575,6 +596,7 @@ int g_variant = 0;
 bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0; }
 
 bool argus_pair_tiled_can_fuse(uint32_t num_regions) { return num_regions <= kFuseMaxRegions; }
+bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs) { return num_pairs <= kFuseMaxPairs; }
 
 #ifdef ARGUS_TILE_TIMING
 // Debug build only: cycles thread 0 of every CTA spent per phase (other, wait, A, B, C), summed; resets them.

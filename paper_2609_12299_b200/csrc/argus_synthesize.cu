@@ -30,6 +30,7 @@ int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* lis
                                      uint64_t list_capacity, uint32_t num_sms, uint32_t num_pairs, argus_overlap_t* out,
                                      argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 bool argus_pair_tiled_can_fuse(uint32_t num_regions);
+bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs);
 
 namespace {
 
@@ -91,7 +92,7 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
     f.warp_tab = (u64*)warp_work;
     ARGUS_CUDA_TRY(cudaMemsetAsync(warp_work, 0, (size_t)num_streams * row_bytes, stream));
   }
-  if (can_fuse && num_pairs) {
+  if (can_fuse && num_pairs && argus_pair_tiled_can_fuse_overlap(num_pairs)) {
     f.ov_spans = (ulonglong2*)(ws + L.list_spans);
     f.ov_seg = (u32*)(ws + L.list_seg);
     f.ov_capacity = max_overlap_spans;
