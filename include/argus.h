@@ -280,6 +280,78 @@ int argus_overlap(const argus_interval_t* intervals /*device*/, uint64_t max_int
                   size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Scope selection — Section 1 (the observe(region, signals, scope) query) and Section 3.2
+ * "Region and scope": the region is the code being asked about, the scope picks which of
+ * its dynamic executions count, by the role of the warp, by a window of iterations or by a
+ * subset of SMs.
+ *
+ * An interval belongs to a scope when all four tests hold:
+ *   iteration window : ctx_lo <= interval.ctx <= ctx_hi  (ctx is the begin marker's)
+ *   warp role        : bit (interval.stream % warps_per_cta) of warp_mask is set
+ *                      (warps 64 and up of a CTA are never selected unless warp_mask is all ones)
+ *   SM subset        : bit cta_sm[interval.stream / warps_per_cta] of sm_mask is set
+ *   region set       : bit interval.region of region_mask is set
+ * sm_mask and region_mask are DEVICE arrays of ceil(num_sms / 32) and ceil(num_regions / 32)
+ * words (bit i of word i / 32); NULL selects everything. The struct itself is read on the
+ * host at call time. An ambiguity record is tested the same way with its own ctx, stream and
+ * tag >> 1. Inclusive and exclusive times are those pairing computed over the whole stream:
+ * selection does not change them.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  uint32_t ctx_lo, ctx_hi;       /* inclusive on both ends; 0 .. UINT32_MAX selects all      */
+  uint64_t warp_mask;            /* UINT64_MAX selects all                                    */
+  const uint32_t* sm_mask;       /* device, nullable                                          */
+  const uint32_t* region_mask;   /* device, nullable                                          */
+} argus_scope_t;
+
+#define ARGUS_MAX_ITER_ROWS 65536u /* rows of an iteration table (ctx_hi - ctx_lo + 1)        */
+
+/* ---------------------------------------------------------------------------------------
+ * argus_aggregate_scoped — argus_aggregate over the intervals (and ambiguity records) of one
+ * scope, plus two tables keyed the way the paper's queries select executions:
+ *   role_tab[W][R] : key = warp index inside its CTA (stream % warps_per_cta), which is the
+ *                    role of the warp in a warp-specialised kernel (the GEMM example of
+ *                    Section 1 measures per role and per iteration), reduced over all CTAs;
+ *   iter_tab[I][R] : key = ctx - ctx_lo, I = ctx_hi - ctx_lo + 1 <= ARGUS_MAX_ITER_ROWS:
+ *                    per-iteration statistics across warps (the worked example of Section 3.1
+ *                    selects sixteen pipeline iterations). Needs a non-NULL scope.
+ * scope == NULL selects everything; then warp/cta/sm/kernel tables equal argus_aggregate's.
+ * Every cell of a requested table is written. Workspace: argus_aggregate_workspace_bytes.
+ * Errors as argus_aggregate; ARGUS_ERR_INVALID_ARG also when iter_tab is given without a
+ * scope or with more than ARGUS_MAX_ITER_ROWS rows, or ctx_hi < ctx_lo.
+ * ------------------------------------------------------------------------------------- */
+int argus_aggregate_scoped(const argus_interval_t* intervals /*device*/,
+                           const uint64_t* interval_offsets /*device [S+1]*/,
+                           const argus_ambiguity_t* ambig /*device, nullable*/,
+                           const uint64_t* ambig_offsets /*device [S+1], nullable*/,
+                           uint32_t num_streams, uint32_t warps_per_cta,
+                           const uint32_t* cta_sm /*device [C]*/, uint32_t num_sms,
+                           uint32_t num_regions, const argus_scope_t* scope /*host, nullable*/,
+                           argus_agg_t* warp_tab /*device [S][R], nullable*/,
+                           argus_agg_t* cta_tab /*device [C][R], nullable*/,
+                           argus_agg_t* sm_tab /*device [M][R], nullable*/,
+                           argus_agg_t* kernel_tab /*device [R], nullable*/,
+                           argus_agg_t* role_tab /*device [W][R], nullable*/,
+                           argus_agg_t* iter_tab /*device [I][R], nullable*/,
+                           argus_status_t* status /*device*/, void* workspace /*device*/,
+                           size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
+ * argus_overlap_scoped — argus_overlap over the intervals of one scope (for instance the
+ * producer/consumer overlap of a few pipeline iterations on a subset of SMs). scope == NULL
+ * selects everything. out[k][m] of an SM outside the scope is all zero. Workspace:
+ * argus_overlap_workspace_bytes.
+ * ------------------------------------------------------------------------------------- */
+int argus_overlap_scoped(const argus_interval_t* intervals /*device*/, uint64_t max_intervals,
+                         const uint64_t* interval_offsets /*device [S+1]*/,
+                         uint32_t num_streams, uint32_t warps_per_cta,
+                         const uint32_t* cta_sm /*device [C]*/, uint32_t num_sms,
+                         const uint32_t* pairs /*device [K][2]*/, uint32_t num_pairs,
+                         const argus_scope_t* scope /*host, nullable*/,
+                         argus_overlap_t* out /*device [K][M]*/, argus_status_t* status /*device*/,
+                         void* workspace /*device*/, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
  * argus_synthesize — the three operations above in one call, with identical results
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *

@@ -54,7 +54,10 @@ def _load():
         lib.oracle_pair.argtypes = [vp, vp, u32, u32, vp, u64, vp, vp, u64, vp, vp]
         lib.oracle_aggregate.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp]
         lib.oracle_overlap.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp]
-        for f in (lib.oracle_pair, lib.oracle_aggregate, lib.oracle_overlap):
+        lib.oracle_aggregate_scoped.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_overlap_scoped.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp]
+        for f in (lib.oracle_pair, lib.oracle_aggregate, lib.oracle_overlap, lib.oracle_aggregate_scoped,
+                  lib.oracle_overlap_scoped):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -115,4 +118,77 @@ def overlap(intervals, interval_offsets, warps_per_cta, cta_sm, num_sms, pairs):
     st = np.zeros(1, dtype=STATUS)
     rc = _load().oracle_overlap(_ptr(iv), _ptr(ioffs), S, warps_per_cta, _ptr(cs), num_sms, _ptr(pr), len(pr),
                                 _ptr(out), _ptr(st))
+    return rc, out, st[0]
+
+
+class _OScope(ctypes.Structure):
+    _fields_ = [("ctx_lo", ctypes.c_uint32), ("ctx_hi", ctypes.c_uint32), ("warp_mask", ctypes.c_uint64),
+                ("sm_mask", ctypes.c_void_p), ("region_mask", ctypes.c_void_p)]
+
+
+def _bitmask(selected, n):
+    """Bit i of word i // 32 set for every i in `selected` (an iterable of indices < n)."""
+    words = np.zeros((n + 31) // 32, dtype=np.uint32)
+    for i in selected:
+        assert 0 <= int(i) < n
+        words[int(i) // 32] |= np.uint32(1 << (int(i) % 32))
+    return words
+
+
+def _scope_struct(scope, num_sms, num_regions):
+    """scope: None or a dict with optional keys ctx (lo, hi), warps (indices inside a CTA), sms, regions.
+    Returns (struct or None, arrays to keep alive)."""
+    if scope is None:
+        return None, ()
+    lo, hi = scope.get("ctx", (0, 0xFFFFFFFF))
+    warps = scope.get("warps")
+    wm = 0xFFFFFFFFFFFFFFFF if warps is None else sum(1 << int(w) for w in set(warps))
+    sm = None if scope.get("sms") is None else _bitmask(scope["sms"], num_sms)
+    rg = None if scope.get("regions") is None else _bitmask(scope["regions"], num_regions)
+    return _OScope(int(lo), int(hi), wm, _ptr(sm), _ptr(rg)), (sm, rg)
+
+
+def aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, warps_per_cta, cta_sm, num_sms, num_regions,
+                     scope=None, levels=("warp", "cta", "sm", "kernel", "role", "iter")):
+    """Returns (rc, {level: table [keys, R]}, status); level "iter" needs a scope with a ctx window."""
+    iv = np.ascontiguousarray(intervals, dtype=INTERVAL)
+    ioffs = np.ascontiguousarray(interval_offsets, dtype=np.uint64)
+    S = len(ioffs) - 1
+    am = None if ambig is None else np.ascontiguousarray(ambig, dtype=AMBIG)
+    aoffs = None if ambig_offsets is None else np.ascontiguousarray(ambig_offsets, dtype=np.uint64)
+    cs = np.ascontiguousarray(cta_sm, dtype=np.uint32)
+    C = S // warps_per_cta if warps_per_cta else 0
+    sc, keep = _scope_struct(scope, num_sms, num_regions)
+    n_iter = 0
+    if "iter" in levels and scope is not None and "ctx" in scope:
+        n_iter = int(scope["ctx"][1]) - int(scope["ctx"][0]) + 1
+        if tuple(int(x) for x in scope["ctx"]) == (0, 0xFFFFFFFF):
+            n_iter = 0       # the all-selecting window: no iteration table
+        elif n_iter > 65536:
+            n_iter = 1       # too many rows: the call is refused before it touches the table
+    keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1, "role": warps_per_cta, "iter": n_iter}
+    tabs = {lv: (np.zeros((keys[lv], num_regions), dtype=AGG) if lv in levels and (lv != "iter" or n_iter > 0) else None)
+            for lv in keys}
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_aggregate_scoped(_ptr(iv), _ptr(ioffs), _ptr(am), _ptr(aoffs), S, warps_per_cta, _ptr(cs), num_sms,
+                                         num_regions, None if sc is None else ctypes.addressof(sc), _ptr(tabs["warp"]),
+                                         _ptr(tabs["cta"]), _ptr(tabs["sm"]), _ptr(tabs["kernel"]), _ptr(tabs["role"]),
+                                         _ptr(tabs["iter"]), _ptr(st))
+    del keep
+    return rc, {k: v for k, v in tabs.items() if v is not None}, st[0]
+
+
+def overlap_scoped(intervals, interval_offsets, warps_per_cta, cta_sm, num_sms, pairs, scope=None, num_regions=65536):
+    """Returns (rc, out [K, M], status)."""
+    iv = np.ascontiguousarray(intervals, dtype=INTERVAL)
+    ioffs = np.ascontiguousarray(interval_offsets, dtype=np.uint64)
+    S = len(ioffs) - 1
+    cs = np.ascontiguousarray(cta_sm, dtype=np.uint32)
+    pr = np.ascontiguousarray(pairs, dtype=np.uint32).reshape(-1, 2)
+    out = np.zeros((len(pr), num_sms), dtype=OVERLAP)
+    st = np.zeros(1, dtype=STATUS)
+    sc, keep = _scope_struct(scope, num_sms, num_regions)
+    rc = _load().oracle_overlap_scoped(_ptr(iv), _ptr(ioffs), S, warps_per_cta, _ptr(cs), num_sms, _ptr(pr), len(pr),
+                                       None if sc is None else ctypes.addressof(sc), _ptr(out), _ptr(st))
+    del keep
     return rc, out, st[0]

@@ -261,3 +261,129 @@ extern "C" int oracle_overlap(const OInterval* intervals, const uint64_t* interv
   }
   return OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Scope selection (Section 1, the observe(region, signals, scope) query; Section 3.2 "Region and
+// scope"). The four tests of membership, written out once; everything else repeats the plain
+// definitions above on the selected records.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+bool bit_set(const uint32_t* mask, uint32_t i) { return mask == nullptr || ((mask[i / 32] >> (i % 32)) & 1u) != 0; }
+
+bool in_scope(const OScope* sc, uint32_t stream, uint32_t ctx, uint32_t region, uint32_t warps_per_cta,
+              const uint32_t* cta_sm) {
+  if (sc == nullptr) return true;
+  if (ctx < sc->ctx_lo || ctx > sc->ctx_hi) return false;                       // iteration window
+  const uint32_t w = stream % warps_per_cta;                                      // warp role
+  if (sc->warp_mask != ~0ull && (w >= 64 || ((sc->warp_mask >> w) & 1ull) == 0)) return false;
+  if (sc->sm_mask != nullptr && cta_sm != nullptr && !bit_set(sc->sm_mask, cta_sm[stream / warps_per_cta])) return false;
+  return bit_set(sc->region_mask, region);                                        // region set
+}
+
+}  // namespace
+
+extern "C" int oracle_aggregate_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
+                                       const OAmbig* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                                       uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                                       uint32_t num_regions, const OScope* scope, OAgg* warp_tab, OAgg* cta_tab,
+                                       OAgg* sm_tab, OAgg* kernel_tab, OAgg* role_tab, OAgg* iter_tab, OStatus* st) {
+  if (!interval_offsets || !st || warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ERR_INVALID;
+  if (num_regions == 0 || num_regions > 65536) return ERR_INVALID;
+  if ((sm_tab != nullptr || (scope && scope->sm_mask)) && (!cta_sm || num_sms == 0)) return ERR_INVALID;
+  if (scope && scope->ctx_hi < scope->ctx_lo) return ERR_INVALID;
+  if (iter_tab && (!scope || scope->ctx_hi - scope->ctx_lo >= 65536u)) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  const uint32_t num_ctas = num_streams / warps_per_cta;
+  const uint32_t num_iters = iter_tab ? scope->ctx_hi - scope->ctx_lo + 1 : 0;
+  std::map<Key, Cell> m;  // levels 0..3 as in oracle_aggregate, 4 = warp role, 5 = iteration
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    uint32_t keys[6];
+    keys[0] = s;
+    keys[1] = s / warps_per_cta;
+    keys[2] = cta_sm ? cta_sm[s / warps_per_cta] : 0;
+    keys[3] = 0;
+    keys[4] = s % warps_per_cta;
+    if (cta_sm && keys[2] >= num_sms && (sm_tab || (scope && scope->sm_mask))) return ERR_INVALID;
+    for (uint64_t i = interval_offsets[s]; i < interval_offsets[s + 1]; ++i) {
+      const OInterval& v = intervals[i];
+      if (v.region >= num_regions) { fail(st, ERR_BAD_REGION, s, i); return OK; }
+      if (!in_scope(scope, s, v.ctx, v.region, warps_per_cta, cta_sm)) continue;
+      keys[5] = scope ? v.ctx - scope->ctx_lo : 0;
+      for (int level = 0; level < 6; ++level) {
+        if (level == 5 && !iter_tab) continue;
+        OAgg& a = m[Key(level, keys[level], v.region)].a;
+        a.count++;
+        a.sum_incl += v.inclusive;
+        a.min_incl = std::min(a.min_incl, v.inclusive);
+        a.max_incl = std::max(a.max_incl, v.inclusive);
+        a.sum_excl += v.exclusive;
+        a.n_flagged += (v.flags != 0);
+        a.hist[bin_of(v.inclusive)]++;
+      }
+    }
+    if (ambig && ambig_offsets) {
+      for (uint64_t i = ambig_offsets[s]; i < ambig_offsets[s + 1]; ++i) {
+        const OAmbig& r = ambig[i];
+        const uint32_t region = r.tag >> 1;
+        if (region >= num_regions) { fail(st, ERR_BAD_REGION, s, i); return OK; }
+        if (!in_scope(scope, s, r.ctx, region, warps_per_cta, cta_sm)) continue;
+        keys[5] = scope ? r.ctx - scope->ctx_lo : 0;
+        for (int level = 0; level < 6; ++level) {
+          if (level == 5 && !iter_tab) continue;
+          OAgg& a = m[Key(level, keys[level], region)].a;
+          if (r.kind == AMB_END) a.n_unmatched_end++; else a.n_unmatched_begin++;
+        }
+      }
+    }
+  }
+  materialise(m, 0, num_streams, num_regions, warp_tab);
+  materialise(m, 1, num_ctas, num_regions, cta_tab);
+  materialise(m, 2, num_sms, num_regions, sm_tab);
+  materialise(m, 3, 1, num_regions, kernel_tab);
+  materialise(m, 4, warps_per_cta, num_regions, role_tab);
+  materialise(m, 5, num_iters, num_regions, iter_tab);
+  return OK;
+}
+
+extern "C" int oracle_overlap_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
+                                     uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,
+                                     uint32_t num_sms, const uint32_t* pairs, uint32_t num_pairs,
+                                     const OScope* scope, OOverlap* out, OStatus* st) {
+  if (!interval_offsets || !cta_sm || !st || warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ERR_INVALID;
+  if (num_pairs && (!pairs || !out)) return ERR_INVALID;
+  if (scope && scope->ctx_hi < scope->ctx_lo) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  for (uint32_t s = 0; s < num_streams; ++s)
+    if (cta_sm[s / warps_per_cta] >= num_sms) return ERR_INVALID;
+  for (uint32_t k = 0; k < num_pairs; ++k) {
+    const uint32_t P = pairs[2 * k], Cn = pairs[2 * k + 1];
+    for (uint32_t sm = 0; sm < num_sms; ++sm) {
+      std::vector<Span> p, c;
+      for (uint32_t s = 0; s < num_streams; ++s) {
+        if (cta_sm[s / warps_per_cta] != sm) continue;
+        for (uint64_t i = interval_offsets[s]; i < interval_offsets[s + 1]; ++i) {
+          const OInterval& v = intervals[i];
+          if (v.inclusive == 0) continue;  // empty span
+          if (!in_scope(scope, s, v.ctx, v.region, warps_per_cta, cta_sm)) continue;
+          const Span sp(v.t_begin, v.t_begin + v.inclusive);
+          if (v.region == P) p.push_back(sp);
+          if (v.region == Cn) c.push_back(sp);
+        }
+      }
+      const std::vector<Span> up = merged_union(p), uc = merged_union(c);
+      uint64_t both = 0;
+      for (const Span& x : up)        // every producer piece against every consumer piece
+        for (const Span& y : uc) {
+          const uint64_t lo = std::max(x.first, y.first), hi = std::min(x.second, y.second);
+          if (hi > lo) both += hi - lo;
+        }
+      OOverlap& o = out[static_cast<uint64_t>(k) * num_sms + sm];
+      o.producer_ns = measure(up);
+      o.consumer_ns = measure(uc);
+      o.overlap_ns = both;
+      o.either_ns = o.producer_ns + o.consumer_ns - both;
+    }
+  }
+  return OK;
+}

@@ -58,5 +58,32 @@ int oracle_overlap(const OInterval* intervals, const uint64_t* interval_offsets,
                    uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,
                    uint32_t num_sms, const uint32_t* pairs, uint32_t num_pairs, OOverlap* out,
                    OStatus* st);
+
+// Scope selection (paper Section 1, the observe(region, signals, scope) query; Section 3.2
+// "Region and scope"): which executions of a region count, chosen by iteration window
+// (ctx_lo <= ctx <= ctx_hi), warp role (bit stream % warps_per_cta of warp_mask), SM subset
+// (bit cta_sm[cta] of sm_mask) and region set (bit region of region_mask). Null masks select
+// everything. Host pointers.
+struct OScope {
+  uint32_t ctx_lo, ctx_hi;
+  uint64_t warp_mask;
+  const uint32_t* sm_mask;
+  const uint32_t* region_mask;
+};
+
+// oracle_aggregate over the selected intervals and ambiguity records only, plus role_tab[W][R]
+// (key = stream % warps_per_cta) and iter_tab[ctx_hi - ctx_lo + 1][R] (key = ctx - ctx_lo).
+// scope may be null (everything); iter_tab needs a scope.
+int oracle_aggregate_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
+                            const OAmbig* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                            uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                            uint32_t num_regions, const OScope* scope, OAgg* warp_tab, OAgg* cta_tab,
+                            OAgg* sm_tab, OAgg* kernel_tab, OAgg* role_tab, OAgg* iter_tab, OStatus* st);
+
+// oracle_overlap over the selected intervals only.
+int oracle_overlap_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
+                          uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,
+                          uint32_t num_sms, const uint32_t* pairs, uint32_t num_pairs,
+                          const OScope* scope, OOverlap* out, OStatus* st);
 }
 #endif
