@@ -9,7 +9,8 @@ from .binding import (AGG_DTYPE, AMBIG_DTYPE, EVENT_DTYPE, INTERVAL_DTYPE, OVERL
                       argus_overlap_workspace_bytes, argus_pair_intervals, argus_pair_workspace_bytes,
                       argus_launch_count, argus_profile_enable, argus_profile_read, argus_status_fetch, argus_strerror,
                       argus_version, library_path, load_library, pair_aggregate_host, argus_synthesize,
-                      argus_synthesize_workspace_bytes, SynthesizeResult, argus_pair_intervals_static)
+                      argus_synthesize_workspace_bytes, SynthesizeResult, argus_pair_intervals_static, ArgusScope,
+                      ScopedAggregateResult, argus_aggregate_scoped, argus_overlap_scoped)
 
 __all__ = [
     "AGG_DTYPE", "AMBIG_DTYPE", "EVENT_DTYPE", "INTERVAL_DTYPE", "OVERLAP_DTYPE", "STATUS_DTYPE", "ArgusError",
@@ -17,5 +18,6 @@ __all__ = [
     "argus_overlap_workspace_bytes", "argus_pair_intervals", "argus_pair_workspace_bytes", "argus_status_fetch",
     "argus_strerror", "argus_version", "library_path", "load_library", "pair_aggregate_host", "argus_launch_count",
     "argus_profile_enable", "argus_profile_read", "argus_synthesize", "argus_synthesize_workspace_bytes",
-    "SynthesizeResult", "argus_pair_intervals_static",
+    "SynthesizeResult", "argus_pair_intervals_static", "ArgusScope", "ScopedAggregateResult", "argus_aggregate_scoped",
+    "argus_overlap_scoped",
 ]

@@ -66,6 +66,10 @@ def load_library():
     lib.argus_overlap_workspace_bytes.restype = sz
     lib.argus_overlap.argtypes = [vp, u64, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp, sz, vp]
     lib.argus_overlap.restype = ci
+    lib.argus_aggregate_scoped.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.argus_aggregate_scoped.restype = ci
+    lib.argus_overlap_scoped.argtypes = [vp, u64, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp, vp, sz, vp]
+    lib.argus_overlap_scoped.restype = ci
     lib.argus_status_fetch.argtypes = [vp, vp, vp]
     lib.argus_status_fetch.restype = ci
     lib.argus_strerror.argtypes = [ci]
@@ -285,6 +289,84 @@ def argus_overlap(intervals: torch.Tensor, max_intervals: int, interval_offsets:
                            _stream_ptr(dev))
     if rc != 0:
         raise ArgusError(rc, "argus_overlap")
+    return out, status
+
+
+class _ScopeStruct(ctypes.Structure):  # argus_scope_t
+    _fields_ = [("ctx_lo", ctypes.c_uint32), ("ctx_hi", ctypes.c_uint32), ("warp_mask", ctypes.c_uint64),
+                ("sm_mask", ctypes.c_void_p), ("region_mask", ctypes.c_void_p)]
+
+
+@dataclass
+class ArgusScope:
+    """argus_scope_t: which executions of a region count. `sm_mask` / `region_mask` are device int32
+    tensors of ceil(n / 32) words (bit i of word i // 32), or None for "all"."""
+    ctx_lo: int = 0
+    ctx_hi: int = 0xFFFFFFFF
+    warp_mask: int = 0xFFFFFFFFFFFFFFFF
+    sm_mask: torch.Tensor | None = None
+    region_mask: torch.Tensor | None = None
+
+    @staticmethod
+    def bitmask(selected, n: int, device) -> torch.Tensor:
+        """Device mask of n bits with the bits in `selected` set (argument marshalling only)."""
+        words = np.zeros((n + 31) // 32, dtype=np.uint32)
+        for i in selected:
+            words[int(i) // 32] |= np.uint32(1 << (int(i) % 32))
+        return torch.from_numpy(words.view(np.int32)).to(device)
+
+    def _struct(self) -> _ScopeStruct:
+        return _ScopeStruct(self.ctx_lo, self.ctx_hi, self.warp_mask, _ptr(self.sm_mask), _ptr(self.region_mask))
+
+
+@dataclass
+class ScopedAggregateResult(AggregateResult):
+    role: torch.Tensor | None = None   # uint8 [W * R * 576]
+    iter: torch.Tensor | None = None   # uint8 [(ctx_hi - ctx_lo + 1) * R * 576]
+
+
+def argus_aggregate_scoped(intervals: torch.Tensor, interval_offsets: torch.Tensor, ambig: torch.Tensor | None,
+                           ambig_offsets: torch.Tensor | None, warps_per_cta: int, cta_sm: torch.Tensor, num_sms: int,
+                           num_regions: int, scope: ArgusScope | None,
+                           levels=("warp", "cta", "sm", "kernel", "role")) -> ScopedAggregateResult:
+    """levels may also name "iter" (needs a scope; one row per ctx of its window)."""
+    lib = load_library()
+    dev = intervals.device
+    S = interval_offsets.numel() - 1
+    C = S // warps_per_cta if warps_per_cta else 0
+    n_iter = scope.ctx_hi - scope.ctx_lo + 1 if (scope is not None and "iter" in levels) else 0
+    keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1, "role": warps_per_cta, "iter": max(n_iter, 0)}
+    tabs = {lv: (_bytes(max(keys[lv], 1) * num_regions * 576, dev) if lv in levels else None) for lv in keys}
+    ws = _bytes(lib.argus_aggregate_workspace_bytes(intervals.numel() // 48, S, num_regions), dev)
+    out = ScopedAggregateResult(tabs["warp"], tabs["cta"], tabs["sm"], tabs["kernel"], _bytes(64, dev), ws,
+                                {lv: (keys[lv], num_regions) for lv in keys}, tabs["role"], tabs["iter"])
+    sc = scope._struct() if scope is not None else None
+    rc = lib.argus_aggregate_scoped(_ptr(intervals), _ptr(interval_offsets), _ptr(ambig), _ptr(ambig_offsets), S,
+                                    warps_per_cta, _ptr(cta_sm), num_sms, num_regions,
+                                    ctypes.addressof(sc) if sc is not None else None, _ptr(out.warp), _ptr(out.cta),
+                                    _ptr(out.sm), _ptr(out.kernel), _ptr(out.role), _ptr(out.iter), _ptr(out.status),
+                                    _ptr(out.workspace), out.workspace.numel(), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_aggregate_scoped")
+    return out
+
+
+def argus_overlap_scoped(intervals: torch.Tensor, max_intervals: int, interval_offsets: torch.Tensor, warps_per_cta: int,
+                         cta_sm: torch.Tensor, num_sms: int, pairs: torch.Tensor, scope: ArgusScope | None):
+    """Returns (out uint8 [K * M * 32], status uint8 [64])."""
+    lib = load_library()
+    dev = intervals.device
+    S = interval_offsets.numel() - 1
+    K = pairs.numel() // 2
+    workspace = _bytes(lib.argus_overlap_workspace_bytes(max_intervals, S, K, num_sms), dev)
+    out = _bytes(K * num_sms * 32, dev)
+    status = _bytes(64, dev)
+    sc = scope._struct() if scope is not None else None
+    rc = lib.argus_overlap_scoped(_ptr(intervals), max_intervals, _ptr(interval_offsets), S, warps_per_cta, _ptr(cta_sm),
+                                  num_sms, _ptr(pairs), K, ctypes.addressof(sc) if sc is not None else None, _ptr(out),
+                                  _ptr(status), _ptr(workspace), workspace.numel(), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_overlap_scoped")
     return out, status
 
 

@@ -5,6 +5,10 @@
 //                   itself), integer atomics only, so the result does not depend on thread order.
 //   k_agg_cta     : CTA-scope cells = reduction over the warps of each CTA (plain loads, no atomics).
 //   k_agg_init / k_agg_scatter : SM-scope and kernel-scope cells by atomic add/min/max of CTA cells.
+//   k_agg_role    : warp-role cells = reduction over the CTAs of each warp index (plain loads).
+//   k_agg_iter    : per-iteration cells (key = ctx - ctx_lo) of the intervals of a scope.
+// A scope (iteration window, warp mask, SM mask, region mask) filters what k_agg_streams and
+// k_agg_iter take in; without one everything is selected.
 #include "argus_common.cuh"
 
 namespace {
@@ -26,7 +30,37 @@ struct AggArgs {
   u64* kernel_tab;  // nullable
   argus_status_t* status;
   int use_smem;
+  // scope selection
+  int scoped;
+  u32 ctx_lo, ctx_hi;
+  u64 warp_mask;
+  const u32* sm_mask;
+  const u32* region_mask;
+  u64* role_tab;  // [W][R][72], nullable
+  u64* iter_tab;  // [num_iters][R][72], nullable
+  u32 num_iters;
+  int iter_smem;
 };
+
+__device__ __forceinline__ bool mask_bit(const u32* mask, u32 i) { return !mask || ((mask[i >> 5] >> (i & 31)) & 1u); }
+
+// Warp-role and SM tests of a scope: one answer per stream. 2 = bad cta_sm entry.
+__device__ __forceinline__ int stream_in_scope(const AggArgs& a, u32 s) {
+  if (!a.scoped) return 1;
+  const u32 w = s % a.warps_per_cta;
+  if (a.warp_mask != ~0ull && (w >= 64 || !((a.warp_mask >> w) & 1ull))) return 0;
+  if (a.sm_mask) {
+    const u32 m = a.cta_sm[s / a.warps_per_cta];
+    if (m >= a.num_sms) return 2;
+    if (!mask_bit(a.sm_mask, m)) return 0;
+  }
+  return 1;
+}
+
+// Iteration-window and region tests of a scope: one answer per record.
+__device__ __forceinline__ bool record_in_scope(const AggArgs& a, u32 ctx, u32 region) {
+  return !a.scoped || (ctx >= a.ctx_lo && ctx <= a.ctx_hi && mask_bit(a.region_mask, region));
+}
 
 __device__ __forceinline__ u32 log2_bin(u64 d) { return d ? 63u - (u32)__clzll((long long)d) : 0u; }
 
@@ -52,9 +86,11 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams(AggArgs a) {
     if (!a.use_smem) __threadfence();
     __syncthreads();
     const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
+    const int sel = stream_in_scope(a, s);
+    if (sel == 2 && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, a.cta_sm[s / a.warps_per_cta]);
     if (hi < lo) {
       if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
-    } else {
+    } else if (sel == 1) {
       for (u64 i = lo + threadIdx.x; i < hi; i += blockDim.x) {
         const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
         const uint4 q0 = __ldg(p), q1 = __ldg(p + 1), q2 = __ldg(p + 2);
@@ -62,14 +98,16 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams(AggArgs a) {
         const u64 excl = (u64)q1.x | ((u64)q1.y << 32);
         const u32 region = q1.z;
         if (region >= R) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
+        if (!record_in_scope(a, q1.w, region)) continue;
         agg_add_interval(tab, region, incl, excl, q2.w >> 16);
       }
     }
-    if (a.ambig && a.ambig_offsets) {
+    if (a.ambig && a.ambig_offsets && sel == 1) {
       const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
       for (u64 i = alo + threadIdx.x; i < ahi && ahi >= alo; i += blockDim.x) {
         const u32 region = a.ambig[i].tag >> 1;
         if (region >= R) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
+        if (!record_in_scope(a, a.ambig[i].ctx, region)) continue;
         atomicAdd(tab + (size_t)region * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
       }
     }
@@ -121,6 +159,65 @@ __global__ void __launch_bounds__(256) k_agg_scatter(AggArgs a) {
     }
     if (a.kernel_tab) {
       u64* d = a.kernel_tab + rem;
+      if (field == 2) atomicMin(d, v); else if (field == 3) atomicMax(d, v); else atomicAdd(d, v);
+    }
+  }
+}
+
+// role_tab[w][r][j] = reduce over c of warp_tab[c*W + w][r][j]
+__global__ void __launch_bounds__(256) k_agg_role(AggArgs a) {
+  const u64 per_row = (u64)a.num_regions * kCell;
+  const u64 n = (u64)a.warps_per_cta * per_row;
+  for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (u64)gridDim.x * blockDim.x) {
+    const u64 w = i / per_row, rem = i % per_row;
+    const u32 field = (u32)(rem % kCell);
+    const u64* src = a.warp_tab + w * per_row + rem;
+    u64 acc = src[0];
+    for (u32 c = 1; c < a.num_ctas; ++c) acc = combine(field, acc, src[(u64)c * a.warps_per_cta * per_row]);
+    a.role_tab[i] = acc;
+  }
+}
+
+// iter_tab[ctx - ctx_lo][r]: selected intervals and ambiguity records keyed by iteration. A block gathers its
+// streams in a shared-memory copy of the table when that fits and adds the non-empty cells to the global
+// table (initialised by k_agg_init) at the end; otherwise it updates the global table record by record.
+__global__ void __launch_bounds__(kAggThreads) k_agg_iter(AggArgs a) {
+  extern __shared__ __align__(16) u64 sh_tab[];
+  const u32 R = a.num_regions;
+  const u64 cells = (u64)a.num_iters * R * kCell;
+  u64* tab = a.iter_smem ? sh_tab : a.iter_tab;
+  if (a.iter_smem) {
+    for (u64 i = threadIdx.x; i < cells; i += blockDim.x) sh_tab[i] = (i % kCell == 2) ? ~0ull : 0ull;
+    __syncthreads();
+  }
+  for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
+    if (stream_in_scope(a, s) != 1) continue;  // a bad cta_sm entry is reported by k_agg_streams
+    const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
+    for (u64 i = lo + threadIdx.x; i < hi && hi >= lo; i += blockDim.x) {
+      const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
+      const uint4 q1 = __ldg(p + 1);
+      const u32 region = q1.z, ctx = q1.w;
+      if (region >= R || !record_in_scope(a, ctx, region)) continue;
+      const uint4 q0 = __ldg(p), q2 = __ldg(p + 2);
+      agg_add_interval(tab + (u64)(ctx - a.ctx_lo) * R * kCell, region, (u64)q0.z | ((u64)q0.w << 32),
+                       (u64)q1.x | ((u64)q1.y << 32), q2.w >> 16);
+    }
+    if (a.ambig && a.ambig_offsets) {
+      const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
+      for (u64 i = alo + threadIdx.x; i < ahi && ahi >= alo; i += blockDim.x) {
+        const u32 region = a.ambig[i].tag >> 1, ctx = a.ambig[i].ctx;
+        if (region >= R || !record_in_scope(a, ctx, region)) continue;
+        atomicAdd(tab + ((u64)(ctx - a.ctx_lo) * R + region) * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
+      }
+    }
+  }
+  if (a.iter_smem) {
+    __syncthreads();
+    for (u64 i = threadIdx.x; i < cells; i += blockDim.x) {
+      const u32 field = (u32)(i % kCell);
+      const u64 v = sh_tab[i];
+      if (field == 2 ? v == ~0ull : v == 0ull) continue;
+      u64* d = a.iter_tab + i;
       if (field == 2) atomicMin(d, v); else if (field == 3) atomicMax(d, v); else atomicAdd(d, v);
     }
   }
@@ -181,6 +278,8 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
   a.num_sms = num_sms; a.num_regions = num_regions; a.cta_sm = cta_sm;
   a.warp_tab = (u64*)warp_tab; a.cta_tab = (u64*)cta_work; a.sm_tab = (u64*)sm_tab; a.kernel_tab = (u64*)kernel_tab;
   a.status = status; a.use_smem = 0;
+  a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
+  a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0;
   if (ambig && ambig_offsets) {
     k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
     ARGUS_CHECK_LAUNCH();
@@ -192,26 +291,32 @@ extern "C" size_t argus_aggregate_workspace_bytes(uint64_t /*num_intervals*/, ui
   return agg_layout(num_streams, num_regions).total + 256;
 }
 
-int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
-                             const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                             uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                             argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
-                             argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
-                             bool reset_status) {
+int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                                    const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                                    uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                                    const argus_scope_t* scope, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                                    argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
+                                    argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
+                                    size_t workspace_bytes, void* cuda_stream, bool reset_status) {
   if (!interval_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
-  if (sm_tab && (!cta_sm || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
+  if ((sm_tab || (scope && scope->sm_mask)) && (!cta_sm || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
+  if (scope && scope->ctx_hi < scope->ctx_lo) return ARGUS_ERR_INVALID_ARG;
+  if (iter_tab && (!scope || scope->ctx_hi - scope->ctx_lo >= ARGUS_MAX_ITER_ROWS)) return ARGUS_ERR_INVALID_ARG;
   if (((uintptr_t)intervals & 15) || ((uintptr_t)workspace & 255) || ((uintptr_t)warp_tab & 7) || ((uintptr_t)cta_tab & 7) ||
-      ((uintptr_t)sm_tab & 7) || ((uintptr_t)kernel_tab & 7))
+      ((uintptr_t)sm_tab & 7) || ((uintptr_t)kernel_tab & 7) || ((uintptr_t)role_tab & 7) || ((uintptr_t)iter_tab & 7))
     return ARGUS_ERR_INVALID_ARG;
   const AggLayout L = agg_layout(num_streams, num_regions);
   if (workspace_bytes < L.total) return ARGUS_ERR_WORKSPACE;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
+  const u32 num_iters = iter_tab ? scope->ctx_hi - scope->ctx_lo + 1 : 0;
+  if (kernel_tab) { k_agg_init<<<16, 256, 0, stream>>>((u64*)kernel_tab, (u64)num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
+  if (sm_tab) { k_agg_init<<<296, 256, 0, stream>>>((u64*)sm_tab, (u64)num_sms * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
+  if (iter_tab) { k_agg_init<<<296, 256, 0, stream>>>((u64*)iter_tab, (u64)num_iters * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
   if (num_streams == 0) {
-    if (kernel_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)kernel_tab, (u64)num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
-    if (sm_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)sm_tab, (u64)num_sms * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
+    if (role_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)role_tab, (u64)warps_per_cta * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
     return ARGUS_OK;
   }
   AggArgs a;
@@ -221,15 +326,52 @@ int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* 
   a.warp_tab = warp_tab ? (u64*)warp_tab : (u64*)((char*)workspace + L.warp);
   a.cta_tab = cta_tab ? (u64*)cta_tab : (u64*)((char*)workspace + L.cta);
   a.sm_tab = (u64*)sm_tab; a.kernel_tab = (u64*)kernel_tab; a.status = status;
+  a.scoped = scope != nullptr;
+  a.ctx_lo = scope ? scope->ctx_lo : 0; a.ctx_hi = scope ? scope->ctx_hi : 0xffffffffu;
+  a.warp_mask = scope ? scope->warp_mask : ~0ull;
+  a.sm_mask = scope ? scope->sm_mask : nullptr; a.region_mask = scope ? scope->region_mask : nullptr;
+  a.role_tab = (u64*)role_tab; a.iter_tab = (u64*)iter_tab; a.num_iters = num_iters;
   const size_t smem = (size_t)num_regions * sizeof(argus_agg_t);
   a.use_smem = smem <= kAggSmemLimit;
-  if (a.use_smem && smem > 48 * 1024)
-    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const size_t iter_bytes = (size_t)num_iters * smem;
+  a.iter_smem = iter_tab && iter_bytes <= kAggSmemLimit;
+  const size_t need = a.use_smem ? smem : 0, need_iter = a.iter_smem ? iter_bytes : 0;
+  if (need > 48 * 1024)
+    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need));
+  if (need_iter > 48 * 1024)
+    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_iter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need_iter));
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 0);
-  k_agg_streams<<<num_streams, kAggThreads, a.use_smem ? smem : 0, stream>>>(a);
+  k_agg_streams<<<num_streams, kAggThreads, need, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 1);
-  return agg_rollup(a, cta_tab, sm_tab, kernel_tab, stream);
+  if (iter_tab) {
+    k_agg_iter<<<num_streams < 296 ? num_streams : 296, kAggThreads, need_iter, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  if (role_tab) {
+    k_agg_role<<<296, 256, 0, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  if (cta_tab || sm_tab || kernel_tab) {
+    k_agg_cta<<<1184, 256, 0, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  if (sm_tab || kernel_tab) {
+    k_agg_scatter<<<1184, 256, 0, stream>>>(a);
+    ARGUS_CHECK_LAUNCH();
+  }
+  return ARGUS_OK;
+}
+
+int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                             const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                             uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                             argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
+                             argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                             bool reset_status) {
+  return argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
+                                         num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab, nullptr,
+                                         nullptr, status, workspace, workspace_bytes, cuda_stream, reset_status);
 }
 
 extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
@@ -240,4 +382,16 @@ extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t
   return argus_internal_aggregate(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
                                   num_sms, num_regions, warp_tab, cta_tab, sm_tab, kernel_tab, status, workspace,
                                   workspace_bytes, cuda_stream, true);
+}
+
+extern "C" int argus_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                                      const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                                      uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                                      const argus_scope_t* scope, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                                      argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
+                                      argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream) {
+  return argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
+                                         num_sms, num_regions, scope, warp_tab, cta_tab, sm_tab, kernel_tab, role_tab, iter_tab,
+                                         status, workspace, workspace_bytes, cuda_stream, true);
 }

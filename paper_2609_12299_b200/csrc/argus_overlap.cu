@@ -31,7 +31,15 @@ struct OvArgs {
   u64* cum;           // [capacity] covered length before piece i within its segment
   u64 capacity;
   u32 nseg;
+  // scope selection (argus_overlap_scoped): iteration window, warp mask, SM mask, region mask
+  int scoped;
+  u32 ctx_lo, ctx_hi;
+  u64 warp_mask;
+  const u32* sm_mask;
+  const u32* region_mask;
 };
+
+__device__ __forceinline__ bool ov_mask_bit(const u32* mask, u32 i) { return !mask || ((mask[i >> 5] >> (i & 31)) & 1u); }
 
 __global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatter) {
   // One stream per block iteration: all of its spans belong to one SM, so the block counts per
@@ -49,6 +57,11 @@ __global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatt
       if (threadIdx.x == 0) argus_set_error(a.status, m >= a.num_sms ? ARGUS_ERR_INVALID_ARG : ARGUS_ERR_BAD_OFFSETS, s, m);
       continue;
     }
+    if (a.scoped) {  // warp-role and SM tests: one answer per stream
+      const u32 w = s % a.warps_per_cta;
+      if (a.warp_mask != ~0ull && (w >= 64 || !((a.warp_mask >> w) & 1ull))) continue;
+      if (!ov_mask_bit(a.sm_mask, m)) continue;
+    }
     for (u32 i = threadIdx.x; i < 2 * a.num_pairs; i += blockDim.x) sh_cnt[i] = 0;
     __syncthreads();
     for (int pass = 0; pass < (scatter ? 2 : 1); ++pass) {
@@ -58,6 +71,10 @@ __global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatt
         const u64 incl = (u64)q0.z | ((u64)q0.w << 32);
         if (incl == 0) continue;
         const u32 region = __ldg(reinterpret_cast<const u32*>(p + 1) + 2);
+        if (a.scoped) {  // iteration-window and region tests: one answer per interval
+          const u32 ctx = __ldg(reinterpret_cast<const u32*>(p + 1) + 3);
+          if (ctx < a.ctx_lo || ctx > a.ctx_hi || !ov_mask_bit(a.region_mask, region)) continue;
+        }
         const u64 t0 = (u64)q0.x | ((u64)q0.y << 32);
         for (u32 k = 0; k < 2 * a.num_pairs; ++k) {
           if (sh_pairs[k] != region) continue;
@@ -362,6 +379,7 @@ static int ov_setup(OvArgs& a, uint32_t num_streams, uint32_t warps_per_cta, con
   a.spans = (ulonglong2*)(ws + L.spans);
   a.cum = (u64*)(ws + L.spans + argus_align_up((size_t)a.capacity * 16, 16));
   a.nseg = nseg;
+  a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
   ARGUS_CUDA_TRY(cudaMemsetAsync(ws, 0, L.seg_base, stream));
   ARGUS_CUDA_TRY(cudaMemsetAsync(out, 0, (size_t)num_pairs * num_sms * sizeof(argus_overlap_t), stream));
   return ARGUS_OK;
@@ -381,11 +399,13 @@ int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* lis
   return ov_run(a, &l, stream);
 }
 
-int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
-                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
-                           const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
-                           void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status) {
+static int overlap_scoped(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                          uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                          const uint32_t* pairs, uint32_t num_pairs, const argus_scope_t* scope, argus_overlap_t* out,
+                          argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                          bool reset_status) {
   if (!interval_offsets || !cta_sm || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
+  if (scope && scope->ctx_hi < scope->ctx_lo) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0 || num_sms == 0) return ARGUS_ERR_INVALID_ARG;
   if (num_pairs > kMaxPairs || (num_pairs && (!pairs || !out))) return ARGUS_ERR_INVALID_ARG;
   if ((max_intervals && !intervals) || ((uintptr_t)intervals & 15) || ((uintptr_t)workspace & 255) || ((uintptr_t)out & 7))
@@ -399,7 +419,28 @@ int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_inter
                           workspace_bytes, stream);
   if (rc != ARGUS_OK) return rc;
   a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets;
+  if (scope) {
+    a.scoped = 1; a.ctx_lo = scope->ctx_lo; a.ctx_hi = scope->ctx_hi; a.warp_mask = scope->warp_mask;
+    a.sm_mask = scope->sm_mask; a.region_mask = scope->region_mask;
+  }
   return ov_run(a, nullptr, stream);
+}
+
+int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                           const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status) {
+  return overlap_scoped(intervals, max_intervals, interval_offsets, num_streams, warps_per_cta, cta_sm, num_sms, pairs,
+                        num_pairs, nullptr, out, status, workspace, workspace_bytes, cuda_stream, reset_status);
+}
+
+extern "C" int argus_overlap_scoped(const argus_interval_t* intervals, uint64_t max_intervals,
+                                    const uint64_t* interval_offsets, uint32_t num_streams, uint32_t warps_per_cta,
+                                    const uint32_t* cta_sm, uint32_t num_sms, const uint32_t* pairs, uint32_t num_pairs,
+                                    const argus_scope_t* scope, argus_overlap_t* out, argus_status_t* status,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return overlap_scoped(intervals, max_intervals, interval_offsets, num_streams, warps_per_cta, cta_sm, num_sms, pairs,
+                        num_pairs, scope, out, status, workspace, workspace_bytes, cuda_stream, true);
 }
 
 extern "C" int argus_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,

@@ -141,3 +141,40 @@ def test_malformed_full_size_sampled():
     assert amb > 0
     del res
     torch.cuda.empty_cache()
+
+
+def test_decode_full_size_scoped_aggregate():
+    """Scope selection at the bench size: 16 of the 256 iterations, three warp roles, on the 614 M intervals
+    the path produced; sampled CTAs against the oracle, size-independent properties on the whole tables."""
+    spec = tg.config(3)
+    res, st, n, offs = _run_full(spec)
+    W, R, M = spec.warps_per_cta, spec.num_regions, spec.num_sms
+    lo, hi, warps = 100, 115, [0, 1, 5]
+    scope = argus.ArgusScope(ctx_lo=lo, ctx_hi=hi, warp_mask=sum(1 << w for w in warps))
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    sc = argus.argus_aggregate_scoped(res.pair.intervals, res.pair.interval_offsets, res.pair.ambig, res.pair.ambig_offsets,
+                                      W, cta_sm, M, R, scope, levels=("warp", "cta", "sm", "kernel", "role", "iter"))
+    assert int(argus.argus_status_fetch(sc.status)["code"]) == 0
+    ker, role, it = sc.table_numpy("kernel"), sc.table_numpy("role"), sc.table_numpy("iter")
+    warp = sc.table_numpy("warp")
+    assert it.shape == (16, R) and role.shape == (W, R)
+    for f in ("count", "sum_incl", "sum_excl", "n_flagged", "hist"):
+        for tab in (warp, role, it, sc.table_numpy("cta"), sc.table_numpy("sm")):
+            assert np.array_equal(tab[f].sum(0, dtype=np.uint64), ker[f][0]), f
+    assert not role["count"][[w for w in range(W) if w not in warps]].any()
+    # every stream runs the same program: 16 iterations x 1013 intervals in each selected stream
+    assert np.array_equal(warp["count"].sum(1), np.where(np.isin(np.arange(spec.num_streams) % W, warps), 16 * 1013, 0))
+    assert np.all(it["count"].sum(1) == 1013 * len(warps) * spec.num_ctas)
+    for c in (0, 91):
+        s0, s1 = c * W, (c + 1) * W
+        ev = tg.host_streams(spec, offs, s0, s1)
+        sub = (offs[s0:s1 + 1] - offs[s0]).astype(np.uint64)
+        rc, o_iv, o_ioffs, o_am, o_aoffs, _ = oracle.pair(ev, sub, R)
+        assert rc == 0
+        rc, want, _ = oracle.aggregate_scoped(o_iv, o_ioffs, o_am, o_aoffs, W, np.zeros(1, np.uint32), 1, R,
+                                              scope={"ctx": (lo, hi), "warps": warps}, levels=("warp", "cta"))
+        assert rc == 0
+        assert warp[s0:s1].tobytes() == want["warp"].tobytes(), f"warp rows of CTA {c} differ"
+        assert sc.table_numpy("cta")[c:c + 1].tobytes() == want["cta"].tobytes(), f"CTA row {c} differs"
+    del res, sc
+    torch.cuda.empty_cache()
