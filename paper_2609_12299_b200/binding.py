@@ -101,6 +101,12 @@ def argus_set_tile_variant(v: int) -> None:
     lib.argus_set_tile_variant(int(v))
 
 
+def argus_set_synthesize_mode(mode: int) -> None:
+    """Where argus_synthesize aggregates: -1 automatic, 0 in the pairing kernel, 1 in one pass over the
+    intervals, 2 the plain calls (tuning and test aid; results are identical)."""
+    load_library().argus_set_synthesize_mode(int(mode))
+
+
 def argus_launch_count() -> int:
     return int(load_library().argus_launch_count())
 

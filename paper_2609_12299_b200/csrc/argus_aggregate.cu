@@ -1,21 +1,24 @@
 // argus_aggregate.cu — argus_aggregate: intervals (+ ambiguity records) -> per-(scope, region) tables.
 //
-//   k_agg_streams : one CTA per stream accumulates that stream's row of the warp-scope table
-//                   (a shared-memory private copy when num_regions * 576 B fits, else the global row
-//                   itself), integer atomics only, so the result does not depend on thread order.
+//   k_agg_streams_compact : one CTA per stream accumulates that stream's row of the warp-scope table in
+//                   the compact shared-memory form the fused pairing kernel uses (112 B per region, so
+//                   several CTAs fit an SM), for up to kAggCompactRegions regions;
+//   k_agg_streams : the same with a full 576 B-per-region copy in shared memory when that fits, else on
+//                   the global row itself. Integer atomics only: the result does not depend on thread order.
 //   k_agg_cta     : CTA-scope cells = reduction over the warps of each CTA (plain loads, no atomics).
 //   k_agg_init / k_agg_scatter : SM-scope and kernel-scope cells by atomic add/min/max of CTA cells.
 //   k_agg_role    : warp-role cells = reduction over the CTAs of each warp index (plain loads).
 //   k_agg_iter    : per-iteration cells (key = ctx - ctx_lo) of the intervals of a scope.
 // A scope (iteration window, warp mask, SM mask, region mask) filters what k_agg_streams and
 // k_agg_iter take in; without one everything is selected.
-#include "argus_common.cuh"
+#include "argus_fuse.cuh"
 
 namespace {
 
 constexpr int kAggThreads = 256;
 constexpr u32 kCell = 72;  // u64 words per argus_agg_t
 constexpr size_t kAggSmemLimit = 200 * 1024;
+constexpr u32 kAggCompactRegions = 400;  // 112 B each: 44.8 KB of shared memory at most
 
 struct AggArgs {
   const argus_interval_t* intervals;
@@ -40,7 +43,11 @@ struct AggArgs {
   u64* iter_tab;  // [num_iters][R][72], nullable
   u32 num_iters;
   int iter_smem;
+  // overlap span selection in the same pass over the intervals (argus_synthesize); ov.ov_spans null = off
+  ArgusFuseArgs ov;
 };
+
+constexpr u32 kAggOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
 
 __device__ __forceinline__ bool mask_bit(const u32* mask, u32 i) { return !mask || ((mask[i >> 5] >> (i & 31)) & 1u); }
 
@@ -116,6 +123,107 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams(AggArgs a) {
       for (u32 i = threadIdx.x; i < cells; i += blockDim.x) row[i] = sh_tab[i];
       __syncthreads();
     }
+  }
+}
+
+__global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) {
+  extern __shared__ __align__(16) unsigned char sh_raw[];
+  ArgusAggCell* const ctab = reinterpret_cast<ArgusAggCell*>(sh_raw);
+  const u32 R = a.num_regions;
+  const u32 cells = R * kCell;
+  const u32 lane = threadIdx.x & 31;
+  // overlap selection: bitmap of the regions that appear in a pair, and the pair list, after the table
+  u32* const pairbits = reinterpret_cast<u32*>(ctab + R);
+  u32* const pairs_sm = pairbits + (R + 31) / 32;
+  const bool has_ov = a.ov.ov_spans != nullptr && a.ov.num_pairs != 0;
+  u64 ovc_base = 0;             // warp-uniform: current chunk of the global span list
+  u32 ovc_used = kAggOvChunk;
+  if (has_ov) {
+    for (u32 i = threadIdx.x; i < (R + 31) / 32; i += blockDim.x) pairbits[i] = 0;
+    __syncthreads();
+    for (u32 i = threadIdx.x; i < 2 * a.ov.num_pairs; i += blockDim.x) {
+      const u32 r = a.ov.pairs[i];
+      pairs_sm[i] = r;
+      if (r < R) atomicOr(&pairbits[r >> 5], 1u << (r & 31));
+    }
+    __syncthreads();
+  }
+  for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
+    u64* row = a.warp_tab + (size_t)s * cells;
+    // the global row takes flag counts' overflow path, bins outside the window and the ambiguity counters directly
+    for (u32 i = threadIdx.x; i < cells; i += blockDim.x) row[i] = (i % kCell == 2) ? ~0ull : 0ull;
+    argus_fuse_init(ctab, R, threadIdx.x, blockDim.x);
+    __threadfence();
+    __syncthreads();
+    ArgusFuseCtx fx;
+    fx.tab = ctab; fx.pairbits = nullptr; fx.row = row; fx.sm_index = 0;
+    const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
+    const int sel = stream_in_scope(a, s);
+    if (sel == 2 && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, a.cta_sm[s / a.warps_per_cta]);
+    u32 sm_index = 0;
+    if (has_ov) {
+      const u32 m = a.cta_sm[s / a.warps_per_cta];
+      if (m >= a.num_sms && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
+      sm_index = m < a.num_sms ? m : 0;
+    }
+    if (hi < lo) {
+      if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
+    } else if (sel == 1) {
+      // every lane of a warp runs the same number of rounds, so that spans can be appended a warp at a time
+      for (u64 base = lo + (threadIdx.x & ~31u); base < hi; base += blockDim.x) {
+        const u64 i = base + lane;
+        bool cand = false;
+        u32 region = 0;
+        u64 t0 = 0, incl = 0;
+        if (i < hi) {
+          const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
+          const uint4 q0 = __ldg(p), q1 = __ldg(p + 1), q2 = __ldg(p + 2);
+          region = q1.z;
+          if (region >= R) {
+            argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i);
+          } else if (record_in_scope(a, q1.w, region)) {
+            t0 = (u64)q0.x | ((u64)q0.y << 32);
+            incl = (u64)q0.z | ((u64)q0.w << 32);
+            argus_fuse_aggregate(fx, region, incl, (u64)q1.x | ((u64)q1.y << 32), q2.w >> 16);
+            cand = has_ov && incl && ((pairbits[region >> 5] >> (region & 31)) & 1u);
+          }
+        }
+        if (has_ov && __ballot_sync(0xffffffffu, cand)) {
+          for (u32 k = 0; k < 2 * a.ov.num_pairs; ++k) {
+            const bool pick = cand && pairs_sm[k] == region;
+            const u32 bal = __ballot_sync(0xffffffffu, pick);
+            if (!bal) continue;
+            const u32 c = __popc(bal);
+            if (ovc_used + c > kAggOvChunk) {
+              u64 nb64 = 0;
+              if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)kAggOvChunk);
+              ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
+              ovc_used = 0;
+            }
+            if (pick) {
+              const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
+              if (slot < a.ov.ov_capacity) {
+                a.ov.ov_spans[slot] = make_ulonglong2(t0, t0 + incl);
+                a.ov.ov_seg[slot] = ((k >> 1) * a.num_sms + sm_index) * 2 + (k & 1u);
+              }
+            }
+            ovc_used += c;
+          }
+        }
+      }
+    }
+    if (a.ambig && a.ambig_offsets && sel == 1) {
+      const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
+      for (u64 i = alo + threadIdx.x; i < ahi && ahi >= alo; i += blockDim.x) {
+        const u32 region = a.ambig[i].tag >> 1;
+        if (region >= R) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
+        if (!record_in_scope(a, a.ambig[i].ctx, region)) continue;
+        atomicAdd(row + (size_t)region * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
+      }
+    }
+    __syncthreads();
+    argus_fuse_flush(ctab, row, R, threadIdx.x, blockDim.x);
+    __syncthreads();
   }
 }
 
@@ -280,6 +388,7 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
   a.status = status; a.use_smem = 0;
   a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
   a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0;
+  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0;
   if (ambig && ambig_offsets) {
     k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
     ARGUS_CHECK_LAUNCH();
@@ -297,8 +406,10 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
                                     const argus_scope_t* scope, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
                                     argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
                                     argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
-                                    size_t workspace_bytes, void* cuda_stream, bool reset_status) {
+                                    size_t workspace_bytes, void* cuda_stream, bool reset_status,
+                                    const ArgusFuseArgs* ov_select) {
   if (!interval_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
+  if (ov_select && (num_regions > kAggCompactRegions || ov_select->num_pairs > kFuseMaxPairs)) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
   if ((sm_tab || (scope && scope->sm_mask)) && (!cta_sm || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
@@ -331,6 +442,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   a.warp_mask = scope ? scope->warp_mask : ~0ull;
   a.sm_mask = scope ? scope->sm_mask : nullptr; a.region_mask = scope ? scope->region_mask : nullptr;
   a.role_tab = (u64*)role_tab; a.iter_tab = (u64*)iter_tab; a.num_iters = num_iters;
+  if (ov_select) { a.ov = *ov_select; } else { a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; }
   const size_t smem = (size_t)num_regions * sizeof(argus_agg_t);
   a.use_smem = smem <= kAggSmemLimit;
   const size_t iter_bytes = (size_t)num_iters * smem;
@@ -341,7 +453,14 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   if (need_iter > 48 * 1024)
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_iter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need_iter));
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 0);
-  k_agg_streams<<<num_streams, kAggThreads, need, stream>>>(a);
+  if (num_regions <= kAggCompactRegions) {
+    const size_t compact = (size_t)num_regions * sizeof(ArgusAggCell) + ((num_regions + 31) / 32) * 4 + (size_t)a.ov.num_pairs * 8;
+    if (compact > 48 * 1024)
+      ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams_compact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compact));
+    k_agg_streams_compact<<<num_streams, kAggThreads, compact, stream>>>(a);
+  } else {
+    k_agg_streams<<<num_streams, kAggThreads, need, stream>>>(a);
+  }
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 1);
   if (iter_tab) {
@@ -371,7 +490,11 @@ int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* 
                              bool reset_status) {
   return argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
                                          num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab, nullptr,
-                                         nullptr, status, workspace, workspace_bytes, cuda_stream, reset_status);
+                                         nullptr, status, workspace, workspace_bytes, cuda_stream, reset_status, nullptr);
+}
+
+bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs) {
+  return num_regions <= kAggCompactRegions && num_pairs <= kFuseMaxPairs;
 }
 
 extern "C" int argus_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
@@ -393,5 +516,5 @@ extern "C" int argus_aggregate_scoped(const argus_interval_t* intervals, const u
                                       size_t workspace_bytes, void* cuda_stream) {
   return argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
                                          num_sms, num_regions, scope, warp_tab, cta_tab, sm_tab, kernel_tab, role_tab, iter_tab,
-                                         status, workspace, workspace_bytes, cuda_stream, true);
+                                         status, workspace, workspace_bytes, cuda_stream, true, nullptr);
 }

@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   // (pointers into shared memory stay plain locals derived from the shared array, so that the compiler keeps
   // their address space; a generic pointer would turn every table access into a generic load or atomic)
   ArgusAggCell* const tabp = reinterpret_cast<ArgusAggCell*>(smem_raw + ((sizeof(SM) + 15) & ~(size_t)15));
-  u32* const pairbitsp = reinterpret_cast<u32*>(tabp + (FUSE ? a.num_regions : 0u));
+  u32* const pairbitsp = reinterpret_cast<u32*>(tabp + (FUSE && a.fuse.warp_tab ? a.num_regions : 0u));  // no table, no room for it
   u32* const pairs_sm = pairbitsp + (a.num_regions + 31) / 32;  // copy of the (producer, consumer) list: [2 K]
   const bool has_tab = FUSE && !a.redo && a.fuse.warp_tab != nullptr;
   const bool has_pairs = FUSE && !a.redo && a.fuse.ov_spans != nullptr && a.fuse.num_pairs != 0;
@@ -565,7 +565,7 @@ int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   static int grid_cache = 0;
   static size_t smem_cache = 0;
   size_t smem = ((sizeof(TileSmem<NT, E>) + 15) & ~(size_t)15) + 128;
-  if (FUSE) smem += (size_t)a.num_regions * sizeof(ArgusAggCell) + ((a.num_regions + 31) / 32) * 4 + (size_t)a.fuse.num_pairs * 8 + 16;
+  if (FUSE) smem += (a.fuse.warp_tab ? (size_t)a.num_regions * sizeof(ArgusAggCell) : 0) + ((a.num_regions + 31) / 32) * 4 + (size_t)a.fuse.num_pairs * 8 + 16;
   if (!grid_cache || smem_cache != smem) {
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int dev = 0, sms = 0, per_sm = 0;

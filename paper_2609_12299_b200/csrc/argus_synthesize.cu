@@ -1,9 +1,11 @@
 // argus_synthesize.cu — the whole hot path in one call: pair -> aggregate -> overlap.
 //
-// When the tiled pairing kernel can host the aggregation table (num_regions <= 256) the intervals
-// are aggregated and the overlap spans selected while they are still in registers, so the interval
-// array is written once and never read back. Otherwise this is the three plain calls in sequence.
-// Results are identical either way.
+// Pairing runs plain, then ONE pass over the intervals both aggregates them and selects the overlap spans;
+// that pass runs at HBM speed, while hosting the table in the pairing kernel (which is bound by instruction
+// issue and occupancy, not by HBM) measured slower on every trace shape. The pairing kernel's own hooks
+// (aggregate and select while the interval is in registers: the interval array is never read back) remain
+// for calls that ask for overlap without tables and as a tuning choice (argus_set_synthesize_mode). More than 400
+// regions or 128 pairs: the three plain calls. Results are identical in every mode.
 #include "argus_fuse.cuh"
 
 int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
@@ -29,10 +31,21 @@ int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_inter
 int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* list_seg, const uint64_t* list_count,
                                      uint64_t list_capacity, uint32_t num_sms, uint32_t num_pairs, argus_overlap_t* out,
                                      argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                                    const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                                    uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                                    const argus_scope_t* scope, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                                    argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
+                                    argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
+                                    size_t workspace_bytes, void* cuda_stream, bool reset_status,
+                                    const ArgusFuseArgs* ov_select);
+bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs);
 bool argus_pair_tiled_can_fuse(uint32_t num_regions);
 bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs);
 
 namespace {
+
+int g_synth_mode = -1;  // -1 = automatic
 
 struct SynLayout {
   size_t pair, pair_bytes, agg, agg_bytes, list_count, list_seg, list_spans, ov, ov_bytes, total;
@@ -55,6 +68,10 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
 }
 
 }  // namespace
+
+// Where argus_synthesize aggregates and selects overlap spans: -1 automatic, 0 inside the pairing kernel,
+// 1 in one pass over the intervals, 2 the plain calls (tuning and test aid; results are identical).
+extern "C" void argus_set_synthesize_mode(int mode) { g_synth_mode = mode; }
 
 extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint32_t num_regions,
                                                    uint64_t ambig_capacity, uint32_t num_pairs, uint32_t num_sms,
@@ -87,12 +104,21 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
   ArgusFuseArgs f;
   f.warp_tab = nullptr; f.cta_sm = cta_sm; f.warps_per_cta = warps_per_cta; f.num_sms = num_sms;
   f.pairs = pairs; f.num_pairs = num_pairs; f.ov_spans = nullptr; f.ov_seg = nullptr; f.ov_capacity = 0; f.ov_count = nullptr;
-  const bool can_fuse = num_streams > 0 && argus_pair_tiled_can_fuse(num_regions);
-  if (can_fuse && want_agg) {
+  // where aggregation and overlap selection happen: 0 = in the pairing kernel, 1 = in one pass over the
+  // intervals after plain pairing, 2 = the plain calls
+  const bool can_fuse = num_streams > 0 && argus_pair_tiled_can_fuse(num_regions) && argus_pair_tiled_can_fuse_overlap(num_pairs);
+  int mode = 2;
+  if (num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs)) mode = 1;
+  else if (can_fuse) mode = 0;
+  if (g_synth_mode == 0 && can_fuse) mode = 0;  // tuning aid: a forced mode applies when the inputs allow it
+  if (g_synth_mode == 1 && num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs)) mode = 1;
+  if (g_synth_mode == 2) mode = 2;
+  const bool list = mode != 2 && num_pairs;
+  if (mode == 0 && want_agg) {
     f.warp_tab = (u64*)warp_work;
     ARGUS_CUDA_TRY(cudaMemsetAsync(warp_work, 0, (size_t)num_streams * row_bytes, stream));
   }
-  if (can_fuse && num_pairs && argus_pair_tiled_can_fuse_overlap(num_pairs)) {
+  if (list) {
     f.ov_spans = (ulonglong2*)(ws + L.list_spans);
     f.ov_seg = (u32*)(ws + L.list_seg);
     f.ov_capacity = max_overlap_spans;
@@ -103,22 +129,24 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
   bool fused = false;
   int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
                                interval_offsets, ambig, ambig_capacity, ambig_offsets, status, ws + L.pair, L.pair_bytes,
-                               cuda_stream, 0, (f.warp_tab || f.ov_spans) ? &f : nullptr, true, &fused);
+                               cuda_stream, 0, mode == 0 && (f.warp_tab || f.ov_spans) ? &f : nullptr, true, &fused);
   if (rc != ARGUS_OK) return rc;
+  if (mode == 0 && !fused) mode = 2;  // the pairing front end chose a kernel without the hooks
 
   if (want_agg) {
-    if (fused && f.warp_tab) {
+    if (mode == 0) {
       rc = argus_internal_agg_finish(ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm, num_sms, num_regions, warp_work,
                                      cta_work, cta_tab != nullptr, sm_tab, kernel_tab, status, cuda_stream);
     } else {
-      rc = argus_internal_aggregate(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
-                                    num_sms, num_regions, warp_tab, cta_tab, sm_tab, kernel_tab, status, ws + L.agg,
-                                    L.agg_bytes, cuda_stream, false);
+      rc = argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta,
+                                           cta_sm, num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab,
+                                           nullptr, nullptr, status, ws + L.agg, L.agg_bytes, cuda_stream, false,
+                                           mode == 1 && list ? &f : nullptr);
     }
     if (rc != ARGUS_OK) return rc;
   }
   if (num_pairs) {
-    if (fused && f.ov_spans) {
+    if (mode != 2) {
       rc = argus_internal_overlap_from_list(f.ov_spans, f.ov_seg, (const uint64_t*)f.ov_count, f.ov_capacity, num_sms, num_pairs, overlap_out,
                                             status, ws + L.ov, L.ov_bytes, cuda_stream);
     } else {

@@ -276,9 +276,18 @@ def _synthesize_matches(spec, ev, offs, **kw):
     return res, st
 
 
+@pytest.fixture(params=[-1, 0, 1, 2], ids=["auto", "in-pairing-kernel", "one-pass", "plain-calls"])
+def synth_mode(request):
+    """Where argus_synthesize aggregates and selects overlap spans; results must not depend on it."""
+    from paper_2609_12299_b200.binding import argus_set_synthesize_mode
+    argus_set_synthesize_mode(request.param)
+    yield request.param
+    argus_set_synthesize_mode(-1)
+
+
 @pytest.mark.parametrize("idx,ctas,iters", [(0, 4, 626), (1, 7, 300), (2, 3, 3), (3, 3, 9), (4, 9, 400)])
-def test_synthesize_fused_matches_oracle(idx, ctas, iters):
-    """One-call pipeline (aggregation and overlap selection fused into the pairing kernel)."""
+def test_synthesize_fused_matches_oracle(idx, ctas, iters, synth_mode):
+    """One-call pipeline in each of its modes."""
     spec = tg.config(idx).scaled(ctas, iters)
     ev, offs = tg.generate_host(spec)
     res, st = _synthesize_matches(spec, ev, offs)
@@ -286,7 +295,7 @@ def test_synthesize_fused_matches_oracle(idx, ctas, iters):
         assert int(st["n_sequential_tiles"]) == 0
 
 
-def test_synthesize_wide_histogram_and_flags():
+def test_synthesize_wide_histogram_and_flags(synth_mode):
     """Durations spread over many log2 bins (outside the 16-bin shared-memory window), flagged intervals,
     min/max extremes and a region that never occurs."""
     rng = np.random.default_rng(21)
@@ -312,9 +321,11 @@ def test_synthesize_wide_histogram_and_flags():
     _synthesize_matches(spec, np.concatenate(evs), np.array(offs, np.uint64))
 
 
-def test_synthesize_many_regions_falls_back_to_plain_calls():
+@pytest.mark.parametrize("R", [300, 500])
+def test_synthesize_many_regions(R):
+    """300 regions: more than the pairing kernel's table holds (one pass over the intervals instead);
+    500: more than the compact aggregation table holds (the plain calls)."""
     rng = np.random.default_rng(5)
-    R = 300  # more than the fused table holds
     spec = tg.TraceSpec(tg.TINY, 2, 1)
     evs, offs = [], [0]
     for s in range(spec.num_streams):
@@ -325,7 +336,7 @@ def test_synthesize_many_regions_falls_back_to_plain_calls():
 
     class Spec:  # same fields _synthesize_matches reads
         num_regions, warps_per_cta, cta_sm, num_sms = R, 4, spec.cta_sm, spec.num_sms
-        overlap_pairs = np.array([(1, 2), (7, 299)], np.uint32)
+        overlap_pairs = np.array([(1, 2), (7, R - 1)], np.uint32)
     _synthesize_matches(Spec, ev, offs)
 
 
