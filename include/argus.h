@@ -356,10 +356,10 @@ int argus_overlap_scoped(const argus_interval_t* intervals /*device*/, uint64_t 
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *
  * Arguments have the meaning they have in argus_pair_intervals, argus_aggregate and
- * argus_overlap. When num_regions <= 256 the pairing kernel aggregates every interval and
- * selects the overlap spans while the interval is still in registers, so the interval array
- * is written once and never read back; otherwise the three operations run one after the
- * other. Any of the four tables may be NULL; num_pairs may be 0. max_overlap_spans bounds
+ * argus_overlap. Pairing is followed by one pass over the intervals that both aggregates
+ * them and selects the overlap spans (up to 400 regions and 128 pairs; beyond that the three
+ * operations run one after the other). Any of the four tables may be NULL; without tables
+ * the pairing kernel selects the overlap spans itself. num_pairs may be 0. max_overlap_spans bounds
  * the spans selected for overlap over all pairs (an interval counts once per pair and role
  * its region appears in); more than that -> ARGUS_ERR_CAPACITY with the count in
  * status->intervals_required. One status block reports the first error of any stage.
