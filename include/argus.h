@@ -203,7 +203,7 @@ int argus_pair_intervals_ex(const argus_event_t* events /*device*/, uint64_t num
  * the allocator because an allocation could synchronise the device or fail late. This entry
  * point needs no workspace argument: its scratch (control block, per-stream counters, event
  * bitmap and its prefix tables, ambiguity notes) lives in a fixed array inside the library's
- * device image, about 0.9 MB per GPU that loads the library, held until the process exits.
+ * device image, about 1 MB per GPU that loads the library, held until the process exits.
  * Inputs and outputs are still the caller's buffers. The call makes no cudaMalloc, cudaFree
  * or other allocating call.
  *

@@ -176,8 +176,9 @@ __global__ void __launch_bounds__(256) k_ambig_offsets(AmbigArgs g) {
 }
 
 struct Layout {
-  size_t ctl, counts, bits, word_prefix, block_prefix, notes, total;
-  u64 num_words, num_blocks;
+  size_t ctl, counts, queue, bits, word_prefix, block_prefix, notes, records, total;
+  u64 num_words, num_blocks, queue_capacity;
+  u32 record_capacity;
 };
 
 Layout make_layout(uint64_t num_events, uint32_t num_streams, uint64_t ambig_capacity) {
@@ -187,10 +188,15 @@ Layout make_layout(uint64_t num_events, uint32_t num_streams, uint64_t ambig_cap
   size_t o = 0;
   L.ctl = o; o += argus_align_up(sizeof(ArgusPairCtl), 256);
   L.counts = o; o += argus_align_up(((size_t)num_streams + 1) * 8, 256);
+  // every hand-over follows a chunk of at least kChunkEvents events, and only streams longer than that hand over
+  L.queue_capacity = num_events / kChunkEvents + 1;
+  L.record_capacity = (u32)(L.queue_capacity < num_streams ? L.queue_capacity : num_streams);
+  L.queue = o; o += argus_align_up((size_t)L.queue_capacity * 4, 256);
   L.bits = o; o += argus_align_up((size_t)L.num_words * 4 + 4, 256);
   L.word_prefix = o; o += argus_align_up((size_t)L.num_words * 4 + 4, 256);
   L.block_prefix = o; o += argus_align_up(((size_t)L.num_blocks + 1) * 8, 256);
   L.notes = o; o += argus_align_up((size_t)ambig_capacity * 8 + 8, 256);
+  L.records = o; o += argus_align_up((size_t)L.record_capacity * sizeof(ArgusStreamRecord), 256);
   L.total = o;
   return L;
 }
@@ -238,6 +244,8 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   a.ctl = (ArgusPairCtl*)(ws + L.ctl);
   a.status = status;
   a.redo = 0;
+  a.queue = (u32*)(ws + L.queue); a.queue_capacity = L.queue_capacity;
+  a.records = (ArgusStreamRecord*)(ws + L.records); a.record_capacity = L.record_capacity;
   memset(&a.fuse, 0, sizeof(a.fuse));
 
   if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));

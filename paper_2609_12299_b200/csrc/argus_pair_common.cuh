@@ -28,9 +28,30 @@ struct ArgusPairCtl {  // control block in the workspace, zeroed at the start of
   u32 spec_overflow;   // a provisional position fell outside interval_capacity
   u64 total_intervals;
   u64 total_ambig;
-  u64 ticket;          // dynamic work counter of the tiled kernel
-  u64 ticket2;         // same, second (redo) pass
+  // work queue of the tiled kernel, one set per pass (0 = first, 1 = redo): positions below num_streams are the
+  // streams themselves, later positions are streams handed on after a chunk (see ArgusStreamRecord)
+  u64 q_head[2];       // positions taken
+  u64 q_tail[2];       // hand-overs published (queue entries written)
+  u32 n_records[2];    // hand-over records allocated
+  u32 n_done[2];       // streams walked to their end (or given up on)
   u64 reserved[2];
+};
+
+// A long stream is walked in chunks of about kChunkEvents events. After a chunk the CTA stores the stream's
+// state here and puts the record into the work queue, so that whichever CTA is free next carries on: all
+// streams advance at the same pace and the kernel has no long tail, whatever the number of streams per SM.
+// Queue positions are taken with one atomic add each. A CTA whose position has no entry yet is idle anyway
+// (every unfinished stream is in some CTA's hands): it polls until the entry appears or every stream is
+// done, and gives up with ARGUS_ERR_TIMEOUT if no hand-over at all is published for about a second.
+constexpr u32 kChunkEvents = 32768;
+struct ArgusStreamRecord {
+  u32 stream, next_tile;
+  int ch;                             // stack height at the hand-over
+  u32 pad;
+  u64 n_int;                          // intervals emitted so far
+  uint4 frames[ARGUS_MAX_DEPTH];      // open begin markers as event records
+  u64 child[ARGUS_MAX_DEPTH];         // their child time so far
+  u32 idx[ARGUS_MAX_DEPTH];           // their index within the stream
 };
 
 struct ArgusPairArgs {
@@ -49,6 +70,10 @@ struct ArgusPairArgs {
   ArgusPairCtl* ctl;
   argus_status_t* status;
   int redo;               // 0 = first pass with provisional bases, 1 = second pass with final bases
+  u32* queue;             // hand-over queue entries (record index + 1; zeroed), null = streams are never split
+  u64 queue_capacity;
+  ArgusStreamRecord* records;
+  u32 record_capacity;
   ArgusFuseArgs fuse;     // optional aggregation / overlap selection fed from the pairing kernel (first pass only)
 };
 

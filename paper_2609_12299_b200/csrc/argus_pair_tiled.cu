@@ -65,6 +65,40 @@ constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 
 constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
 constexpr int kBadRef = 0x3fff;   // reference that marks a window as not well nested
 constexpr int kSeqChunk = 128;    // markers handed to the sequential machine at once when cuts come densely
+constexpr u32 kNoRec = 0xffffffffu;
+
+// Takes the next piece of work of pass `p`: a stream nobody has started (position below num_streams) or a
+// hand-over from the queue. Returns false when every stream is done (or on a timeout). One thread per CTA.
+__device__ __forceinline__ bool tile_pop_work(const ArgusPairArgs& a, int p, u64* stream, u32* rec) {
+  const u64 h = atomicAdd(reinterpret_cast<unsigned long long*>(&a.ctl->q_head[p]), 1ull);
+  if (h < a.num_streams) { *stream = h; *rec = kNoRec; return true; }
+  const u64 slot = h - a.num_streams;
+  if (!a.queue || slot >= a.queue_capacity) return false;  // more positions than hand-overs can ever be published
+  volatile u32* q = a.queue + slot;
+  volatile u32* done = &a.ctl->n_done[p];
+  volatile u64* tail = &a.ctl->q_tail[p];
+  u64 seen = *tail;
+  u32 idle = 0, nap = 64;
+  for (;;) {
+    const u32 v = *q;
+    if (v) {
+      *q = 0;  // the second pass uses the same entries
+      __threadfence();
+      *rec = v - 1;
+      *stream = *reinterpret_cast<volatile u32*>(&a.records[v - 1].stream);
+      return true;
+    }
+    if (*done >= a.num_streams) return false;
+    const u64 t = *tail;
+    if (t != seen) { seen = t; idle = 0; }
+    if (++idle > (1u << 19)) {  // ~1 s without any hand-over anywhere
+      argus_set_error(a.status, ARGUS_ERR_TIMEOUT, 0, slot);
+      return false;
+    }
+    __nanosleep(nap);
+    if (nap < 2048) nap *= 2;
+  }
+}
 
 // Shared memory of one CTA. Events of the two tile buffers and the frames carried from earlier tiles
 // share one index space, so that "the frame an end closes" and "its parent" are plain indices:
@@ -81,14 +115,17 @@ struct TileSmem {
   uint4 evall[2 * T + 2 * kCar];
   u64 accall[T + 4 * kCar];        // child time per frame, same index space shifted by 2 kCar
   u32 desc[MAXI];                  // per end, in end order: event index | level << 16
-  u32 bm[kLevelWindow][NWORDS];    // per level: bit e set = event e of the tile is a begin at that level
+  union {
+    u32 bm[kLevelWindow][NWORDS];    // per level: bit e set = event e of the tile is a begin at that level
+    ArgusFrame fstk[ARGUS_MAX_DEPTH];  // stack in the layout the sequential path uses (no bitmap is live while it runs)
+  };
   u64 summ[kLevelWindow];          // per level: bit w set = bm[level][w] != 0
   u32 cidx[2][ARGUS_MAX_DEPTH];    // begin index (within the stream) of each carried frame
   u64 cchild[2][ARGUS_MAX_DEPTH];  // child time of each carried frame as the window found it
-  ArgusFrame fstk[ARGUS_MAX_DEPTH];  // stack in the layout the sequential redo path uses
   u32 warp_tot[32];
   u64 bar[2];
   u64 cur_stream;
+  u32 cur_rec;                     // hand-over record of the stream being walked (kNoRec: none)
   u64 n_int;                       // written by the sequential redo path
   int ch;
   int badpos;                      // first position of the window where the parallel rules fail (INT_MAX = none)
@@ -165,16 +202,24 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
 #endif
 
   for (;;) {
-    if (tid == 0) sm.cur_stream = atomicAdd(a.redo ? &a.ctl->ticket2 : &a.ctl->ticket, 1ull);
+    if (tid == 0) {
+      u64 st = ~0ull;
+      u32 rc = kNoRec;
+      if (!tile_pop_work(a, a.redo ? 1 : 0, &st, &rc)) st = ~0ull;
+      sm.cur_stream = st;
+      sm.cur_rec = rc;
+    }
     __syncthreads();
     const u64 s64 = sm.cur_stream;
     if (s64 >= a.num_streams) break;
     const u32 s = (u32)s64;
+    u32 rec = sm.cur_rec;
     const u64 lo = a.stream_offsets[s], hi = a.stream_offsets[s + 1];
     if (hi < lo || hi > a.num_events || lo < off0 || ((hi - lo) >> 32)) {
       if (tid == 0) {
         argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
         if (!a.redo) a.counts[s] = 0;
+        atomicAdd(&a.ctl->n_done[a.redo ? 1 : 0], 1u);
       }
       __syncthreads();
       continue;
@@ -187,6 +232,32 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     int ch = 0;          // carried stack height (uniform)
     u64 n_int = 0;       // intervals of this stream so far (uniform)
     bool stream_failed = false;
+    // Long streams are walked a chunk at a time (never when the aggregation table lives in this kernel: it
+    // belongs to the stream). A resumed stream takes its state from the record; a new one reserves a record.
+    u32 ti0 = 0;
+    constexpr u32 kChunkTiles = (kChunkEvents + T - 1) / T;
+    bool chunked = !FUSE && a.queue != nullptr && ntiles > kChunkTiles;
+    if (rec != kNoRec) {
+      const ArgusStreamRecord* r = a.records + rec;
+      ti0 = __ldcg(&r->next_tile);
+      ch = __ldcg(&r->ch);
+      n_int = __ldcg(&r->n_int);
+      if (tid < ch) {  // the carried block 0 is where the first window looks
+        sm.evall[T + tid] = __ldcg(&r->frames[tid]);
+        sm.cchild[0][tid] = __ldcg(&r->child[tid]);
+        sm.cidx[0][tid] = __ldcg(&r->idx[tid]);
+      }
+    } else if (chunked) {
+      __syncthreads();  // everyone has read sm.cur_rec
+      if (tid == 0) {
+        const u32 r = atomicAdd(&a.ctl->n_records[a.redo ? 1 : 0], 1u);
+        sm.cur_rec = r < a.record_capacity ? r : kNoRec;
+      }
+      __syncthreads();
+      rec = sm.cur_rec;
+      if (rec == kNoRec) chunked = false;  // cannot happen (one record per long stream); then the stream is walked whole
+    }
+    const u32 ti_end = chunked && ti0 + kChunkTiles < ntiles ? ti0 + kChunkTiles : ntiles;
     if (FUSE && !a.redo) {
       if (has_tab) {
         argus_fuse_init(tabp, a.num_regions, tid, NT);
@@ -201,14 +272,15 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       }
       __syncthreads();
     }
-    if (tid == 0 && ntiles > 0) {
-      const u32 bytes = (n < (u32)T ? n : (u32)T) * 16u;
-      mbar_expect_tx(&sm.bar[0], bytes);
-      tma_load_1d(sm.evall, src, bytes, &sm.bar[0]);
+    if (tid == 0 && ti0 < ti_end) {  // first tile of this chunk, into the buffer its index selects
+      const u32 start = ti0 * (u32)T;
+      const u32 bytes = ((n - start) < (u32)T ? (n - start) : (u32)T) * 16u;
+      mbar_expect_tx(&sm.bar[ti0 & 1], bytes);
+      tma_load_1d((ti0 & 1) ? sm.evall + T + 2 * kCar : sm.evall, src + start, bytes, &sm.bar[ti0 & 1]);
     }
 
     int cpar = 0;        // which carried-frame block holds the current stack
-    for (u32 ti = 0; ti < ntiles; ++ti) {
+    for (u32 ti = ti0; ti < ti_end; ++ti) {
       const int b = ti & 1;
       const u32 tile_start = ti * (u32)T;
       const int tn = (int)((n - tile_start) < (u32)T ? (n - tile_start) : (u32)T);
@@ -217,7 +289,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       const uint4* evb = b ? ev1 : ev0;                  // evb[ref] for every reference of this tile
       u64* accb = sm.accall + 2 * kCar;                  // accb[ref], ref in [-2 kCar, T + 2 kCar)
       const int carlo = b ? -2 * kCar : T;               // reference of slot 0 of carried block 0, seen from this buffer
-      if (tid == 0 && ti + 1 < ntiles) {  // prefetch the next tile into the other buffer
+      if (tid == 0 && ti + 1 < ti_end) {  // prefetch the next tile into the other buffer
         const u32 nstart = tile_start + T;
         const u32 bytes = ((n - nstart) < (u32)T ? (n - nstart) : (u32)T) * 16u;
         mbar_expect_tx(&sm.bar[b ^ 1], bytes);
@@ -516,7 +588,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         }
       }  // windows
       if (stream_failed) {
-        if (ti + 1 < ntiles) {  // drain the prefetched tile before the buffer is reused
+        if (ti + 1 < ti_end) {  // drain the prefetched tile before the buffer is reused
           const bool ok = mbar_wait_bounded(&sm.bar[b ^ 1], (b ^ 1) ? ph1 : ph0);
           if (b ^ 1) ph1 ^= 1; else ph0 ^= 1;
           if (!ok) sm.dead = 1;
@@ -531,10 +603,28 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, 0);
       return;
     }
-    if (!a.redo) {
-      // frames still open at the end of the stream (they sit in the block the next tile would read)
-      if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[cpar][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
-      if (tid == 0) a.counts[s] = n_int;
+    if (!stream_failed && ti_end < ntiles) {
+      // hand the stream on: its state goes into the record, the record into the queue
+      ArgusStreamRecord* r = a.records + rec;
+      if (tid == 0) { r->stream = s; r->next_tile = ti_end; r->ch = ch; r->n_int = n_int; }
+      if (tid < ch) {
+        r->frames[tid] = sm.evall[T + cpar * kCar + tid];
+        r->child[tid] = sm.cchild[cpar][tid];
+        r->idx[tid] = sm.cidx[cpar][tid];
+      }
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) {
+        const u64 slot = atomicAdd(reinterpret_cast<unsigned long long*>(&a.ctl->q_tail[a.redo ? 1 : 0]), 1ull);
+        if (slot < a.queue_capacity) *reinterpret_cast<volatile u32*>(a.queue + slot) = rec + 1;
+      }
+    } else {
+      if (!a.redo) {
+        // frames still open at the end of the stream (they sit in the block the next tile would read)
+        if (!stream_failed && tid < ch) argus_note_ambiguity(a, gpos0 + sm.cidx[cpar][tid], ARGUS_AMBIG_BEGIN_EOS, (u32)tid);
+        if (tid == 0) a.counts[s] = n_int;
+      }
+      if (tid == 0) atomicAdd(&a.ctl->n_done[a.redo ? 1 : 0], 1u);
     }
     if (has_tab) {
       if (hot0 != 0xffffffffu) argus_fuse_agg_sums(tabp[hot0], hsi0, hse0);
@@ -628,10 +718,16 @@ int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
     case 13: return launch_tiled_any<512, 3, 1>(a, stream);
     case 14: return launch_tiled_any<224, 7, 2>(a, stream);
     case 15: return launch_tiled_any<256, 5, 3>(a, stream);
+    case 16: return launch_tiled_any<160, 5, 5>(a, stream);
+    case 17: return launch_tiled_any<96, 5, 8>(a, stream);
+    case 18: return launch_tiled_any<128, 5, 6>(a, stream);
     default: {
-      // automatic: four CTAs of 192 threads per SM, unless the fused aggregation table is large enough
-      // to cost a CTA slot; then two CTAs of 320 threads (streams per CTA stay balanced either way)
-      const bool big_table = !a.redo && a.fuse.warp_tab && (size_t)a.num_regions * sizeof(ArgusAggCell) > 6 * 1024;
+      // automatic. Plain pairing: six CTAs of 128 threads per SM (with streams walked in chunks the number of
+      // streams per SM does not have to divide evenly). With the aggregation table inside the kernel: four CTAs
+      // of 192 threads, or two of 320 when the table is large enough to cost CTA slots.
+      const bool hooks = !a.redo && (a.fuse.warp_tab || a.fuse.ov_spans);
+      if (!hooks) return launch_tiled_any<128, 5, 6>(a, stream);
+      const bool big_table = a.fuse.warp_tab && (size_t)a.num_regions * sizeof(ArgusAggCell) > 6 * 1024;
       return big_table ? launch_tiled_any<320, 5, 2>(a, stream) : launch_tiled_any<192, 5, 4>(a, stream);
     }
   }

@@ -15,9 +15,9 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
 
 namespace {
 
-// Enough for the pairing pipeline at the documented maxima (control block, per-stream counters,
-// one bit per event plus its prefix tables, 8-byte ambiguity notes): a little under 0.9 MB.
-constexpr size_t kStaticScratchBytes = 896 * 1024;
+// Enough for the pairing pipeline at the documented maxima (control block, per-stream counters, work queue
+// and hand-over records, one bit per event plus its prefix tables, 8-byte ambiguity notes): 0.92 MB.
+constexpr size_t kStaticScratchBytes = 960 * 1024;
 static __device__ __align__(256) unsigned char g_pair_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
