@@ -387,3 +387,32 @@ def test_single_long_stream_and_many_empty_streams():
     offs = np.cumsum([0] + [len(e) for e in evs]).astype(np.uint64)
     for kernel in KERNELS:
         assert_pair_matches(np.concatenate(evs), offs, 5, kernel)
+
+
+def test_long_streams_walked_in_chunks():
+    """Streams several chunks long (the tiled kernel hands a stream from CTA to CTA every 32 K events, with the
+    open frames and their child time in a record): deep stacks carried across hand-overs, defects, a stream
+    shorter than a chunk beside them, and more CTAs than streams (idle CTAs wait for hand-overs)."""
+    rng = np.random.default_rng(35)
+    evs = [random_wellformed(rng, 150_000, 6, max_height=40), random_wellformed(rng, 5_000, 6, max_height=3),
+           random_wellformed(rng, 70_000, 6, max_height=12)]
+    # defects in the third stream: dropped ends and duplicated begins
+    ev = evs[2]
+    keep = np.ones(len(ev), bool)
+    ends = np.nonzero(ev["tag"] & 1)[0]
+    keep[rng.choice(ends, 40, replace=False)] = False
+    ev = ev[keep]
+    dup = np.sort(rng.choice(np.nonzero((ev["tag"] & 1) == 0)[0], 25, replace=False))
+    evs[2] = np.insert(ev, dup, ev[dup])
+    offs = np.cumsum([0] + [len(e) for e in evs]).astype(np.uint64)
+    pr, _ = assert_pair_matches(np.concatenate(evs), offs, 6, KERNEL_TILED)
+    assert int(pr.last_status["ambig_required"]) > 0
+
+
+@pytest.mark.parametrize("idx,ctas,iters", [(3, 1, 40), (4, 2, 3000)])
+def test_synthesize_long_streams(idx, ctas, iters):
+    """The one-call pipeline on streams of 80 K to 110 K events (several hand-overs each), bit for bit."""
+    spec = tg.config(idx).scaled(ctas, iters)
+    ev, offs = tg.generate_host(spec)
+    assert np.diff(offs).max() > 70_000
+    _synthesize_matches(spec, ev, offs)
