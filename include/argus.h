@@ -352,6 +352,46 @@ int argus_overlap_scoped(const argus_interval_t* intervals /*device*/, uint64_t 
                          void* workspace /*device*/, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------
+ * PC-to-region attribution — Section 3.2 (the figure on dynamic PC-to-region mapping: each
+ * execution of the instruction at PC p is credited to the innermost region active in its
+ * warp at that moment) and Section 3.5 "Ambiguity-aware attribution" (the weights alpha,
+ * the lifted metric and the association entropy).
+ *
+ * Mapping-run traces reuse the marker record. Regions keep ids 0 .. R-1. "The instruction
+ * at PC index p executed k times here" is written as a begin/end pair of the extra region
+ * id R (exec_region) placed at that point of the stream:
+ *     { ts = 0, tag = R << 1,       ctx = p }     { ts = k, tag = (R << 1) | 1, ctx = p }
+ * so that argus_pair_intervals (called with num_regions = R + 1) turns it into an interval
+ * with region R, ctx p, inclusive k and parent_region = the innermost active region, under
+ * exactly the stack rules of pairing, mis-nested and unmatched markers included. (Times of
+ * real regions are meaningless in such a trace; only the counts are used.)
+ *
+ * argus_map_pc_counts: counts[r][p] (u64, [(R + 1)][P], row R = outside every region) =
+ * sum of inclusive over the intervals with region exec_region, ctx p and parent_region r
+ * (parent NONE or >= R goes to row R). Every cell is written. Intervals of exec_region
+ * whose ctx >= num_pcs set status->code = ARGUS_ERR_INVALID_ARG.
+ *
+ * argus_attribute (fp64): with N_p = sum_r counts[r][p], alpha[r][p] = counts[r][p] / N_p
+ * (0 where N_p = 0), mhat[r] = sum_p alpha[r][p] * metric[p], entropy[p] = - sum over
+ * r with alpha > 0 of alpha * ln(alpha). alpha may be NULL. The sums over p are taken in a
+ * fixed order (block partial sums, then their sum), so results repeat from run to run; they
+ * agree with a sequential sum to rounding (relative 1e-12 of sum_p |alpha * metric|).
+ * ------------------------------------------------------------------------------------- */
+int argus_map_pc_counts(const argus_interval_t* intervals /*device*/,
+                        const uint64_t* interval_offsets /*device [S+1]*/, uint32_t num_streams,
+                        uint32_t exec_region /* = R */, uint32_t num_pcs,
+                        uint64_t* counts /*device [(R+1)][P]*/, argus_status_t* status /*device*/,
+                        void* cuda_stream);
+
+size_t argus_attribute_workspace_bytes(uint32_t num_rows, uint32_t num_pcs);
+
+int argus_attribute(const uint64_t* counts /*device [rows][P]*/, uint32_t num_rows,
+                    uint32_t num_pcs, const double* metric /*device [P]*/,
+                    double* mhat /*device [rows]*/, double* entropy /*device [P]*/,
+                    double* alpha /*device [rows][P], nullable*/, void* workspace /*device*/,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
  * argus_synthesize — the three operations above in one call, with identical results
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *

@@ -56,8 +56,10 @@ def _load():
         lib.oracle_overlap.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp]
         lib.oracle_aggregate_scoped.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_overlap_scoped.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp]
+        lib.oracle_map_pc_counts.argtypes = [vp, vp, u32, u32, u32, vp, vp]
+        lib.oracle_attribute.argtypes = [vp, u32, u32, vp, vp, vp, vp]
         for f in (lib.oracle_pair, lib.oracle_aggregate, lib.oracle_overlap, lib.oracle_aggregate_scoped,
-                  lib.oracle_overlap_scoped):
+                  lib.oracle_overlap_scoped, lib.oracle_map_pc_counts, lib.oracle_attribute):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -192,3 +194,28 @@ def overlap_scoped(intervals, interval_offsets, warps_per_cta, cta_sm, num_sms, 
                                        None if sc is None else ctypes.addressof(sc), _ptr(out), _ptr(st))
     del keep
     return rc, out, st[0]
+
+
+MAP_EVENT = np.dtype([("kind", "<u4"), ("id", "<u4"), ("count", "<u8")])  # kind 0 begin, 1 end, 2 exec
+assert MAP_EVENT.itemsize == 16
+
+
+def map_pc_counts(map_events, stream_offsets, num_regions, num_pcs):
+    """Returns (rc, counts [(R + 1), P] uint64, status); row R = outside every region."""
+    ev = np.ascontiguousarray(map_events, dtype=MAP_EVENT)
+    offs = np.ascontiguousarray(stream_offsets, dtype=np.uint64)
+    counts = np.zeros((num_regions + 1, num_pcs), dtype=np.uint64)
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_map_pc_counts(_ptr(ev), _ptr(offs), len(offs) - 1, num_regions, num_pcs, _ptr(counts), _ptr(st))
+    return rc, counts, st[0]
+
+
+def attribute(counts, metric, want_alpha=True):
+    """Returns (rc, mhat [rows], entropy [P], alpha [rows, P] or None), all float64."""
+    n = np.ascontiguousarray(counts, dtype=np.uint64)
+    rows, P = n.shape
+    m = np.ascontiguousarray(metric, dtype=np.float64)
+    mhat, ent = np.zeros(rows, np.float64), np.zeros(P, np.float64)
+    alpha = np.zeros((rows, P), np.float64) if want_alpha else None
+    rc = _load().oracle_attribute(_ptr(n), rows, P, _ptr(m), _ptr(mhat), _ptr(ent), _ptr(alpha))
+    return rc, mhat, ent, alpha

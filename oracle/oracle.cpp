@@ -6,6 +6,7 @@
 #include "oracle.h"
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <map>
 #include <tuple>
@@ -384,6 +385,60 @@ extern "C" int oracle_overlap_scoped(const OInterval* intervals, const uint64_t*
       o.overlap_ns = both;
       o.either_ns = o.producer_ns + o.consumer_ns - both;
     }
+  }
+  return OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// PC-to-region mapping (Section 3.2) and ambiguity-aware attribution (Section 3.5).
+// ---------------------------------------------------------------------------------------------
+extern "C" int oracle_map_pc_counts(const OMapEvent* events, const uint64_t* stream_offsets, uint32_t num_streams,
+                                    uint32_t num_regions, uint32_t num_pcs, uint64_t* counts, OStatus* st) {
+  if (!stream_offsets || !counts || !st || num_regions == 0 || num_pcs == 0) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  std::memset(counts, 0, sizeof(uint64_t) * (static_cast<size_t>(num_regions) + 1) * num_pcs);
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    std::vector<uint32_t> stack;  // region ids of the open frames, innermost last
+    for (uint64_t i = stream_offsets[s]; i < stream_offsets[s + 1]; ++i) {
+      const OMapEvent& e = events[i];
+      if (e.kind == 2) {  // exec: the innermost active region receives the execution count
+        if (e.id >= num_pcs) return ERR_INVALID;
+        if (stack.size() == kMaxDepth) { fail(st, ERR_DEPTH, s, i - stream_offsets[s]); return OK; }
+        const uint32_t owner = stack.empty() ? num_regions : stack.back();
+        counts[static_cast<size_t>(owner) * num_pcs + e.id] += e.count;
+      } else if (e.kind == 0) {
+        if (e.id >= num_regions) { fail(st, ERR_BAD_REGION, s, i - stream_offsets[s]); return OK; }
+        if (stack.size() == kMaxDepth) { fail(st, ERR_DEPTH, s, i - stream_offsets[s]); return OK; }
+        stack.push_back(e.id);
+      } else {
+        if (e.id >= num_regions) { fail(st, ERR_BAD_REGION, s, i - stream_offsets[s]); return OK; }
+        size_t k = stack.size();
+        while (k > 0 && stack[k - 1] != e.id) --k;   // innermost open frame of this region
+        if (k > 0) stack.resize(k - 1);              // it closes, and so does everything above it
+      }
+    }
+  }
+  return OK;
+}
+
+extern "C" int oracle_attribute(const uint64_t* counts, uint32_t num_rows, uint32_t num_pcs, const double* metric,
+                                double* mhat, double* entropy, double* alpha) {
+  if (!counts || !metric || !mhat || !entropy || num_rows == 0 || num_pcs == 0) return ERR_INVALID;
+  for (uint32_t r = 0; r < num_rows; ++r) mhat[r] = 0.0;
+  for (uint32_t p = 0; p < num_pcs; ++p) {
+    uint64_t total = 0;
+    for (uint32_t r = 0; r < num_rows; ++r) total += counts[static_cast<size_t>(r) * num_pcs + p];
+    double h = 0.0;
+    for (uint32_t r = 0; r < num_rows; ++r) {
+      const uint64_t n = counts[static_cast<size_t>(r) * num_pcs + p];
+      const double a = (total == 0 || n == 0) ? 0.0 : static_cast<double>(n) / static_cast<double>(total);
+      if (alpha) alpha[static_cast<size_t>(r) * num_pcs + p] = a;
+      if (a > 0.0) {
+        mhat[r] += a * metric[p];
+        h -= a * std::log(a);
+      }
+    }
+    entropy[p] = h;
   }
   return OK;
 }

@@ -80,6 +80,22 @@ int oracle_aggregate_scoped(const OInterval* intervals, const uint64_t* interval
                             uint32_t num_regions, const OScope* scope, OAgg* warp_tab, OAgg* cta_tab,
                             OAgg* sm_tab, OAgg* kernel_tab, OAgg* role_tab, OAgg* iter_tab, OStatus* st);
 
+// PC-to-region mapping (paper Section 3.2, the dynamic PC-to-region mapping figure): a mapping-run stream is a
+// sequence of begin(region), end(region) and exec(pc, k) records; every exec credits k executions of that PC
+// to the innermost region active at that point of the stream (row num_regions = outside every region). The
+// stack follows the rules of oracle_pair (an end closes the innermost open frame of its region and drops the
+// frames above it; an end without such a frame changes nothing; at most 64 open frames, an exec record
+// counting as one more). counts is [(num_regions + 1)][num_pcs].
+struct OMapEvent { uint32_t kind; uint32_t id; uint64_t count; };  // kind 0 begin, 1 end, 2 exec
+int oracle_map_pc_counts(const OMapEvent* events, const uint64_t* stream_offsets, uint32_t num_streams,
+                         uint32_t num_regions, uint32_t num_pcs, uint64_t* counts, OStatus* st);
+
+// Ambiguity-aware attribution (paper Section 3.5): alpha[r][p] = n[r][p] / sum_r' n[r'][p],
+// mhat[r] = sum_p alpha[r][p] * metric[p], entropy[p] = - sum_{alpha > 0} alpha ln alpha. fp64, plain loops.
+// alpha may be null.
+int oracle_attribute(const uint64_t* counts, uint32_t num_rows, uint32_t num_pcs, const double* metric,
+                     double* mhat, double* entropy, double* alpha);
+
 // oracle_overlap over the selected intervals only.
 int oracle_overlap_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,

@@ -10,7 +10,8 @@ from .binding import (AGG_DTYPE, AMBIG_DTYPE, EVENT_DTYPE, INTERVAL_DTYPE, OVERL
                       argus_launch_count, argus_profile_enable, argus_profile_read, argus_status_fetch, argus_strerror,
                       argus_version, library_path, load_library, pair_aggregate_host, argus_synthesize,
                       argus_synthesize_workspace_bytes, SynthesizeResult, argus_pair_intervals_static, ArgusScope,
-                      ScopedAggregateResult, argus_aggregate_scoped, argus_overlap_scoped)
+                      ScopedAggregateResult, argus_aggregate_scoped, argus_overlap_scoped, encode_map_events,
+                      argus_map_pc_counts, argus_attribute)
 
 __all__ = [
     "AGG_DTYPE", "AMBIG_DTYPE", "EVENT_DTYPE", "INTERVAL_DTYPE", "OVERLAP_DTYPE", "STATUS_DTYPE", "ArgusError",
@@ -19,5 +20,5 @@ __all__ = [
     "argus_strerror", "argus_version", "library_path", "load_library", "pair_aggregate_host", "argus_launch_count",
     "argus_profile_enable", "argus_profile_read", "argus_synthesize", "argus_synthesize_workspace_bytes",
     "SynthesizeResult", "argus_pair_intervals_static", "ArgusScope", "ScopedAggregateResult", "argus_aggregate_scoped",
-    "argus_overlap_scoped",
+    "argus_overlap_scoped", "encode_map_events", "argus_map_pc_counts", "argus_attribute",
 ]

@@ -70,6 +70,12 @@ def load_library():
     lib.argus_aggregate_scoped.restype = ci
     lib.argus_overlap_scoped.argtypes = [vp, u64, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp, vp, sz, vp]
     lib.argus_overlap_scoped.restype = ci
+    lib.argus_map_pc_counts.argtypes = [vp, vp, u32, u32, u32, vp, vp, vp]
+    lib.argus_map_pc_counts.restype = ci
+    lib.argus_attribute_workspace_bytes.argtypes = [u32, u32]
+    lib.argus_attribute_workspace_bytes.restype = sz
+    lib.argus_attribute.argtypes = [vp, u32, u32, vp, vp, vp, vp, vp, sz, vp]
+    lib.argus_attribute.restype = ci
     lib.argus_status_fetch.argtypes = [vp, vp, vp]
     lib.argus_status_fetch.restype = ci
     lib.argus_strerror.argtypes = [ci]
@@ -374,6 +380,56 @@ def argus_overlap_scoped(intervals: torch.Tensor, max_intervals: int, interval_o
     if rc != 0:
         raise ArgusError(rc, "argus_overlap_scoped")
     return out, status
+
+
+def encode_map_events(kind: np.ndarray, ident: np.ndarray, count: np.ndarray, exec_region: int) -> np.ndarray:
+    """Mapping-run records (kind 0 begin / 1 end of region `ident`, 2 = PC index `ident` executed `count`
+    times) in the marker encoding argus.h documents: an exec record becomes a begin/end pair of region
+    `exec_region` with ctx = PC index and ts 0 / count. Returns (events, source index of each event).
+    Argument marshalling only."""
+    kind = np.asarray(kind)
+    is_exec = kind == 2
+    reps = np.where(is_exec, 2, 1)
+    src = np.repeat(np.arange(len(kind)), reps)
+    second = np.zeros(len(src), dtype=bool)
+    second[np.cumsum(reps)[is_exec] - 1] = True           # the end half of every exec pair
+    ev = np.zeros(len(src), dtype=EVENT_DTYPE)
+    ex = is_exec[src]
+    ev["tag"] = np.where(ex, (exec_region << 1) | second, (np.asarray(ident)[src] << 1) | (kind[src] & 1)).astype(np.uint32)
+    ev["ctx"] = np.where(ex, np.asarray(ident)[src], 0).astype(np.uint32)
+    ev["ts"] = np.where(second, np.asarray(count)[src], 0).astype(np.uint64)
+    return ev, src
+
+
+def argus_map_pc_counts(intervals: torch.Tensor, interval_offsets: torch.Tensor, exec_region: int, num_pcs: int):
+    """Returns (counts int64 tensor [(exec_region + 1), num_pcs] (bit pattern of u64), status uint8 [64])."""
+    lib = load_library()
+    dev = intervals.device
+    S = interval_offsets.numel() - 1
+    counts = torch.empty((exec_region + 1, num_pcs), dtype=torch.int64, device=dev)
+    status = _bytes(64, dev)
+    rc = lib.argus_map_pc_counts(_ptr(intervals), _ptr(interval_offsets), S, exec_region, num_pcs, _ptr(counts),
+                                 _ptr(status), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_map_pc_counts")
+    return counts, status
+
+
+def argus_attribute(counts: torch.Tensor, metric: torch.Tensor, want_alpha: bool = True):
+    """counts: int64 [rows, P] (u64 bit pattern); metric: float64 [P]. Returns (mhat [rows], entropy [P],
+    alpha [rows, P] or None), float64 device tensors."""
+    lib = load_library()
+    dev = counts.device
+    rows, P = counts.shape
+    mhat = torch.empty(rows, dtype=torch.float64, device=dev)
+    entropy = torch.empty(P, dtype=torch.float64, device=dev)
+    alpha = torch.empty((rows, P), dtype=torch.float64, device=dev) if want_alpha else None
+    ws = _bytes(lib.argus_attribute_workspace_bytes(rows, P), dev)
+    rc = lib.argus_attribute(_ptr(counts), rows, P, _ptr(metric), _ptr(mhat), _ptr(entropy), _ptr(alpha), _ptr(ws),
+                             ws.numel(), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_attribute")
+    return mhat, entropy, alpha
 
 
 @dataclass
