@@ -85,3 +85,32 @@ def test_pc_index_out_of_range_is_reported():
     pr = argus.argus_pair_intervals(d_ev, d_off, 2)
     counts, status = argus.argus_map_pc_counts(pr.intervals, pr.interval_offsets, 1, 4)
     assert int(argus.argus_status_fetch(status)["code"]) == 1
+
+
+def test_decode_shaped_mapping_run():
+    """The synthetic mapping run used for measurements (decode-megakernel markers with exec records after every
+    begin, 203 region ids, 70,560 PCs, eight helper PCs shared by all regions): counts bit for bit, attribution
+    to rounding, and shared PCs do come out ambiguous."""
+    from paper_2609_12299_b200 import tracegen as tg
+    from paper_2609_12299_b200.tracegen.mapping import decode_mapping_trace, mapping_trace
+    spec = tg.config(3).scaled(num_ctas=2, iters=6)
+    R, P = spec.num_regions, 70_560
+    d_ev, d_off = tg.generate_cuda(spec, DEV)
+    m_ev, m_off = mapping_trace(d_ev, d_off, R, P, execs_per_begin=2)
+    pr = argus.argus_pair_intervals(m_ev, m_off, R + 1)
+    assert int(pr.fetch_status()["code"]) == 0
+    counts, status = argus.argus_map_pc_counts(pr.intervals, pr.interval_offsets, R, P)
+    assert int(argus.argus_status_fetch(status)["code"]) == 0
+    host = m_ev.cpu().numpy().view(argus.EVENT_DTYPE)
+    offs = m_off.cpu().numpy().astype(np.int64)
+    kind, ident, count, removed_before = decode_mapping_trace(host, R)
+    a_offs = (offs - np.concatenate([[0], removed_before])[offs]).astype(np.uint64)
+    abstract = np.zeros(len(kind), dtype=oracle.MAP_EVENT)
+    abstract["kind"], abstract["id"], abstract["count"] = kind, ident, count
+    rc, want, st = oracle.map_pc_counts(abstract, a_offs, R, P)
+    assert rc == 0 and int(st["code"]) == 0
+    assert np.array_equal(counts.cpu().numpy().view(np.uint64), want)
+    metric = np.random.default_rng(2).gamma(2.0, 50.0, size=P)
+    check_attribution(counts, want, metric)
+    _, _, ent, _ = oracle.attribute(want, metric)
+    assert np.all(ent[-8:] > 0.1) and np.count_nonzero(ent[:-8]) == 0
