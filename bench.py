@@ -164,10 +164,12 @@ def main():
     ap.add_argument("--three-calls", action="store_true",
                     help="time argus_pair_intervals + argus_aggregate + argus_overlap instead of the one-call argus_synthesize")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-combine", action="store_true",
+                    help="N > 1: do not combine the ranks' kernel-scope tables at the end of every step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    from paper_2609_12299_b200.multirank import max_over_ranks, rank_env, rank_spec, whole_job_rate
+    from paper_2609_12299_b200.multirank import combine_kernel_tables, max_over_ranks, rank_env, rank_spec, whole_job_rate
     rank, world, local_rank = rank_env()
 
     from paper_2609_12299_b200 import tracegen as tg
@@ -225,7 +227,13 @@ def main():
                                                   max_overlap_spans=mos, out=state["syn"])
         state["pair"], state["agg"], state["ov"] = r.pair, r.agg, (r.overlap, r.status)
 
-    step = step_three_calls if args.three_calls else step_one_call
+    local_step = step_three_calls if args.three_calls else step_one_call
+    combine = world > 1 and not args.no_combine
+
+    def step():
+        local_step()
+        if combine:  # the path's one exchange step: R x 576 bytes, all-reduced (sum / min / max)
+            combine_kernel_tables(state["agg"].kernel, world)
 
     def barrier():
         if world > 1:
@@ -363,7 +371,8 @@ def main():
             "config": {"workload": spec.name, "events_per_gpu": n_events, "streams": S, "regions": spec.num_regions,
                        "input_bytes_per_gpu": n_events * 16, "l2": "inputs (>= 1 GB) are larger than the 126 MB L2",
                        "step": ("argus_pair_intervals + argus_aggregate + argus_overlap" if args.three_calls else
-                                "argus_synthesize (pair + aggregate + overlap in one call)") + " on one trace per GPU"},
+                                "argus_synthesize (pair + aggregate + overlap in one call)") + " on one trace per GPU",
+                       "exchange": "kernel-scope tables of all ranks combined by all-reduce every step" if combine else "none"},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline, "kernel_ms": kernel_ms,
         }
