@@ -392,6 +392,39 @@ int argus_attribute(const uint64_t* counts /*device [rows][P]*/, uint32_t num_ro
                     size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Cross-run join with distribution statistics — Section 3.3 (a probe measurement is joined
+ * back to the reference trace through its stable region / operation id and its dynamic
+ * scope), Section 3.5 "Qualified synthesis" (a probe of iteration i is matched to the same
+ * operation of reference iteration i, never by comparing timestamps of different runs) and
+ * the appendix on the asynchronous-timeline trace (mean and 0th / 20th / 40th / 60th / 80th
+ * percentile of the repeated samples of every operation).
+ *
+ * Query q names one interval of the reference run, ref_index[q] (an index into `reference`).
+ * Its key is (stream, region, ctx). Every interval of `samples` (the intervals of any number
+ * of probe runs, in any order) with the same key is a sample of it; its value is the sample's
+ * inclusive time. out[q] = number of samples, their sum (mean = sum / count), minimum ... :
+ * pct[j] = sorted_values[(j * count) / 5] for j = 0..4 (0th = minimum, 80th close to the
+ * maximum), all zero when there is no sample. Reference intervals that share a key share
+ * their samples. At most ARGUS_JOIN_MAX_SAMPLES samples per query are ranked; a query with
+ * more sets status->code = ARGUS_ERR_CAPACITY (count and sum are still exact).
+ * Cost is num_queries passes over `samples`: meant for the selected operations of a query
+ * (tens to thousands), not for joining whole traces.
+ * ------------------------------------------------------------------------------------- */
+#define ARGUS_JOIN_MAX_SAMPLES 4096u
+
+typedef struct {
+  uint64_t count, sum;   /* samples joined, sum of their inclusive times                  */
+  uint64_t pct[5];       /* 0th, 20th, 40th, 60th, 80th percentile                        */
+  uint64_t max;          /* largest sample                                                */
+} argus_join_t;          /* 64 bytes */
+
+int argus_join_samples(const argus_interval_t* reference /*device*/, uint64_t num_reference,
+                       const uint64_t* ref_index /*device [Q]*/, uint32_t num_queries,
+                       const argus_interval_t* samples /*device*/, uint64_t num_samples,
+                       argus_join_t* out /*device [Q]*/, argus_status_t* status /*device*/,
+                       void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
  * argus_synthesize — the three operations above in one call, with identical results
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *

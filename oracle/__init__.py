@@ -56,6 +56,8 @@ def _load():
         lib.oracle_overlap.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp]
         lib.oracle_aggregate_scoped.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_overlap_scoped.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp]
+        lib.oracle_join_samples.argtypes = [vp, u64, vp, u32, vp, u64, vp, vp]
+        lib.oracle_join_samples.restype = ctypes.c_int
         lib.oracle_map_pc_counts.argtypes = [vp, vp, u32, u32, u32, vp, vp]
         lib.oracle_attribute.argtypes = [vp, u32, u32, vp, vp, vp, vp]
         for f in (lib.oracle_pair, lib.oracle_aggregate, lib.oracle_overlap, lib.oracle_aggregate_scoped,
@@ -219,3 +221,18 @@ def attribute(counts, metric, want_alpha=True):
     alpha = np.zeros((rows, P), np.float64) if want_alpha else None
     rc = _load().oracle_attribute(_ptr(n), rows, P, _ptr(m), _ptr(mhat), _ptr(ent), _ptr(alpha))
     return rc, mhat, ent, alpha
+
+
+JOIN = np.dtype([("count", "<u8"), ("sum", "<u8"), ("pct", "<u8", (5,)), ("max", "<u8")])
+assert JOIN.itemsize == 64
+
+
+def join_samples(reference, ref_index, samples):
+    """Returns (rc, out [Q] of JOIN, status)."""
+    ref = np.ascontiguousarray(reference, dtype=INTERVAL)
+    idx = np.ascontiguousarray(ref_index, dtype=np.uint64)
+    smp = np.ascontiguousarray(samples, dtype=INTERVAL)
+    out = np.zeros(len(idx), dtype=JOIN)
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_join_samples(_ptr(ref), len(ref), _ptr(idx), len(idx), _ptr(smp), len(smp), _ptr(out), _ptr(st))
+    return rc, out, st[0]

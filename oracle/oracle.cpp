@@ -442,3 +442,33 @@ extern "C" int oracle_attribute(const uint64_t* counts, uint32_t num_rows, uint3
   }
   return OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Cross-run join with distribution statistics (Sections 3.3 and 3.5; appendix percentiles).
+// ---------------------------------------------------------------------------------------------
+extern "C" int oracle_join_samples(const OInterval* reference, uint64_t num_reference, const uint64_t* ref_index,
+                                   uint32_t num_queries, const OInterval* samples, uint64_t num_samples, OJoin* out,
+                                   OStatus* st) {
+  if (!st || (num_queries && (!reference || !ref_index || !out)) || (num_samples && !samples)) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  for (uint32_t q = 0; q < num_queries; ++q) {
+    if (ref_index[q] >= num_reference) return ERR_INVALID;
+    const OInterval& ref = reference[ref_index[q]];
+    std::vector<uint64_t> values;
+    for (uint64_t i = 0; i < num_samples; ++i) {
+      const OInterval& x = samples[i];
+      if (x.stream == ref.stream && x.region == ref.region && x.ctx == ref.ctx) values.push_back(x.inclusive);
+    }
+    std::sort(values.begin(), values.end());
+    OJoin& o = out[q];
+    std::memset(&o, 0, sizeof(o));
+    o.count = values.size();
+    for (uint64_t v : values) o.sum += v;
+    if (!values.empty()) {
+      for (int j = 0; j < 5; ++j) o.pct[j] = values[(static_cast<size_t>(j) * values.size()) / 5];
+      o.max = values.back();
+    }
+    if (values.size() > 4096 && st->code == 0) fail(st, ERR_CAPACITY, ref.stream, ref_index[q]);
+  }
+  return OK;
+}

@@ -96,6 +96,14 @@ int oracle_map_pc_counts(const OMapEvent* events, const uint64_t* stream_offsets
 int oracle_attribute(const uint64_t* counts, uint32_t num_rows, uint32_t num_pcs, const double* metric,
                      double* mhat, double* entropy, double* alpha);
 
+// Cross-run join (paper Sections 3.3 and 3.5: probe samples are joined to the reference run by region id and
+// dynamic scope, not by timestamps; appendix: mean and 0/20/40/60/80th percentiles over repeated samples).
+// Query q = reference[ref_index[q]]; its samples are all intervals of `samples` with the same
+// (stream, region, ctx); values = their inclusive times, sorted; pct[j] = sorted[(j * count) / 5].
+struct OJoin { uint64_t count, sum; uint64_t pct[5]; uint64_t max; };
+int oracle_join_samples(const OInterval* reference, uint64_t num_reference, const uint64_t* ref_index,
+                        uint32_t num_queries, const OInterval* samples, uint64_t num_samples, OJoin* out, OStatus* st);
+
 // oracle_overlap over the selected intervals only.
 int oracle_overlap_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,

@@ -76,6 +76,8 @@ def load_library():
     lib.argus_attribute_workspace_bytes.restype = sz
     lib.argus_attribute.argtypes = [vp, u32, u32, vp, vp, vp, vp, vp, sz, vp]
     lib.argus_attribute.restype = ci
+    lib.argus_join_samples.argtypes = [vp, u64, vp, u32, vp, u64, vp, vp, vp]
+    lib.argus_join_samples.restype = ci
     lib.argus_status_fetch.argtypes = [vp, vp, vp]
     lib.argus_status_fetch.restype = ci
     lib.argus_strerror.argtypes = [ci]
@@ -430,6 +432,24 @@ def argus_attribute(counts: torch.Tensor, metric: torch.Tensor, want_alpha: bool
     if rc != 0:
         raise ArgusError(rc, "argus_attribute")
     return mhat, entropy, alpha
+
+
+JOIN_DTYPE = np.dtype([("count", "<u8"), ("sum", "<u8"), ("pct", "<u8", (5,)), ("max", "<u8")])  # argus_join_t
+
+
+def argus_join_samples(reference: torch.Tensor, ref_index: torch.Tensor, samples: torch.Tensor):
+    """reference, samples: uint8 tensors of 48-byte interval records; ref_index: int64 [Q].
+    Returns (out uint8 [Q * 64] of argus_join_t, status uint8 [64])."""
+    lib = load_library()
+    dev = reference.device
+    Q = ref_index.numel()
+    out = _bytes(Q * 64, dev)
+    status = _bytes(64, dev)
+    rc = lib.argus_join_samples(_ptr(reference), reference.numel() // 48, _ptr(ref_index), Q, _ptr(samples),
+                                samples.numel() // 48, _ptr(out), _ptr(status), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_join_samples")
+    return out, status
 
 
 @dataclass
