@@ -425,6 +425,28 @@ int argus_join_samples(const argus_interval_t* reference /*device*/, uint64_t nu
                        void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Ring-buffer input — a second container for the marker records of Section 3.2: tracers
+ * commonly give every warp a fixed slot of slot_capacity records and let it wrap. The paper
+ * does not fix a container; this one exercises the recovery path (after a wrap the surviving
+ * records may start with ends whose begins were overwritten: they come out as unmatched-end
+ * ambiguity records).
+ *
+ * ring[s * slot_capacity + (i % slot_capacity)] holds the i-th record stream s wrote;
+ * written[s] counts all records it ever wrote. The surviving records of stream s are the
+ * last min(written[s], slot_capacity), oldest first. argus_ring_linearise copies them into
+ * `events` in packed CSR form and writes stream_offsets[S + 1] (stream_offsets[0] = 0), ready
+ * for argus_pair_intervals; dropped[s] (nullable) = records lost to the wrap. If the packed
+ * records exceed event_capacity nothing is copied and status->code = ARGUS_ERR_CAPACITY with
+ * the required count in status->intervals_required.
+ * ------------------------------------------------------------------------------------- */
+int argus_ring_linearise(const argus_event_t* ring /*device [S][slot_capacity]*/,
+                         uint32_t slot_capacity, const uint64_t* written /*device [S]*/,
+                         uint32_t num_streams, argus_event_t* events /*device*/,
+                         uint64_t event_capacity, uint64_t* stream_offsets /*device [S+1] out*/,
+                         uint64_t* dropped /*device [S] out, nullable*/,
+                         argus_status_t* status /*device*/, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
  * argus_synthesize — the three operations above in one call, with identical results
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *

@@ -56,6 +56,8 @@ def _load():
         lib.oracle_overlap.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp]
         lib.oracle_aggregate_scoped.argtypes = [vp, vp, vp, vp, u32, u32, vp, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_overlap_scoped.argtypes = [vp, vp, u32, u32, vp, u32, vp, u32, vp, vp, vp]
+        lib.oracle_ring_linearise.argtypes = [vp, u32, vp, u32, vp, u64, vp, vp, vp]
+        lib.oracle_ring_linearise.restype = ctypes.c_int
         lib.oracle_join_samples.argtypes = [vp, u64, vp, u32, vp, u64, vp, vp]
         lib.oracle_join_samples.restype = ctypes.c_int
         lib.oracle_map_pc_counts.argtypes = [vp, vp, u32, u32, u32, vp, vp]
@@ -236,3 +238,17 @@ def join_samples(reference, ref_index, samples):
     st = np.zeros(1, dtype=STATUS)
     rc = _load().oracle_join_samples(_ptr(ref), len(ref), _ptr(idx), len(idx), _ptr(smp), len(smp), _ptr(out), _ptr(st))
     return rc, out, st[0]
+
+
+def ring_linearise(ring, slot_capacity, written, event_capacity=None):
+    """ring: EVENT array [S * slot_capacity]; written: [S]. Returns (rc, events, stream_offsets, dropped, status)."""
+    rg = np.ascontiguousarray(ring, dtype=EVENT)
+    wr = np.ascontiguousarray(written, dtype=np.uint64)
+    S = len(wr)
+    cap = int(np.minimum(wr, slot_capacity).sum()) if event_capacity is None else int(event_capacity)
+    ev = np.zeros(max(cap, 1), dtype=EVENT)
+    offs = np.zeros(S + 1, dtype=np.uint64)
+    dropped = np.zeros(max(S, 1), dtype=np.uint64)
+    st = np.zeros(1, dtype=STATUS)
+    rc = _load().oracle_ring_linearise(_ptr(rg), slot_capacity, _ptr(wr), S, _ptr(ev), cap, _ptr(offs), _ptr(dropped), _ptr(st))
+    return rc, ev[:int(offs[-1])] if int(offs[-1]) <= cap else ev[:0], offs, dropped[:S], st[0]

@@ -472,3 +472,29 @@ extern "C" int oracle_join_samples(const OInterval* reference, uint64_t num_refe
   }
   return OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Ring-buffer container -> packed CSR (input handling only; no paper arithmetic involved).
+// ---------------------------------------------------------------------------------------------
+extern "C" int oracle_ring_linearise(const OEvent* ring, uint32_t slot_capacity, const uint64_t* written,
+                                     uint32_t num_streams, OEvent* events, uint64_t event_capacity,
+                                     uint64_t* stream_offsets, uint64_t* dropped, OStatus* st) {
+  if (!st || !stream_offsets || slot_capacity == 0 || (num_streams && (!ring || !written))) return ERR_INVALID;
+  std::memset(st, 0, sizeof(*st));
+  uint64_t total = 0;
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    stream_offsets[s] = total;
+    total += std::min<uint64_t>(written[s], slot_capacity);
+    if (dropped) dropped[s] = written[s] > slot_capacity ? written[s] - slot_capacity : 0;
+  }
+  stream_offsets[num_streams] = total;
+  st->intervals_required = total;
+  if (total > event_capacity) { fail(st, ERR_CAPACITY, 0, total); return OK; }
+  for (uint32_t s = 0; s < num_streams; ++s) {
+    const uint64_t kept = std::min<uint64_t>(written[s], slot_capacity);
+    const uint64_t first = written[s] - kept;  // index of the oldest surviving record
+    for (uint64_t i = 0; i < kept; ++i)
+      events[stream_offsets[s] + i] = ring[static_cast<uint64_t>(s) * slot_capacity + (first + i) % slot_capacity];
+  }
+  return OK;
+}

@@ -104,6 +104,12 @@ struct OJoin { uint64_t count, sum; uint64_t pct[5]; uint64_t max; };
 int oracle_join_samples(const OInterval* reference, uint64_t num_reference, const uint64_t* ref_index,
                         uint32_t num_queries, const OInterval* samples, uint64_t num_samples, OJoin* out, OStatus* st);
 
+// Ring-buffer container (one fixed slot of slot_capacity records per stream, record i at position
+// i % slot_capacity, written[s] records ever written): the surviving records, oldest first, packed in CSR form.
+// The paper fixes no container; this is the layout declared in the library's header.
+int oracle_ring_linearise(const OEvent* ring, uint32_t slot_capacity, const uint64_t* written, uint32_t num_streams,
+                          OEvent* events, uint64_t event_capacity, uint64_t* stream_offsets, uint64_t* dropped, OStatus* st);
+
 // oracle_overlap over the selected intervals only.
 int oracle_overlap_scoped(const OInterval* intervals, const uint64_t* interval_offsets,
                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm,

@@ -78,6 +78,8 @@ def load_library():
     lib.argus_attribute.restype = ci
     lib.argus_join_samples.argtypes = [vp, u64, vp, u32, vp, u64, vp, vp, vp]
     lib.argus_join_samples.restype = ci
+    lib.argus_ring_linearise.argtypes = [vp, u32, vp, u32, vp, u64, vp, vp, vp, vp]
+    lib.argus_ring_linearise.restype = ci
     lib.argus_status_fetch.argtypes = [vp, vp, vp]
     lib.argus_status_fetch.restype = ci
     lib.argus_strerror.argtypes = [ci]
@@ -450,6 +452,24 @@ def argus_join_samples(reference: torch.Tensor, ref_index: torch.Tensor, samples
     if rc != 0:
         raise ArgusError(rc, "argus_join_samples")
     return out, status
+
+
+def argus_ring_linearise(ring: torch.Tensor, slot_capacity: int, written: torch.Tensor, event_capacity: int | None = None):
+    """ring: uint8 [S * slot_capacity * 16]; written: int64 [S] (records each stream ever wrote).
+    Returns (events uint8 [event_capacity * 16], stream_offsets int64 [S + 1], dropped int64 [S], status)."""
+    lib = load_library()
+    dev = ring.device
+    S = written.numel()
+    cap = S * slot_capacity if event_capacity is None else int(event_capacity)
+    events = _bytes(cap * 16, dev)
+    offsets = torch.empty(S + 1, dtype=torch.int64, device=dev)
+    dropped = torch.empty(max(S, 1), dtype=torch.int64, device=dev)
+    status = _bytes(64, dev)
+    rc = lib.argus_ring_linearise(_ptr(ring), slot_capacity, _ptr(written), S, _ptr(events), cap, _ptr(offsets),
+                                  _ptr(dropped), _ptr(status), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_ring_linearise")
+    return events, offsets, dropped[:S], status
 
 
 @dataclass
