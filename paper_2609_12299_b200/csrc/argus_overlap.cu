@@ -1,9 +1,10 @@
 // argus_overlap.cu — argus_overlap: per-SM overlap time of producer/consumer region pairs.
 //
 // Segment = (pair k, SM m, role) with role 0 = producer, 1 = consumer.
-//   k_ov_count   : spans selected per segment
+//   k_ov_select  : one pass over the intervals: selected spans appended to an unordered list with their segment
+//                  (argus_synthesize gets the same list from the aggregation pass or the pairing kernel instead)
+//   k_ov_list_count_or_scatter : spans counted per segment, then copied into their segment (order irrelevant)
 //   k_ov_scan    : segment bases; capacity check
-//   k_ov_scatter : spans (start, end) copied into their segment (order irrelevant)
 //   k_ov_sort    : one CTA per segment: sort by (start, end); then turn the sorted spans into the
 //                  disjoint pieces of their union, piece i = [max(start_i, E_{i-1}), E_i) with
 //                  E_i = max end of spans 0..i, and the running length before each piece
@@ -41,15 +42,30 @@ struct OvArgs {
 
 __device__ __forceinline__ bool ov_mask_bit(const u32* mask, u32 i) { return !mask || ((mask[i >> 5] >> (i & 31)) & 1u); }
 
-__global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatter) {
-  // One stream per block iteration: all of its spans belong to one SM, so the block counts per
-  // (pair, role) in shared memory and touches each global counter once.
+// One pass over the intervals: spans of intervals whose region appears in a pair are appended to an unordered
+// list with their segment. A warp reserves `chunk` list slots at a time (one global atomic per chunk) and
+// marks the slots it leaves unused, so the list needs no clearing.
+struct OvSelectOut {
+  ulonglong2* spans;
+  u32* seg;
+  u64* count;      // slots reserved so far (zeroed before the kernel)
+  u64 capacity;
+  u32 chunk;       // power of two, at most 256
+};
+
+__device__ __forceinline__ void ov_retire_chunk(const OvSelectOut& o, u64 base, u32 used, u32 lane) {
+  for (u32 i = used + lane; i < o.chunk; i += 32)
+    if (base + i < o.capacity) o.seg[base + i] = 0xffffffffu;
+}
+
+__global__ void __launch_bounds__(256) k_ov_select(OvArgs a, OvSelectOut o) {
   __shared__ u32 sh_pairs[2 * kMaxPairs];
-  __shared__ u32 sh_cnt[2 * kMaxPairs];
-  __shared__ u64 sh_base[2 * kMaxPairs];
   for (u32 i = threadIdx.x; i < 2 * a.num_pairs; i += blockDim.x) sh_pairs[i] = a.pairs[i];
   __syncthreads();
-  if (scatter && a.status->code != 0) return;
+  const u32 lane = threadIdx.x & 31;
+  u64 ovc_base = 0;          // warp-uniform: the chunk this warp is filling
+  u32 ovc_used = o.chunk;    // chunk size = none held yet
+  bool held = false;
   for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
     const u32 m = a.cta_sm[s / a.warps_per_cta];
     const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
@@ -62,41 +78,54 @@ __global__ void __launch_bounds__(256) k_ov_count_or_scatter(OvArgs a, int scatt
       if (a.warp_mask != ~0ull && (w >= 64 || !((a.warp_mask >> w) & 1ull))) continue;
       if (!ov_mask_bit(a.sm_mask, m)) continue;
     }
-    for (u32 i = threadIdx.x; i < 2 * a.num_pairs; i += blockDim.x) sh_cnt[i] = 0;
-    __syncthreads();
-    for (int pass = 0; pass < (scatter ? 2 : 1); ++pass) {
-      for (u64 i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+    // every lane of a warp runs the same number of rounds, so that spans can be appended a warp at a time
+    for (u64 base = lo + (threadIdx.x & ~31u); base < hi; base += blockDim.x) {
+      const u64 i = base + lane;
+      bool cand = false;
+      u32 region = 0;
+      u64 t0 = 0, incl = 0;
+      if (i < hi) {
         const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
         const uint4 q0 = __ldg(p);
-        const u64 incl = (u64)q0.z | ((u64)q0.w << 32);
-        if (incl == 0) continue;
-        const u32 region = __ldg(reinterpret_cast<const u32*>(p + 1) + 2);
-        if (a.scoped) {  // iteration-window and region tests: one answer per interval
+        incl = (u64)q0.z | ((u64)q0.w << 32);
+        t0 = (u64)q0.x | ((u64)q0.y << 32);
+        region = __ldg(reinterpret_cast<const u32*>(p + 1) + 2);
+        cand = incl != 0;
+        if (cand && a.scoped) {  // iteration-window and region tests: one answer per interval
           const u32 ctx = __ldg(reinterpret_cast<const u32*>(p + 1) + 3);
-          if (ctx < a.ctx_lo || ctx > a.ctx_hi || !ov_mask_bit(a.region_mask, region)) continue;
+          cand = ctx >= a.ctx_lo && ctx <= a.ctx_hi && ov_mask_bit(a.region_mask, region);
         }
-        const u64 t0 = (u64)q0.x | ((u64)q0.y << 32);
-        for (u32 k = 0; k < 2 * a.num_pairs; ++k) {
-          if (sh_pairs[k] != region) continue;
-          const u32 local = atomicAdd(&sh_cnt[k], 1u);
-          if (pass == 1) {
-            const u64 slot = sh_base[k] + local;
-            if (slot < a.capacity) a.spans[slot] = make_ulonglong2(t0, t0 + incl);
+      }
+      for (u32 k = 0; k < 2 * a.num_pairs; ++k) {
+        const bool pick = cand && sh_pairs[k] == region;
+        const u32 bal = __ballot_sync(0xffffffffu, pick);
+        if (!bal) continue;
+        u32 todo = __popc(bal), done = 0;
+        while (todo) {  // a ballot may straddle chunks when the chunks are small
+          if (ovc_used == o.chunk) {
+            u64 nb64 = 0;
+            if (lane == 0) nb64 = atomicAdd(reinterpret_cast<unsigned long long*>(o.count), (unsigned long long)o.chunk);
+            ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
+            ovc_used = 0;
+            held = true;
           }
+          const u32 room = o.chunk - ovc_used, take = todo < room ? todo : room;
+          if (pick) {
+            const u32 rank = __popc(bal & ((1u << lane) - 1u));
+            if (rank >= done && rank < done + take) {
+              const u64 slot = ovc_base + ovc_used + (rank - done);
+              if (slot < o.capacity) {
+                o.spans[slot] = make_ulonglong2(t0, t0 + incl);
+                o.seg[slot] = ((k >> 1) * a.num_sms + m) * 2 + (k & 1u);
+              }
+            }
+          }
+          ovc_used += take; done += take; todo -= take;
         }
       }
-      __syncthreads();
-      for (u32 k = threadIdx.x; k < 2 * a.num_pairs; k += blockDim.x) {
-        const u32 seg = ((k >> 1) * a.num_sms + m) * 2 + (k & 1u);
-        if (pass == 0 && sh_cnt[k]) {
-          if (!scatter) atomicAdd(&a.seg_count[seg], (u64)sh_cnt[k]);
-          else sh_base[k] = a.seg_base[seg] + atomicAdd(&a.seg_cursor[seg], (u64)sh_cnt[k]);
-        }
-        sh_cnt[k] = 0;
-      }
-      __syncthreads();
     }
   }
+  if (held) ov_retire_chunk(o, ovc_base, ovc_used, lane);
 }
 
 // Same two roles for spans that the pairing kernel already selected: list entries carry their segment;
@@ -331,25 +360,25 @@ OvLayout ov_layout(uint32_t nseg) {
 
 }  // namespace
 
+constexpr size_t kBytesPerSortedSpan = 24;  // (begin, end) + covered length before it
+constexpr size_t kBytesPerListedSpan = 20;  // (begin, end) + segment
+constexpr unsigned kSelectGrid = 148 * 8;
+constexpr unsigned kSelectWarps = kSelectGrid * 8;
+
 extern "C" size_t argus_overlap_workspace_bytes(uint64_t max_intervals, uint32_t /*num_streams*/, uint32_t num_pairs,
                                                 uint32_t num_sms) {
   const OvLayout L = ov_layout(num_pairs * num_sms * 2);
-  // worst case: every interval selected in both roles of every pair; 24 bytes per selected span
-  return L.total_fixed + argus_align_up((size_t)max_intervals * 2 * num_pairs * 24 + 256, 256);
+  // worst case: every interval selected in both roles of every pair, listed and then sorted; a third more
+  // list slots than spans cover the slots that warps reserve and leave unused
+  const size_t spans = (size_t)max_intervals * 2 * num_pairs;
+  return L.total_fixed + argus_align_up((spans + spans / 3 + 64) * (kBytesPerSortedSpan + kBytesPerListedSpan) + 1024, 256);
 }
 
-// Shared tail of both entry paths. `list` null: spans are selected from the interval array;
-// otherwise they come from the list the pairing kernel appended.
+// Shared tail of both entry paths: from the list of selected spans to the overlap measures.
 static int ov_run(OvArgs& a, const OvList* list, cudaStream_t stream) {
-  const unsigned sel_grid = a.num_streams < 2368 ? (a.num_streams ? a.num_streams : 1) : 2368;
   for (int pass = 0; pass < 2; ++pass) {
-    if (list) {
-      k_ov_list_count_or_scatter<<<592, 256, 0, stream>>>(a, *list, pass);
-      ARGUS_CHECK_LAUNCH();
-    } else if (a.num_streams) {
-      k_ov_count_or_scatter<<<sel_grid, 256, 0, stream>>>(a, pass);
-      ARGUS_CHECK_LAUNCH();
-    }
+    k_ov_list_count_or_scatter<<<592, 256, 0, stream>>>(a, *list, pass);
+    ARGUS_CHECK_LAUNCH();
     if (pass == 0) {
       k_ov_scan<<<1, kOvThreads, 0, stream>>>(a);
       ARGUS_CHECK_LAUNCH();
@@ -366,10 +395,11 @@ static int ov_run(OvArgs& a, const OvList* list, cudaStream_t stream) {
 
 static int ov_setup(OvArgs& a, uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
                     const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status, void* workspace,
-                    size_t workspace_bytes, cudaStream_t stream) {
+                    size_t workspace_bytes, cudaStream_t stream, size_t own_list_bytes = 0) {
   const u32 nseg = num_pairs * num_sms * 2;
   const OvLayout L = ov_layout(nseg);
-  if (workspace_bytes < L.total_fixed + 256) return ARGUS_ERR_WORKSPACE;
+  if (workspace_bytes < L.total_fixed + 256 + own_list_bytes) return ARGUS_ERR_WORKSPACE;
+  workspace_bytes -= own_list_bytes;  // the caller keeps its list behind the part laid out here
   char* ws = (char*)workspace;
   a.intervals = nullptr; a.interval_offsets = nullptr; a.num_streams = num_streams;
   a.warps_per_cta = warps_per_cta; a.num_sms = num_sms; a.num_pairs = num_pairs; a.cta_sm = cta_sm; a.pairs = pairs;
@@ -415,15 +445,38 @@ static int overlap_scoped(const argus_interval_t* intervals, uint64_t max_interv
   if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
   if (num_pairs == 0) return ARGUS_OK;
   OvArgs a;
+  // split what the workspace offers beyond the fixed part between the list (20 B a slot) and the sorted spans
+  // (24 B each), with a third more list slots than sorted spans
+  const OvLayout L0 = ov_layout(num_pairs * num_sms * 2);
+  if (workspace_bytes < L0.total_fixed + 2048) return ARGUS_ERR_WORKSPACE;
+  const u64 span_cap = (workspace_bytes - L0.total_fixed - 1536) * 3 / (3 * kBytesPerSortedSpan + 4 * kBytesPerListedSpan);
+  const u64 list_cap = span_cap + span_cap / 3;
+  const size_t list_bytes = argus_align_up(256 + argus_align_up((size_t)list_cap * 4, 256) + (size_t)list_cap * 16, 256);
   const int rc = ov_setup(a, num_streams, warps_per_cta, cta_sm, num_sms, pairs, num_pairs, out, status, workspace,
-                          workspace_bytes, stream);
+                          workspace_bytes, stream, list_bytes);
   if (rc != ARGUS_OK) return rc;
   a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets;
   if (scope) {
     a.scoped = 1; a.ctx_lo = scope->ctx_lo; a.ctx_hi = scope->ctx_hi; a.warp_mask = scope->warp_mask;
     a.sm_mask = scope->sm_mask; a.region_mask = scope->region_mask;
   }
-  return ov_run(a, nullptr, stream);
+  // the list of selected spans sits at the end of the workspace: counter, segments, spans
+  char* lbase = (char*)workspace + (workspace_bytes - list_bytes);
+  OvSelectOut o;
+  o.count = (u64*)lbase;
+  o.seg = (u32*)(lbase + 256);
+  o.spans = (ulonglong2*)(lbase + 256 + argus_align_up((size_t)list_cap * 4, 256));
+  o.capacity = list_cap;
+  o.chunk = 256;  // slots left unused are bounded by a quarter of the list: smaller chunks for small lists
+  while (o.chunk > 1 && (u64)kSelectWarps * o.chunk * 4 > list_cap) o.chunk >>= 1;
+  ARGUS_CUDA_TRY(cudaMemsetAsync(o.count, 0, 256, stream));
+  if (num_streams) {
+    k_ov_select<<<num_streams < kSelectGrid ? num_streams : kSelectGrid, 256, 0, stream>>>(a, o);
+    ARGUS_CHECK_LAUNCH();
+  }
+  OvList l;
+  l.spans = o.spans; l.seg = o.seg; l.count = o.count; l.capacity = list_cap;
+  return ov_run(a, &l, stream);
 }
 
 int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,

@@ -78,7 +78,7 @@ def run_scoped(iters: int):
                                               levels=("warp", "cta", "sm", "kernel", "role", "iter")), 1.0),
         ("argus_overlap_scoped, 16 iterations", lambda: argus.argus_overlap_scoped(p.intervals, n // 2, p.interval_offsets, W,
                                                                                    cta_sm, M, pairs,
-                                                                                   argus.ArgusScope(lo, lo + 15)), 2.0),
+                                                                                   argus.ArgusScope(lo, lo + 15)), 1.0),
     ]
     for what, fn, passes in cases:
         _line(what, _time(fn), iv_bytes * passes, intervals=iv_bytes // 48, workload=spec.name,
