@@ -698,29 +698,17 @@ extern "C" int argus_debug_tile_timing(unsigned long long* out8) {
 }
 #endif
 
-// Tile shape used by the tiled kernel: 0 = default. Other values select alternative shapes (tuning aid).
+// Tile shape used by the tiled kernel: 0 = automatic; 1..5 select the other compiled shapes
+// <threads, events per thread, CTAs per SM> (tuning and test aid; results do not depend on it).
 extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   switch (g_variant) {
-    case 1: return launch_tiled_any<128, 5, 4>(a, stream);
-    case 2: return launch_tiled_any<128, 7, 4>(a, stream);
-    case 3: return launch_tiled_any<256, 7, 2>(a, stream);
-    case 4: return launch_tiled_any<128, 9, 3>(a, stream);
-    case 5: return launch_tiled_any<256, 5, 2>(a, stream);
-    case 6: return launch_tiled_any<64, 5, 8>(a, stream);
-    case 7: return launch_tiled_any<64, 7, 8>(a, stream);
-    case 8: return launch_tiled_any<192, 5, 4>(a, stream);
-    case 9: return launch_tiled_any<256, 3, 4>(a, stream);
-    case 10: return launch_tiled_any<320, 5, 2>(a, stream);
-    case 11: return launch_tiled_any<352, 5, 2>(a, stream);
-    case 12: return launch_tiled_any<288, 5, 2>(a, stream);
-    case 13: return launch_tiled_any<512, 3, 1>(a, stream);
-    case 14: return launch_tiled_any<224, 7, 2>(a, stream);
-    case 15: return launch_tiled_any<256, 5, 3>(a, stream);
-    case 16: return launch_tiled_any<160, 5, 5>(a, stream);
-    case 17: return launch_tiled_any<96, 5, 8>(a, stream);
-    case 18: return launch_tiled_any<128, 5, 6>(a, stream);
+    case 1: return launch_tiled_any<192, 5, 4>(a, stream);
+    case 2: return launch_tiled_any<320, 5, 2>(a, stream);
+    case 3: return launch_tiled_any<64, 5, 8>(a, stream);
+    case 4: return launch_tiled_any<256, 7, 2>(a, stream);
+    case 5: return launch_tiled_any<160, 5, 5>(a, stream);
     default: {
       // automatic. Plain pairing: six CTAs of 128 threads per SM (with streams walked in chunks the number of
       // streams per SM does not have to divide evenly). With the aggregation table inside the kernel: four CTAs

@@ -416,3 +416,21 @@ def test_synthesize_long_streams(idx, ctas, iters):
     ev, offs = tg.generate_host(spec)
     assert np.diff(offs).max() > 70_000
     _synthesize_matches(spec, ev, offs)
+
+
+@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5])
+def test_other_tile_shapes_give_the_same_result(variant):
+    """The compiled alternatives to the default tile shape (threads x events per thread x CTAs per SM), on a
+    malformed trace with streams several tiles long and on the one-call pipeline in every mode."""
+    from paper_2609_12299_b200.binding import argus_set_synthesize_mode, argus_set_tile_variant
+    spec = tg.config(4).scaled(3, 700)
+    ev, offs = tg.generate_host(spec)
+    argus_set_tile_variant(variant)
+    try:
+        assert_pair_matches(ev, offs, spec.num_regions, KERNEL_TILED)
+        for mode in (0, 1):
+            argus_set_synthesize_mode(mode)
+            _synthesize_matches(spec, ev, offs)
+    finally:
+        argus_set_tile_variant(0)
+        argus_set_synthesize_mode(-1)
