@@ -19,6 +19,8 @@ constexpr int kAggThreads = 256;
 constexpr u32 kCell = 72;  // u64 words per argus_agg_t
 constexpr size_t kAggSmemLimit = 200 * 1024;
 constexpr u32 kAggCompactRegions = 400;  // 112 B each: 44.8 KB of shared memory at most
+constexpr size_t kIterScratchBytes = 32u << 20;  // workspace for private copies of an iteration table
+constexpr u32 kIterMaxCopies = 32;
 
 struct AggArgs {
   const argus_interval_t* intervals;
@@ -43,6 +45,9 @@ struct AggArgs {
   u64* iter_tab;  // [num_iters][R][72], nullable
   u32 num_iters;
   int iter_smem;
+  u64* iter_copies;   // global path: private copies of the iteration table, one per group of blocks (null: none)
+  u32 num_copies;
+  int iter_inline;    // global path taken inside k_agg_streams_compact (one read of the intervals serves both)
   // overlap span selection in the same pass over the intervals (argus_synthesize); ov.ov_spans null = off
   ArgusFuseArgs ov;
 };
@@ -77,6 +82,19 @@ __device__ __forceinline__ void agg_add_interval(u64* tab, u32 region, u64 incl,
   atomicAdd(c + 1, incl);
   atomicMin(c + 2, incl);
   atomicMax(c + 3, incl);
+  atomicAdd(c + 4, excl);
+  if (flags) atomicAdd(c + 7, 1ull);
+  atomicAdd(c + 8 + log2_bin(incl), 1ull);
+}
+
+// The same for a table in global memory that many blocks share: three atomics per interval instead of six. The
+// count is left out (it is the sum of the histogram bins and is filled in afterwards) and min / max are
+// only updated while they still move (a stale read only costs a redundant atomic).
+__device__ __forceinline__ void agg_add_interval_lean(u64* tab, u32 region, u64 incl, u64 excl, u32 flags) {
+  u64* c = tab + (size_t)region * kCell;
+  atomicAdd(c + 1, incl);
+  if (incl < __ldcg(c + 2)) atomicMin(c + 2, incl);
+  if (incl > __ldcg(c + 3)) atomicMax(c + 3, incl);
   atomicAdd(c + 4, excl);
   if (flags) atomicAdd(c + 7, 1ull);
   atomicAdd(c + 8 + log2_bin(incl), 1ull);
@@ -136,6 +154,9 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
   u32* const pairbits = reinterpret_cast<u32*>(ctab + R);
   u32* const pairs_sm = pairbits + (R + 31) / 32;
   const bool has_ov = a.ov.ov_spans != nullptr && a.ov.num_pairs != 0;
+  // iteration table too large for shared memory: this block's private copy in global memory (or the table itself)
+  u64* const iter_base = !a.iter_inline ? nullptr
+                         : a.iter_copies ? a.iter_copies + (u64)(blockIdx.x % a.num_copies) * a.num_iters * cells : a.iter_tab;
   u64 ovc_base = 0;             // warp-uniform: current chunk of the global span list
   u32 ovc_used = kAggOvChunk;
   if (has_ov) {
@@ -184,7 +205,9 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
           } else if (record_in_scope(a, q1.w, region)) {
             t0 = (u64)q0.x | ((u64)q0.y << 32);
             incl = (u64)q0.z | ((u64)q0.w << 32);
-            argus_fuse_aggregate(fx, region, incl, (u64)q1.x | ((u64)q1.y << 32), q2.w >> 16);
+            const u64 excl = (u64)q1.x | ((u64)q1.y << 32);
+            argus_fuse_aggregate(fx, region, incl, excl, q2.w >> 16);
+            if (a.iter_inline) agg_add_interval_lean(iter_base + (u64)(q1.w - a.ctx_lo) * cells, region, incl, excl, q2.w >> 16);
             cand = has_ov && incl && ((pairbits[region >> 5] >> (region & 31)) & 1u);
           }
         }
@@ -218,7 +241,9 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
         const u32 region = a.ambig[i].tag >> 1;
         if (region >= R) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
         if (!record_in_scope(a, a.ambig[i].ctx, region)) continue;
-        atomicAdd(row + (size_t)region * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
+        const u32 which = a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5;
+        atomicAdd(row + (size_t)region * kCell + which, 1ull);
+        if (a.iter_inline) atomicAdd(iter_base + ((u64)(a.ambig[i].ctx - a.ctx_lo) * R + region) * kCell + which, 1ull);
       }
     }
     __syncthreads();
@@ -293,7 +318,9 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_iter(AggArgs a) {
   extern __shared__ __align__(16) u64 sh_tab[];
   const u32 R = a.num_regions;
   const u64 cells = (u64)a.num_iters * R * kCell;
-  u64* tab = a.iter_smem ? sh_tab : a.iter_tab;
+  // too large for shared memory: blocks add to one of a few private copies in global memory, which spreads the
+  // atomics over more addresses; k_agg_iter_reduce combines the copies afterwards
+  u64* tab = a.iter_smem ? sh_tab : a.iter_copies ? a.iter_copies + (u64)(blockIdx.x % a.num_copies) * cells : a.iter_tab;
   if (a.iter_smem) {
     for (u64 i = threadIdx.x; i < cells; i += blockDim.x) sh_tab[i] = (i % kCell == 2) ? ~0ull : 0ull;
     __syncthreads();
@@ -307,8 +334,10 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_iter(AggArgs a) {
       const u32 region = q1.z, ctx = q1.w;
       if (region >= R || !record_in_scope(a, ctx, region)) continue;
       const uint4 q0 = __ldg(p), q2 = __ldg(p + 2);
-      agg_add_interval(tab + (u64)(ctx - a.ctx_lo) * R * kCell, region, (u64)q0.z | ((u64)q0.w << 32),
-                       (u64)q1.x | ((u64)q1.y << 32), q2.w >> 16);
+      u64* row = tab + (u64)(ctx - a.ctx_lo) * R * kCell;
+      const u64 incl = (u64)q0.z | ((u64)q0.w << 32), excl = (u64)q1.x | ((u64)q1.y << 32);
+      if (a.iter_smem) agg_add_interval(row, region, incl, excl, q2.w >> 16);
+      else agg_add_interval_lean(row, region, incl, excl, q2.w >> 16);
     }
     if (a.ambig && a.ambig_offsets) {
       const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
@@ -331,6 +360,31 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_iter(AggArgs a) {
   }
 }
 
+// iter_tab[i] = combination of cell word i over the private copies (none: iter_tab holds the sums already);
+// the interval count of a cell, which the global path leaves out, is the sum of its histogram bins.
+__global__ void __launch_bounds__(256) k_agg_iter_reduce(AggArgs a) {
+  const u64 cells = (u64)a.num_iters * a.num_regions * kCell;
+  if (a.iter_copies) {
+    for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < cells; i += (u64)gridDim.x * blockDim.x) {
+      const u32 field = (u32)(i % kCell);
+      if (field == 0) continue;
+      u64 acc = a.iter_copies[i];
+      for (u32 c = 1; c < a.num_copies; ++c) acc = combine(field, acc, a.iter_copies[(u64)c * cells + i]);
+      a.iter_tab[i] = acc;
+    }
+  }
+  for (u64 cell = (u64)blockIdx.x * blockDim.x + threadIdx.x; cell < cells / kCell; cell += (u64)gridDim.x * blockDim.x) {
+    u64 n = 0;
+    for (u32 b = 0; b < 64; ++b) {
+      u64 v = 0;
+      if (a.iter_copies) for (u32 c = 0; c < a.num_copies; ++c) v += a.iter_copies[(u64)c * cells + cell * kCell + 8 + b];
+      else v = a.iter_tab[cell * kCell + 8 + b];
+      n += v;
+    }
+    a.iter_tab[cell * kCell] = n;
+  }
+}
+
 // ambiguity counters into the warp-scope table (used when the intervals were aggregated by the pairing kernel)
 __global__ void __launch_bounds__(256) k_agg_ambig(AggArgs a) {
   for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
@@ -344,14 +398,15 @@ __global__ void __launch_bounds__(256) k_agg_ambig(AggArgs a) {
   }
 }
 
-struct AggLayout { size_t warp, cta, total; };
+struct AggLayout { size_t warp, cta, iter, total; };
 
 AggLayout agg_layout(uint32_t num_streams, uint32_t num_regions) {
   AggLayout L;
   const size_t row = (size_t)num_regions * sizeof(argus_agg_t);
   L.warp = 0;
   L.cta = argus_align_up((size_t)num_streams * row, 256);
-  L.total = L.cta + argus_align_up((size_t)num_streams * row, 256);  // C <= S
+  L.iter = L.cta + argus_align_up((size_t)num_streams * row, 256);  // C <= S
+  L.total = L.iter + kIterScratchBytes;
   return L;
 }
 
@@ -387,7 +442,8 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
   a.warp_tab = (u64*)warp_tab; a.cta_tab = (u64*)cta_work; a.sm_tab = (u64*)sm_tab; a.kernel_tab = (u64*)kernel_tab;
   a.status = status; a.use_smem = 0;
   a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
-  a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0;
+  a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0; a.iter_copies = nullptr; a.num_copies = 0;
+  a.iter_inline = 0;
   a.ov.ov_spans = nullptr; a.ov.num_pairs = 0;
   if (ambig && ambig_offsets) {
     k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
@@ -425,9 +481,9 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   const u32 num_iters = iter_tab ? scope->ctx_hi - scope->ctx_lo + 1 : 0;
   if (kernel_tab) { k_agg_init<<<16, 256, 0, stream>>>((u64*)kernel_tab, (u64)num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
   if (sm_tab) { k_agg_init<<<296, 256, 0, stream>>>((u64*)sm_tab, (u64)num_sms * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
-  if (iter_tab) { k_agg_init<<<296, 256, 0, stream>>>((u64*)iter_tab, (u64)num_iters * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
   if (num_streams == 0) {
     if (role_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)role_tab, (u64)warps_per_cta * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
+    if (iter_tab) { k_agg_init<<<64, 256, 0, stream>>>((u64*)iter_tab, (u64)num_iters * num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
     return ARGUS_OK;
   }
   AggArgs a;
@@ -447,11 +503,26 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   a.use_smem = smem <= kAggSmemLimit;
   const size_t iter_bytes = (size_t)num_iters * smem;
   a.iter_smem = iter_tab && iter_bytes <= kAggSmemLimit;
+  a.iter_copies = nullptr; a.num_copies = 0;
+  if (iter_tab && !a.iter_smem && 2 * iter_bytes <= kIterScratchBytes) {
+    a.num_copies = (u32)(kIterScratchBytes / iter_bytes < kIterMaxCopies ? kIterScratchBytes / iter_bytes : kIterMaxCopies);
+    a.iter_copies = (u64*)((char*)workspace + L.iter);
+  }
   const size_t need = a.use_smem ? smem : 0, need_iter = a.iter_smem ? iter_bytes : 0;
   if (need > 48 * 1024)
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need));
   if (need_iter > 48 * 1024)
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_iter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need_iter));
+  const u64 iter_cells = (u64)num_iters * num_regions * kCell;
+  a.iter_inline = iter_tab && !a.iter_smem && num_regions <= kAggCompactRegions;
+  if (iter_tab) {
+    if (a.iter_copies) {
+      k_agg_init<<<592, 256, 0, stream>>>(a.iter_copies, iter_cells * a.num_copies);
+    } else {
+      k_agg_init<<<296, 256, 0, stream>>>((u64*)iter_tab, iter_cells);
+    }
+    ARGUS_CHECK_LAUNCH();
+  }
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 0);
   if (num_regions <= kAggCompactRegions) {
     const size_t compact = (size_t)num_regions * sizeof(ArgusAggCell) + ((num_regions + 31) / 32) * 4 + (size_t)a.ov.num_pairs * 8;
@@ -464,8 +535,15 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_AGGREGATE, stream, 1);
   if (iter_tab) {
-    k_agg_iter<<<num_streams < 296 ? num_streams : 296, kAggThreads, need_iter, stream>>>(a);
-    ARGUS_CHECK_LAUNCH();
+    if (!a.iter_inline) {
+      const unsigned iter_grid = a.iter_smem ? 296u : 148u * 8u;
+      k_agg_iter<<<num_streams < iter_grid ? num_streams : iter_grid, kAggThreads, need_iter, stream>>>(a);
+      ARGUS_CHECK_LAUNCH();
+    }
+    if (!a.iter_smem) {
+      k_agg_iter_reduce<<<296, 256, 0, stream>>>(a);
+      ARGUS_CHECK_LAUNCH();
+    }
   }
   if (role_tab) {
     k_agg_role<<<296, 256, 0, stream>>>(a);
