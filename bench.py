@@ -24,7 +24,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "marker events/sec (pair+aggregate+overlap, whole hot path)"
+METRIC = "marker events/sec (pair+aggregate, 1 B200) and % of HBM roofline"  # the step also runs the overlap stage
 UNIT = "events/s"
 ALG_BYTES_PER_EVENT = 40.0  # 16 B event read + 48 B interval written per 2 events
 NCU_DRAM_BYTES_PER_EVENT = (614.345216e6 + 866.522368e6) / 38380544  # pairing kernel, ncu capture summarised in profiles/
