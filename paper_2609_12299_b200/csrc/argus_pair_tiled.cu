@@ -652,21 +652,26 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
 
 template <int NT, int E, int MINB, bool FUSE>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
-  static int grid_cache = 0;
-  static size_t smem_cache = 0;
+  // the shared-memory opt-in and the occupancy belong to one device: cached per device, redone when the size changes
+  constexpr int kMaxDevices = 64;
+  static int grid_of[kMaxDevices];
+  static size_t smem_of[kMaxDevices];
   size_t smem = ((sizeof(TileSmem<NT, E>) + 15) & ~(size_t)15) + 128;
   if (FUSE) smem += (a.fuse.warp_tab ? (size_t)a.num_regions * sizeof(ArgusAggCell) : 0) + ((a.num_regions + 31) / 32) * 4 + (size_t)a.fuse.num_pairs * 8 + 16;
-  if (!grid_cache || smem_cache != smem) {
+  int dev = 0;
+  ARGUS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return ARGUS_ERR_INVALID_ARG;
+  if (!grid_of[dev] || smem_of[dev] != smem) {
     ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int dev = 0, sms = 0, per_sm = 0;
-    ARGUS_CUDA_TRY(cudaGetDevice(&dev));
+    int sms = 0, per_sm = 0;
     ARGUS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB, FUSE>, NT, smem));
     if (per_sm < 1) return ARGUS_ERR_CUDA;
     if (per_sm > MINB) per_sm = MINB;
-    grid_cache = sms * per_sm;
-    smem_cache = smem;
+    grid_of[dev] = sms * per_sm;
+    smem_of[dev] = smem;
   }
+  const int grid_cache = grid_of[dev];
   const u32 grid = a.num_streams < (u32)grid_cache ? a.num_streams : (u32)grid_cache;
   k_pair_tiled<NT, E, MINB, FUSE><<<grid, NT, smem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
