@@ -144,9 +144,16 @@ __device__ __forceinline__ int tile_latest_begin(const TileSmem<NT, E>& sm, int 
     const u32 m = sm.bm[l][w] & ((1u << (pos & 31)) - 1u);
     if (m) return w * 32 + 31 - __clz(m);
   }
-  const u64 s = sm.summ[l] & ((w >= 64) ? ~0ull : ((1ull << w) - 1ull));
-  if (!s) return -1;
-  const int w2 = 63 - __clzll((long long)s);
+  int w2;
+  if (NWORDS <= 32) {  // one 32-bit word of the summary covers the tile
+    const u32 s = reinterpret_cast<const u32*>(&sm.summ[l])[0] & ((w >= 32) ? ~0u : ((1u << w) - 1u));
+    if (!s) return -1;
+    w2 = 31 - __clz(s);
+  } else {
+    const u64 s = sm.summ[l] & ((w >= 64) ? ~0ull : ((1ull << w) - 1ull));
+    if (!s) return -1;
+    w2 = 63 - __clzll((long long)s);
+  }
   const u32 m2 = sm.bm[l][w2];
   return m2 ? w2 * 32 + 31 - __clz(m2) : -1;
 }
