@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         for (int k = 0; k < E; ++k) {
           const int e = w0 + tid * E + k;
           tags[k] = e < wend ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;  // all ones = no event
-          if (e < wend) accb[e] = 0;
+          if (!(tags[k] & 1u)) accb[e] = 0;  // child time is gathered at begins only
           (&sm.bm[0][0])[tid * E + k] = 0;  // kLevelWindow * NWORDS == T words
           if (tags[k] != 0xffffffffu) { if (tags[k] & 1u) ++ne; else ++nb; }
         }
