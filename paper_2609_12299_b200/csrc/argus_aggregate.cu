@@ -11,7 +11,7 @@
 //   k_agg_iter    : per-iteration cells (key = ctx - ctx_lo) of the intervals of a scope.
 // A scope (iteration window, warp mask, SM mask, region mask) filters what k_agg_streams and
 // k_agg_iter take in; without one everything is selected.
-#include "argus_fuse.cuh"
+#include "argus_internal.cuh"
 
 namespace {
 

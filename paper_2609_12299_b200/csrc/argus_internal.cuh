@@ -1,0 +1,53 @@
+// argus_internal.cuh — functions one translation unit of the library offers to the others (not part of the C-ABI).
+#ifndef ARGUS_INTERNAL_CUH_
+#define ARGUS_INTERNAL_CUH_
+
+#include "argus_fuse.cuh"
+
+// argus_pair.cu — the whole pairing pipeline. kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled.
+// `fuse` (nullable) asks the tiled kernel to feed aggregation / overlap selection; *fused_out tells whether it did.
+int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                        uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                        uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                        uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
+                        bool reset_status, bool* fused_out);
+
+// argus_pair_tiled.cu
+bool argus_pair_tiled_can_fuse(uint32_t num_regions);
+bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs);
+
+// argus_aggregate.cu
+int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                             const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                             uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                             argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
+                             argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                             bool reset_status);
+// scope, role_tab, iter_tab nullable; ov_select (nullable): also append the overlap spans of the selected intervals
+int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
+                                    const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                                    uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                                    const argus_scope_t* scope, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                                    argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
+                                    argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
+                                    size_t workspace_bytes, void* cuda_stream, bool reset_status,
+                                    const ArgusFuseArgs* ov_select);
+// second half of aggregation when the pairing kernel already filled the interval statistics of warp_tab
+int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
+                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
+                              argus_agg_t* warp_tab, argus_agg_t* cta_work, bool want_cta, argus_agg_t* sm_tab,
+                              argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream);
+bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs);
+
+// argus_overlap.cu
+int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
+                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
+                           const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status);
+// overlap from a list of selected spans (spans + segment of each; *list_count slots reserved, unused ones tagged 0xffffffff)
+int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* list_seg, const uint64_t* list_count,
+                                     uint64_t list_capacity, uint32_t num_sms, uint32_t num_pairs, argus_overlap_t* out,
+                                     argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#endif  // ARGUS_INTERNAL_CUH_

@@ -10,7 +10,7 @@
 //                  E_i = max end of spans 0..i, and the running length before each piece
 //   k_ov_measure : one CTA per (k, m): |U_P|, |U_C|, and |U_P ∩ U_C| = sum over producer pieces of
 //                  F_C(b) - F_C(a), F_C(t) = covered length of U_C before t (binary search in C pieces)
-#include "argus_common.cuh"
+#include "argus_internal.cuh"
 
 namespace {
 

@@ -8,6 +8,7 @@
 //   pair pass 2   : only does work when `redo` is set (malformed traces): rewrites intervals at the
 //                   final bases
 //   ambiguity     : popcount prefix over the bitmap -> rank of every note -> ordered records, offsets
+#include "argus_internal.cuh"
 #include "argus_pair_common.cuh"
 
 #include <string.h>
@@ -206,7 +207,6 @@ Layout make_layout(uint64_t num_events, uint32_t num_streams, uint64_t ambig_cap
 // implemented in argus_pair_tiled.cu
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream);
 bool argus_pair_tiled_usable(const ArgusPairArgs& a);
-bool argus_pair_tiled_can_fuse(uint32_t num_regions);
 
 extern "C" size_t argus_pair_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint64_t ambig_capacity) {
   return make_layout(num_events, num_streams, ambig_capacity).total;

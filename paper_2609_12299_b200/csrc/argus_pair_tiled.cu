@@ -17,6 +17,7 @@
 // id). Any doubt (region mismatch, negative height, bad region id, depth overflow, level window
 // exceeded) makes the CTA redo that tile with the sequential stack machine on the carried stack, so
 // the result is always the sequential definition's.
+#include "argus_internal.cuh"
 #include "argus_pair_common.cuh"
 
 namespace {

@@ -4,14 +4,8 @@
 // to someone else, paths where an allocation could synchronise or fail): the pairing pipeline's
 // scratch sits in a fixed array in this library's device image. Nothing here calls cudaMalloc,
 // cudaFree or an allocating library routine.
-#include "argus_fuse.cuh"
+#include "argus_internal.cuh"
 
-int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
-                        uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
-                        uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
-                        uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
-                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out);
 
 namespace {
 

@@ -6,42 +6,7 @@
 // (aggregate and select while the interval is in registers: the interval array is never read back) remain
 // for calls that ask for overlap without tables and as a tuning choice (argus_set_synthesize_mode). More than 400
 // regions or 128 pairs: the three plain calls. Results are identical in every mode.
-#include "argus_fuse.cuh"
-
-int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
-                        uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
-                        uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
-                        uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
-                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out);
-int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
-                             const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                             uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                             argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
-                             argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
-                             bool reset_status);
-int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                              argus_agg_t* warp_tab, argus_agg_t* cta_work, bool want_cta, argus_agg_t* sm_tab,
-                              argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream);
-int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
-                           uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,
-                           const uint32_t* pairs, uint32_t num_pairs, argus_overlap_t* out, argus_status_t* status,
-                           void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status);
-int argus_internal_overlap_from_list(const void* list_spans, const uint32_t* list_seg, const uint64_t* list_count,
-                                     uint64_t list_capacity, uint32_t num_sms, uint32_t num_pairs, argus_overlap_t* out,
-                                     argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
-int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
-                                    const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                                    uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                                    const argus_scope_t* scope, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
-                                    argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
-                                    argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
-                                    size_t workspace_bytes, void* cuda_stream, bool reset_status,
-                                    const ArgusFuseArgs* ov_select);
-bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs);
-bool argus_pair_tiled_can_fuse(uint32_t num_regions);
-bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs);
+#include "argus_internal.cuh"
 
 namespace {
 
