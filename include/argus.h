@@ -137,7 +137,8 @@ typedef struct {
   uint64_t n_ctx_mismatch;
   uint64_t n_time_reversed;
   uint64_t n_child_clamped;
-  uint64_t n_sequential_tiles; /* diagnostic: tiles the tiled kernel redid with the sequential stack */
+  uint64_t n_sequential_tiles; /* diagnostic: times the tiled kernel handed markers of a tile that is not
+                                  well nested to the sequential stack machine (0 for well-formed traces) */
 } argus_status_t;
 
 /* ---------------------------------------------------------------------------------------
@@ -182,8 +183,9 @@ int argus_pair_intervals(const argus_event_t* events /*device*/, uint64_t num_ev
 
 /* Same operation with an explicit kernel choice, for tests and profiling:
  * kernel_choice 0 = automatic, 1 = one thread per stream (sequential stack, any input),
- * 2 = tiled kernel (one CTA walks a stream tile by tile; falls back to the sequential stack
- * inside tiles that are not well-nested). All choices produce identical output. */
+ * 2 = tiled kernel (CTAs walk streams tile by tile, long streams a chunk at a time, and hand
+ * the markers that break the nesting to the sequential stack). All choices produce identical
+ * output. */
 int argus_pair_intervals_ex(const argus_event_t* events /*device*/, uint64_t num_events,
                             const uint64_t* stream_offsets /*device [S+1]*/,
                             uint32_t num_streams, uint32_t num_regions,
@@ -201,8 +203,8 @@ int argus_pair_intervals_ex(const argus_event_t* events /*device*/, uint64_t num
  * Some callers run where cudaMalloc is off limits: inside a profiler or tool callback, in a
  * process whose memory pool is owned by another component, or on a path that must not touch
  * the allocator because an allocation could synchronise the device or fail late. This entry
- * point needs no workspace argument: its scratch (control block, per-stream counters, event
- * bitmap and its prefix tables, ambiguity notes) lives in a fixed array inside the library's
+ * point needs no workspace argument: its scratch (control block, per-stream counters, work
+ * queue, event bitmap and its prefix tables, ambiguity notes) lives in a fixed array inside the library's
  * device image, about 1 MB per GPU that loads the library, held until the process exits.
  * Inputs and outputs are still the caller's buffers. The call makes no cudaMalloc, cudaFree
  * or other allocating call.
