@@ -134,29 +134,36 @@ struct TileSmem {
   u32 hot[2];                      // fused aggregation: the two regions whose count and sums threads keep in registers
 };
 
-// Latest begin of the tile at level L and position < pos; -1 if there is none.
+// Latest begin of the tile at level L and position < pos (pos <= T); -1 if there is none. Written without
+// branches: the lanes of a warp would otherwise split over "same word", "earlier word" and "not in this tile"
+// and run all three paths one after the other.
 template <int NT, int E>
 __device__ __forceinline__ int tile_latest_begin(const TileSmem<NT, E>& sm, int L, int lbase, int pos) {
   constexpr int NWORDS = TileSmem<NT, E>::NWORDS;
   const int l = L - lbase;
-  if (l < 0 || l >= kLevelWindow) return -1;
+  const bool valid = (unsigned)l < (unsigned)kLevelWindow;
+  const int lc = valid ? l : 0;
   const int w = pos >> 5;
-  if (w < NWORDS) {
-    const u32 m = sm.bm[l][w] & ((1u << (pos & 31)) - 1u);
-    if (m) return w * 32 + 31 - __clz(m);
-  }
-  int w2;
-  if (NWORDS <= 32) {  // one 32-bit word of the summary covers the tile
-    const u32 s = reinterpret_cast<const u32*>(&sm.summ[l])[0] & ((w >= 32) ? ~0u : ((1u << w) - 1u));
-    if (!s) return -1;
-    w2 = 31 - __clz(s);
+  const bool in_tile = w < NWORDS;               // pos == T: every word lies before it
+  const int wc = in_tile ? w : NWORDS - 1;
+  const u32 below = in_tile ? ((1u << (pos & 31)) - 1u) : 0u;
+  const u32 m = sm.bm[lc][wc] & below;           // begins of the level in the same word, before pos
+  int w2;                                        // last earlier word with a begin of the level
+  bool earlier;
+  if (NWORDS <= 32) {                            // one 32-bit word of the summary covers the tile
+    const u32 s = reinterpret_cast<const u32*>(&sm.summ[lc])[0] & ((w >= 32) ? ~0u : ((1u << w) - 1u));
+    earlier = s != 0;
+    w2 = earlier ? 31 - __clz(s) : 0;
   } else {
-    const u64 s = sm.summ[l] & ((w >= 64) ? ~0ull : ((1ull << w) - 1ull));
-    if (!s) return -1;
-    w2 = 63 - __clzll((long long)s);
+    const u64 s = sm.summ[lc] & ((w >= 64) ? ~0ull : ((1ull << w) - 1ull));
+    earlier = s != 0;
+    w2 = earlier ? 63 - __clzll((long long)s) : 0;
   }
-  const u32 m2 = sm.bm[l][w2];
-  return m2 ? w2 * 32 + 31 - __clz(m2) : -1;
+  const u32 m2 = sm.bm[lc][w2];
+  const int same = wc * 32 + 31 - __clz(m);
+  const int prev = w2 * 32 + 31 - __clz(m2);
+  const int r = m ? same : ((earlier && m2) ? prev : -1);
+  return valid ? r : -1;
 }
 
 constexpr u32 kOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
@@ -396,17 +403,12 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               const u32 d = sm.desc[rk];
               const int e = (int)(d & 0xffffu), L = (int)(d >> 16);
               if (e >= first_bad) continue;
-              int partner = tile_latest_begin<NT, E>(sm, L, lbase, e);
-              int parent;
-              if (partner < 0) {  // opened before this window: so was its parent
-                partner = L < ch ? cbase + L : kBadRef;
-                parent = L == 0 ? cbase + kSink : cbase + L - 1;
-              } else if (L == 0) {
-                parent = cbase + kSink;
-              } else {
-                parent = tile_latest_begin<NT, E>(sm, L - 1, lbase, partner);
-                if (parent < 0) parent = L - 1 < ch ? cbase + L - 1 : kBadRef;
-              }
+              // in the tile, or opened before this window (then so was its parent); selects, not branches
+              const int p_in = tile_latest_begin<NT, E>(sm, L, lbase, e);
+              const bool p_car = p_in < 0;
+              const int q_in = tile_latest_begin<NT, E>(sm, L - 1, lbase, p_car ? 0 : p_in);
+              const int partner = p_car ? (L < ch ? cbase + L : kBadRef) : p_in;
+              const int parent = L == 0 ? cbase + kSink : (q_in >= 0 ? q_in : (L - 1 < ch ? cbase + L - 1 : kBadRef));
               if (partner == kBadRef || parent == kBadRef) { atomicMin(&sm.badpos, e); continue; }
               const uint4 ee = evb[e];
               const uint4 pe = evb[partner];
