@@ -366,25 +366,22 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           int h = h0, rank = (int)(ex >> 16);
           bool seen = false;  // this thread already reported a violation: later markers only keep `desc` complete
 #pragma unroll
-          for (int k = 0; k < E; ++k) {
-            if (tags[k] == 0xffffffffu) continue;
+          for (int k = 0; k < E; ++k) {  // flat, so that begins and ends of a warp are handled by predication, not by two passes
             const int e = w0 + tid * E + k;
+            const bool valid = tags[k] != 0xffffffffu;
+            const bool is_e = valid && (tags[k] & 1u), is_b = valid && !(tags[k] & 1u);
+            const int he = h - 1;            // level of the frame an end closes
+            const int l = h - lbase;         // level of the frame a begin opens, inside the window
             // the parallel rules: known region id, height never negative, at most 64 frames, begins inside the level window
-            bool viol = (tags[k] >> 1) >= a.num_regions;
-            if (tags[k] & 1u) {
-              --h;
-              if (h < 0) viol = true;
-              if (rank < MAXI) sm.desc[rank] = (u32)e | ((u32)(h & 0xff) << 16);
-              ++rank;
-            } else {
-              const int l = h - lbase;
-              if (l < 0 || l >= kLevelWindow || h >= ARGUS_MAX_DEPTH) viol = true;
-              if (!viol && !seen) {
-                atomicOr(&sm.bm[l][e >> 5], 1u << (e & 31));
-                atomicOr(reinterpret_cast<u32*>(&sm.summ[l]) + (e >> 10), 1u << ((e >> 5) & 31));
-              }
-              ++h;
+            const bool viol = (valid && (tags[k] >> 1) >= a.num_regions) || (is_e && he < 0) ||
+                              (is_b && ((unsigned)l >= (unsigned)kLevelWindow || h >= ARGUS_MAX_DEPTH));
+            if (is_e && rank < MAXI) sm.desc[rank] = (u32)e | ((u32)(he & 0xff) << 16);
+            if (is_b && !viol && !seen) {
+              atomicOr(&sm.bm[l][e >> 5], 1u << (e & 31));
+              atomicOr(reinterpret_cast<u32*>(&sm.summ[l]) + (e >> 10), 1u << ((e >> 5) & 31));
             }
+            rank += is_e ? 1 : 0;
+            h += is_b ? 1 : (is_e ? -1 : 0);
             if (viol && !seen) { atomicMin(&sm.badpos, e); seen = true; }
           }
         }
