@@ -400,6 +400,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               const u32 d = sm.desc[rk];
               const int e = (int)(d & 0xffffu), L = (int)(d >> 16);
               if (e >= first_bad) continue;
+              const uint4 ee = evb[e];  // needed after the lookups; asked for now, so that it arrives meanwhile
               // in the tile, or opened before this window (then so was its parent); selects, not branches
               const int p_in = tile_latest_begin<NT, E>(sm, L, lbase, e);
               const bool p_car = p_in < 0;
@@ -407,7 +408,6 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               const int partner = p_car ? (L < ch ? cbase + L : kBadRef) : p_in;
               const int parent = L == 0 ? cbase + kSink : (q_in >= 0 ? q_in : (L - 1 < ch ? cbase + L - 1 : kBadRef));
               if (partner == kBadRef || parent == kBadRef) { atomicMin(&sm.badpos, e); continue; }
-              const uint4 ee = evb[e];
               const uint4 pe = evb[partner];
               if ((pe.z >> 1) != (ee.z >> 1)) { atomicMin(&sm.badpos, e); continue; }
               const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
