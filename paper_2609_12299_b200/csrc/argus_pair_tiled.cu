@@ -402,9 +402,11 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               if (e >= first_bad) continue;
               const uint4 ee = evb[e];  // needed after the lookups; asked for now, so that it arrives meanwhile
               // in the tile, or opened before this window (then so was its parent); selects, not branches
+              // (no begin of level L - 1 can lie between the partner and e while the partner's frame is open, so the
+              // parent is also the latest begin of level L - 1 before e: the two lookups do not depend on each other)
               const int p_in = tile_latest_begin<NT, E>(sm, L, lbase, e);
               const bool p_car = p_in < 0;
-              const int q_in = tile_latest_begin<NT, E>(sm, L - 1, lbase, p_car ? 0 : p_in);
+              const int q_in = tile_latest_begin<NT, E>(sm, L - 1, lbase, e);
               const int partner = p_car ? (L < ch ? cbase + L : kBadRef) : p_in;
               const int parent = L == 0 ? cbase + kSink : (q_in >= 0 ? q_in : (L - 1 < ch ? cbase + L - 1 : kBadRef));
               if (partner == kBadRef || parent == kBadRef) { atomicMin(&sm.badpos, e); continue; }
