@@ -50,6 +50,7 @@ struct AggArgs {
   int iter_inline;    // global path taken inside k_agg_streams_compact (one read of the intervals serves both)
   // overlap span selection in the same pass over the intervals (argus_synthesize); ov.ov_spans null = off
   ArgusFuseArgs ov;
+  const u64* digest;  // digests of the intervals (k_agg_streams_digest), null = read the records
 };
 
 constexpr u32 kAggOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
@@ -252,6 +253,266 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
   }
 }
 
+// ---- the pass over the intervals' 8-byte digests (what argus_synthesize's pairing wrote beside the records) ----
+// One CTA per stream, no scope. The stream's row is gathered in shared memory as 32-bit words, one array per
+// field (field f of region r at word f * R + r, so the lanes of a warp that hold different regions hit different
+// banks). A few regions usually own most intervals of a stream, and 32 lanes adding to one address serialise;
+// so after a probe of the stream's first intervals the kDigestHot most frequent regions get 32 copies of their
+// cell, one per lane (field f of copy l at word f * 32 + l: bank = lane, never a conflict), which are folded into
+// the region's cell when the stream ends. One word per region (meta) holds what a lane needs to know about its
+// region: histogram window base, copy slot, whether the region appears in an overlap pair. A digest marked
+// wide (a duration of 2^23 ticks or more) sends its lane to the record and to 64-bit atomics on the global row.
+// Overlap candidates take their start time from the record.
+constexpr u32 kDigestHot = 4;
+constexpr u32 kDgSumInclLo = 0, kDgSumInclHi = 1, kDgSumExclLo = 2, kDgSumExclHi = 3, kDgMin = 4, kDgMax = 5, kDgFlag = 6,
+              kDgCountOut = 7, kDgBins = 8, kDgMeta = kDgBins + kAggWindow, kDgFields = kDgMeta + 1;
+constexpr u32 kDgHotFields = kDgMeta;          // a copy has no meta word
+constexpr u32 kDgNone = 0xffu;                 // meta: bits 0-7 window base, 8-15 copy slot (kDgNone = unset), bit 16 in a pair
+constexpr u32 kDigestProbe = 1024;             // intervals looked at before the hot regions are chosen
+constexpr u32 kDigestMinStream = 8192;         // shorter streams are gathered without copies
+
+__host__ __device__ constexpr size_t digest_table_words(u32 R) { return (size_t)kDgFields * R + (size_t)kDigestHot * kDgHotFields * 32; }
+
+// The histogram bin of an interval whose bin is not inside the region's window as the lane saw it: the window
+// may not be chosen yet (then this lane tries to), or the bin really lies outside (then it is counted here).
+// Returns the bin's place in the window, or kAggWindow and beyond when it has been dealt with.
+__device__ __noinline__ u32 digest_bin_rare(u32* meta_word, u32 bin, u32* base, u32 stride, u64* row_bins) {
+  const u32 m = *reinterpret_cast<volatile u32*>(meta_word);
+  u32 hb = m & 0xffu;
+  if (hb == kDgNone) {
+    const u32 want = bin > 6u ? bin - 6u : 0u;   // bin <= 22: the window never passes bin 63
+    const u32 prev = atomicCAS(meta_word, m, (m & ~0xffu) | want);  // only the window base changes while intervals are added
+    hb = (prev & 0xffu) == kDgNone ? want : (prev & 0xffu);
+  }
+  const u32 rel = bin - hb;
+  if (rel < kAggWindow) return rel;
+  atomicAdd(base + kDgCountOut * stride, 1u);
+  atomicAdd(row_bins + bin, 1ull);
+  return 0xffffffffu;
+}
+
+__global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
+  extern __shared__ __align__(16) unsigned char sh_raw[];
+  u32* const cold = reinterpret_cast<u32*>(sh_raw);
+  const u32 R = a.num_regions;
+  u32* const hot = cold + (size_t)kDgFields * R;
+  u32* const pairbits = hot + kDigestHot * kDgHotFields * 32;
+  u32* const pairs_sm = pairbits + (R + 31) / 32;
+  __shared__ u32 hot_region[kDigestHot];
+  const u32 cells = R * kCell;
+  const u32 lane = threadIdx.x & 31;
+  const bool has_ov = a.ov.ov_spans != nullptr && a.ov.num_pairs != 0;
+  u64 ovc_base = 0;
+  u32 ovc_used = kAggOvChunk;
+  for (u32 i = threadIdx.x; i < (R + 31) / 32; i += blockDim.x) pairbits[i] = 0;
+  __syncthreads();
+  if (has_ov) {
+    for (u32 i = threadIdx.x; i < 2 * a.ov.num_pairs; i += blockDim.x) {
+      const u32 r = a.ov.pairs[i];
+      pairs_sm[i] = r;
+      if (r < R) atomicOr(&pairbits[r >> 5], 1u << (r & 31));
+    }
+    __syncthreads();
+  }
+  for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
+    u64* row = a.warp_tab + (size_t)s * cells;
+    for (u32 i = threadIdx.x; i < cells; i += blockDim.x) row[i] = (i % kCell == 2) ? ~0ull : 0ull;
+    for (u32 i = threadIdx.x; i < kDgMeta * R; i += blockDim.x) cold[i] = (i / R == kDgMin) ? 0xffffffffu : 0u;
+    for (u32 r = threadIdx.x; r < R; r += blockDim.x)
+      cold[kDgMeta * R + r] = kDgNone | (kDgNone << 8) | (((pairbits[r >> 5] >> (r & 31)) & 1u) << 16);
+    for (u32 i = threadIdx.x; i < kDigestHot * kDgHotFields * 32; i += blockDim.x)
+      hot[i] = ((i >> 5) % kDgHotFields == kDgMin) ? 0xffffffffu : 0u;
+    if (threadIdx.x < kDigestHot) hot_region[threadIdx.x] = 0xffffffffu;
+    __threadfence();
+    __syncthreads();
+    const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
+    u32 sm_index = 0;
+    if (has_ov) {
+      const u32 m = a.cta_sm[s / a.warps_per_cta];
+      if (m >= a.num_sms && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
+      sm_index = m < a.num_sms ? m : 0;
+    }
+    if (hi < lo || ((hi - lo) >> 32)) {
+      if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
+    } else {
+      const u32 n = (u32)(hi - lo);
+      const u64* const dgs = a.digest + lo;
+      const argus_interval_t* const ivs = a.intervals + lo;
+      // two legs: the probe (every cell in the region arrays), then, hot regions chosen, the rest of the stream
+      const u32 probe_end = n >= kDigestMinStream ? kDigestProbe : n;
+      for (int leg = 0; leg < 2; ++leg) {
+        const u32 leg_lo = leg ? probe_end : 0u, leg_hi = leg ? n : probe_end;
+        if (leg && leg_lo < leg_hi) {
+          // warp 0 ranks the regions by their counts so far; kDigestHot rounds of a warp-wide maximum
+          if (threadIdx.x < 32) {
+            for (u32 h = 0; h < kDigestHot; ++h) {
+              u32 best = 0;
+              for (u32 r = lane; r < R; r += 32) {
+                if (((cold[kDgMeta * R + r] >> 8) & 0xffu) != kDgNone) continue;
+                u32 cnt = cold[kDgCountOut * R + r];
+#pragma unroll
+                for (u32 j = 0; j < kAggWindow; ++j) cnt += cold[(kDgBins + j) * R + r];
+                const u32 key = ((cnt > 0xffffu ? 0xffffu : cnt) << 16) | r;
+                best = key > best ? key : best;
+              }
+              const u32 top = __reduce_max_sync(0xffffffffu, best);
+              if ((top >> 16) < kDigestProbe / 64) break;  // not worth a set of copies
+              if (lane == 0) { atomicAnd(&cold[kDgMeta * R + (top & 0xffffu)], ~0xff00u | (h << 8)); hot_region[h] = top & 0xffffu; }
+              __syncwarp();
+            }
+          }
+          __syncthreads();
+        }
+        // every lane of a warp runs the same number of rounds, so that spans can be appended a warp at a time
+        u32 b = leg_lo + (threadIdx.x & ~31u);
+        u64 dg_next = b + lane < leg_hi ? __ldg(dgs + b + lane) : 0ull;
+        for (; b < leg_hi; b += kAggThreads) {
+          const u32 i = b + lane;
+          const u64 dg = dg_next;
+          dg_next = i + kAggThreads < leg_hi ? __ldg(dgs + i + kAggThreads) : 0ull;
+          const u32 dlo = (u32)dg, dhi = (u32)(dg >> 32);
+          const bool in = i < leg_hi;
+          const u32 region = dlo & 0xffffu;
+          const bool ok = in && region < R;
+          const u32 rsafe = ok ? region : 0u;
+          const u32 incl = (dlo >> 18) | ((dhi & 0x1ffu) << 14), excl = dhi >> 9;
+          const u32 meta = cold[kDgMeta * R + rsafe];
+          const u32 slot = (meta >> 8) & 0xffu;
+          u32* const base = slot != kDgNone ? hot + slot * (kDgHotFields * 32) + lane : cold + rsafe;
+          const u32 stride = slot != kDgNone ? 32u : R;
+          // the common case without a branch: a lane that does not take part (past the end, wide, bad region)
+          // adds nothing; whatever is rare (a carry, a flag, a bin outside the window, ...) is settled in one place
+          const bool take = ok && !(dlo & (1u << 17));
+          const u32 vi = take ? incl : 0u, ve = take ? excl : 0u;
+          const u32 old_i = atomicAdd(base + kDgSumInclLo * stride, vi);
+          const u32 old_e = atomicAdd(base + kDgSumExclLo * stride, ve);
+          atomicMin(base + kDgMin * stride, take ? incl : 0xffffffffu);
+          atomicMax(base + kDgMax * stride, vi);
+          const u32 bin = 31u - (u32)__clz((int)(incl | 1u));
+          const u32 rel = bin - (meta & 0xffu);
+          const bool in_win = take && rel < kAggWindow;
+          atomicAdd(base + (kDgBins + (in_win ? rel : 0u)) * stride, in_win ? 1u : 0u);
+          u64 span = vi;
+          const bool rare = in && ((dlo & (3u << 16)) || !ok || old_i + vi < old_i || old_e + ve < old_e || !in_win);
+          if (rare) {
+            if (!ok) {
+              argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, lo + i);
+            } else if (!take) {
+              u64* const row_cell = row + (size_t)region * kCell;
+              const uint4* p = reinterpret_cast<const uint4*>(ivs + i);
+              const uint4 q0 = __ldg(p), q1 = __ldg(p + 1);
+              span = (u64)q0.z | ((u64)q0.w << 32);
+              atomicAdd(row_cell + 0, 1ull);
+              atomicAdd(row_cell + 1, span);
+              atomicMin(row_cell + 2, span);
+              atomicMax(row_cell + 3, span);
+              atomicAdd(row_cell + 4, (u64)q1.x | ((u64)q1.y << 32));
+              if (dlo & (1u << 16)) atomicAdd(row_cell + 7, 1ull);
+              atomicAdd(row_cell + 8 + log2_bin(span), 1ull);
+            } else {
+              if (old_i + vi < old_i) atomicAdd(base + kDgSumInclHi * stride, 1u);
+              if (old_e + ve < old_e) atomicAdd(base + kDgSumExclHi * stride, 1u);
+              if (dlo & (1u << 16)) atomicAdd(base + kDgFlag * stride, 1u);
+              if (!in_win) {
+                const u32 r2 = digest_bin_rare(cold + kDgMeta * R + region, bin, base, stride, row + (size_t)region * kCell + 8);
+                if (r2 < kAggWindow) atomicAdd(base + (kDgBins + r2) * stride, 1u);
+              }
+            }
+          }
+          const bool cand = ok && ((meta >> 16) & 1u) && span;
+          if (has_ov && __ballot_sync(0xffffffffu, cand)) {
+            u64 t0 = 0;
+            if (cand) t0 = __ldg(reinterpret_cast<const u64*>(ivs + i));
+            for (u32 k = 0; k < 2 * a.ov.num_pairs; ++k) {
+              const bool pick = cand && pairs_sm[k] == region;
+              const u32 bal = __ballot_sync(0xffffffffu, pick);
+              if (!bal) continue;
+              const u32 c = __popc(bal);
+              if (ovc_used + c > kAggOvChunk) {
+                u64 nb64 = 0;
+                if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)kAggOvChunk);
+                ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
+                ovc_used = 0;
+              }
+              if (pick) {
+                const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
+                if (slot < a.ov.ov_capacity) {
+                  a.ov.ov_spans[slot] = make_ulonglong2(t0, t0 + span);
+                  a.ov.ov_seg[slot] = ((k >> 1) * a.num_sms + sm_index) * 2 + (k & 1u);
+                }
+              }
+              ovc_used += c;
+            }
+          }
+        }
+        __syncthreads();
+      }
+    }
+    if (a.ambig && a.ambig_offsets) {
+      const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
+      for (u64 i = alo + threadIdx.x; i < ahi && ahi >= alo; i += blockDim.x) {
+        const u32 region = a.ambig[i].tag >> 1;
+        if (region >= R) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
+        atomicAdd(row + (size_t)region * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
+      }
+    }
+    __syncthreads();
+    // fold the lanes' copies into their region's cell: one thread per (hot region, field), lanes taken in a
+    // rotated order so that the threads of a warp read different banks
+    if (threadIdx.x < kDigestHot * kDgHotFields) {
+      const u32 h = threadIdx.x / kDgHotFields, f = threadIdx.x % kDgHotFields;
+      const u32 r = hot_region[h];
+      if (r != 0xffffffffu && f != kDgSumInclHi && f != kDgSumExclHi) {
+        const u32* src = hot + (h * kDgHotFields + f) * 32;
+        if (f == kDgSumInclLo || f == kDgSumExclLo) {
+          u64 sum = (u64)cold[f * R + r] | ((u64)cold[(f + 1) * R + r] << 32);
+          for (u32 l = 0; l < 32; ++l) {
+            const u32 ll = (l + threadIdx.x) & 31u;
+            sum += (u64)src[ll] | ((u64)src[32 + ll] << 32);
+          }
+          cold[f * R + r] = (u32)sum;
+          cold[(f + 1) * R + r] = (u32)(sum >> 32);
+        } else {
+          u32 acc = cold[f * R + r];
+          for (u32 l = 0; l < 32; ++l) {
+            const u32 v = src[(l + threadIdx.x) & 31u];
+            acc = f == kDgMin ? (v < acc ? v : acc) : f == kDgMax ? (v > acc ? v : acc) : acc + v;
+          }
+          cold[f * R + r] = acc;
+        }
+      }
+    }
+    __syncthreads();
+    // the region arrays into the global row, which already holds the wide intervals, the bins outside the
+    // windows and the ambiguity counters: everything is combined, nothing overwritten
+    constexpr u32 kItems = 6 + kAggWindow;
+    for (u32 i = threadIdx.x; i < R * kItems; i += blockDim.x) {
+      const u32 r = i % R, f = i / R;
+      u64* cell = row + (size_t)r * kCell;
+      switch (f) {
+        case 0: {
+          u64 n = cold[kDgCountOut * R + r];
+#pragma unroll
+          for (u32 j = 0; j < kAggWindow; ++j) n += cold[(kDgBins + j) * R + r];
+          if (n) atomicAdd(cell + 0, n);
+          break;
+        }
+        case 1: { const u64 v = (u64)cold[kDgSumInclLo * R + r] | ((u64)cold[kDgSumInclHi * R + r] << 32); if (v) atomicAdd(cell + 1, v); break; }
+        case 2: { const u32 v = cold[kDgMin * R + r]; if (v != 0xffffffffu) atomicMin(cell + 2, (u64)v); break; }
+        case 3: { const u32 v = cold[kDgMax * R + r]; if (v) atomicMax(cell + 3, (u64)v); break; }
+        case 4: { const u64 v = (u64)cold[kDgSumExclLo * R + r] | ((u64)cold[kDgSumExclHi * R + r] << 32); if (v) atomicAdd(cell + 4, v); break; }
+        case 5: { const u32 v = cold[kDgFlag * R + r]; if (v) atomicAdd(cell + 7, (u64)v); break; }
+        default: {
+          const u32 j = f - 6;
+          const u32 v = cold[(kDgBins + j) * R + r];
+          if (v) atomicAdd(cell + 8 + (cold[kDgMeta * R + r] & 0xffu) + j, (u64)v);
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
 __device__ __forceinline__ u64 combine(u32 field, u64 x, u64 y) {
   return field == 2 ? (x < y ? x : y) : field == 3 ? (x > y ? x : y) : x + y;
 }
@@ -444,7 +705,7 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
   a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
   a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0; a.iter_copies = nullptr; a.num_copies = 0;
   a.iter_inline = 0;
-  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0;
+  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.digest = nullptr;
   if (ambig && ambig_offsets) {
     k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
     ARGUS_CHECK_LAUNCH();
@@ -463,7 +724,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
                                     argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
                                     argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
                                     size_t workspace_bytes, void* cuda_stream, bool reset_status,
-                                    const ArgusFuseArgs* ov_select) {
+                                    const ArgusFuseArgs* ov_select, const uint64_t* digest) {
   if (!interval_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if (ov_select && (num_regions > kAggCompactRegions || ov_select->num_pairs > kFuseMaxPairs)) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
@@ -499,6 +760,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   a.sm_mask = scope ? scope->sm_mask : nullptr; a.region_mask = scope ? scope->region_mask : nullptr;
   a.role_tab = (u64*)role_tab; a.iter_tab = (u64*)iter_tab; a.num_iters = num_iters;
   if (ov_select) { a.ov = *ov_select; } else { a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; }
+  a.digest = !scope && !role_tab && !iter_tab && num_regions <= kAggCompactRegions ? (const u64*)digest : nullptr;
   const size_t smem = (size_t)num_regions * sizeof(argus_agg_t);
   a.use_smem = smem <= kAggSmemLimit;
   const size_t iter_bytes = (size_t)num_iters * smem;
@@ -528,7 +790,14 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
     const size_t compact = (size_t)num_regions * sizeof(ArgusAggCell) + ((num_regions + 31) / 32) * 4 + (size_t)a.ov.num_pairs * 8;
     if (compact > 48 * 1024)
       ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams_compact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compact));
-    k_agg_streams_compact<<<num_streams, kAggThreads, compact, stream>>>(a);
+    if (a.digest) {
+      const size_t dg = digest_table_words(num_regions) * 4 + ((num_regions + 31) / 32) * 4 + (size_t)a.ov.num_pairs * 8;
+      if (dg > 48 * 1024)
+        ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams_digest, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dg));
+      k_agg_streams_digest<<<num_streams, kAggThreads, dg, stream>>>(a);
+    } else {
+      k_agg_streams_compact<<<num_streams, kAggThreads, compact, stream>>>(a);
+    }
   } else {
     k_agg_streams<<<num_streams, kAggThreads, need, stream>>>(a);
   }

@@ -43,6 +43,19 @@ struct ArgusFuseCtx {     // per CTA, for the stream it is walking
   u32 sm_index;           // SM of this stream's CTA
 };
 
+// Digest of an interval (8 bytes): all that aggregation needs of it. argus_synthesize lets the pairing kernels
+// write one per interval record, at the same position, so that the aggregation pass reads 8 bytes per interval
+// instead of 48. Bits 0-15 region, 16 any flag set, 17 wide (a duration does not fit: take both from the
+// record; the duration bits then mean nothing), 18-40 inclusive, 41-63 exclusive duration.
+constexpr u32 kDigestBits = 23;
+__device__ __forceinline__ u64 argus_digest_pack(u32 region, u64 incl, u64 excl, u32 flags) {
+  const u32 il = (u32)incl, el = (u32)excl;
+  const bool wide = (((il | el) >> kDigestBits) | (u32)(incl >> 32) | (u32)(excl >> 32)) != 0;
+  const u32 lo = region | (flags ? 1u << 16 : 0u) | (wide ? 1u << 17 : 0u) | (il << 18);
+  const u32 hi = ((il >> 14) & 0x1ffu) | (el << 9);
+  return (u64)lo | ((u64)hi << 32);
+}
+
 __device__ __forceinline__ u32 argus_log2_bin(u64 d) { return d ? 63u - (u32)__clzll((long long)d) : 0u; }
 
 // 64-bit add as native 32-bit atomics; each carry is propagated exactly once

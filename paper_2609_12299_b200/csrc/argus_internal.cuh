@@ -6,12 +6,13 @@
 
 // argus_pair.cu — the whole pairing pipeline. kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled.
 // `fuse` (nullable) asks the tiled kernel to feed aggregation / overlap selection; *fused_out tells whether it did.
+// `digest` (nullable): one 8-byte digest per interval record, at the record's position (see argus_fuse.cuh).
 int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
                         uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
                         uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
                         uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
                         size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out);
+                        bool reset_status, bool* fused_out, uint64_t* digest = nullptr, uint64_t digest_capacity = 0);
 
 // argus_pair_tiled.cu
 bool argus_pair_tiled_can_fuse(uint32_t num_regions);
@@ -24,7 +25,8 @@ int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* 
                              argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
                              argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
                              bool reset_status);
-// scope, role_tab, iter_tab nullable; ov_select (nullable): also append the overlap spans of the selected intervals
+// scope, role_tab, iter_tab nullable; ov_select (nullable): also append the overlap spans of the selected intervals;
+// digest (nullable; needs no scope, no role or iteration table, at most 400 regions): the intervals' digests, read instead of the records
 int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
                                     const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
                                     uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
@@ -32,7 +34,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
                                     argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
                                     argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
                                     size_t workspace_bytes, void* cuda_stream, bool reset_status,
-                                    const ArgusFuseArgs* ov_select);
+                                    const ArgusFuseArgs* ov_select, const uint64_t* digest = nullptr);
 // second half of aggregation when the pairing kernel already filled the interval statistics of warp_tab
 int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
                               uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,

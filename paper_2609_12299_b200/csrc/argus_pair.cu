@@ -220,7 +220,7 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
                         uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
                         uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
                         size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out) {
+                        bool reset_status, bool* fused_out, uint64_t* digest, uint64_t digest_capacity) {
   if (!stream_offsets || !interval_offsets || !ambig_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if ((num_events && !events) || (interval_capacity && !intervals) || (ambig_capacity && !ambig)) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
@@ -247,6 +247,8 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   a.queue = (u32*)(ws + L.queue); a.queue_capacity = L.queue_capacity;
   a.records = (ArgusStreamRecord*)(ws + L.records); a.record_capacity = L.record_capacity;
   memset(&a.fuse, 0, sizeof(a.fuse));
+  // a stream's intervals start at half its first event's position at the latest, so positions stay below num_events / 2 + 1
+  a.digest = digest_capacity >= (interval_capacity < num_events / 2 + 1 ? interval_capacity : num_events / 2 + 1) ? (u64*)digest : nullptr;
 
   if (reset_status) ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
   // control block, counts and bitmap are contiguous at the start of the workspace

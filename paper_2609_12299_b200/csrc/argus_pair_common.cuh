@@ -74,6 +74,8 @@ struct ArgusPairArgs {
   u64 queue_capacity;
   ArgusStreamRecord* records;
   u32 record_capacity;
+  u64* digest;            // one digest per interval record, same positions (null = none); holds every position below
+                          // min(interval_capacity, num_events / 2 + 1), which is all a stream can reach
   ArgusFuseArgs fuse;     // optional aggregation / overlap selection fed from the pairing kernel (first pass only)
 };
 
@@ -143,6 +145,7 @@ __device__ __forceinline__ bool argus_seq_step(const ArgusPairArgs& a, ArgusFram
   if (pos < a.interval_capacity) {
     argus_store_interval(a.intervals + pos, f.ts, incl, excl, f.region, f.ctx, stream,
                          s.h > 0 ? stk[s.h - 1].region : ARGUS_NONE, f.idx, (u32)s.h, flags);
+    if (a.digest) a.digest[pos] = argus_digest_pack(f.region, incl, excl, flags);
   } else if (!a.redo) {
     a.ctl->spec_overflow = 1;
   }

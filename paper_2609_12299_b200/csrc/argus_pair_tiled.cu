@@ -461,6 +461,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
                 q[0] = make_uint4(pe.x, pe.y, (u32)incl, (u32)(incl >> 32));
                 q[1] = make_uint4((u32)excl, (u32)(excl >> 32), pe.z >> 1, pe.w);
                 q[2] = make_uint4(s, preg, bidx, (d >> 16) | (flags << 16));
+                if (a.digest) a.digest[pos] = argus_digest_pack(pe.z >> 1, incl, excl, flags);
               } else if (!a.redo) {
                 a.ctl->spec_overflow = 1;
               }

@@ -1,8 +1,9 @@
 // argus_synthesize.cu — the whole hot path in one call: pair -> aggregate -> overlap.
 //
-// Pairing runs plain, then ONE pass over the intervals both aggregates them and selects the overlap spans;
-// that pass runs at HBM speed, while hosting the table in the pairing kernel (which is bound by instruction
-// issue and occupancy, not by HBM) measured slower on every trace shape. The pairing kernel's own hooks
+// Pairing runs plain and writes, beside every 48-byte interval record, an 8-byte digest (region, both
+// durations, a flag bit); then ONE pass over the digests both aggregates the intervals and selects the overlap
+// spans. Hosting the table in the pairing kernel (which is bound by instruction issue and occupancy, not by
+// HBM) measured slower on every trace shape, and so did a pass over the records themselves (six times the bytes). The pairing kernel's own hooks
 // (aggregate and select while the interval is in registers: the interval array is never read back) remain
 // for calls that ask for overlap without tables and as a tuning choice (argus_set_synthesize_mode). More than 400
 // regions or 128 pairs: the three plain calls. Results are identical in every mode.
@@ -13,7 +14,8 @@ namespace {
 int g_synth_mode = -1;  // -1 = automatic
 
 struct SynLayout {
-  size_t pair, pair_bytes, agg, agg_bytes, list_count, list_seg, list_spans, ov, ov_bytes, total;
+  size_t pair, pair_bytes, agg, agg_bytes, list_count, list_seg, list_spans, ov, ov_bytes, digest, total;
+  uint64_t digest_capacity;
 };
 
 SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_regions, uint64_t ambig_capacity,
@@ -28,6 +30,9 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
   L.ov = o;
   L.ov_bytes = argus_align_up((size_t)num_pairs * num_sms * 2 * 8 * 3 + 1024 + (size_t)max_overlap_spans * 24 + 256, 256);
   o += L.ov_bytes;
+  // one digest per interval (a stream's intervals start at half its first event's position at the latest)
+  L.digest_capacity = argus_aggregate_can_select_overlap(num_regions, num_pairs) ? num_events / 2 + 1 : 0;
+  L.digest = o; o += argus_align_up((size_t)L.digest_capacity * 8, 256);
   L.total = o;
   return L;
 }
@@ -35,7 +40,8 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
 }  // namespace
 
 // Where argus_synthesize aggregates and selects overlap spans: -1 automatic, 0 inside the pairing kernel,
-// 1 in one pass over the intervals, 2 the plain calls (tuning and test aid; results are identical).
+// 1 in one pass over the intervals' digests, 2 the plain calls, 3 in one pass over the interval records
+// (tuning and test aid; results are identical).
 extern "C" void argus_set_synthesize_mode(int mode) { g_synth_mode = mode; }
 
 extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint32_t num_regions,
@@ -76,7 +82,9 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
   if (num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs)) mode = 1;
   else if (can_fuse) mode = 0;
   if (g_synth_mode == 0 && can_fuse) mode = 0;  // tuning aid: a forced mode applies when the inputs allow it
-  if (g_synth_mode == 1 && num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs)) mode = 1;
+  if ((g_synth_mode == 1 || g_synth_mode == 3) && num_streams > 0 && want_agg &&
+      argus_aggregate_can_select_overlap(num_regions, num_pairs))
+    mode = 1;
   if (g_synth_mode == 2) mode = 2;
   const bool list = mode != 2 && num_pairs;
   if (mode == 0 && want_agg) {
@@ -92,9 +100,11 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
     ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)max_overlap_spans * 4 + 4, stream));
   }
   bool fused = false;
+  const bool use_digest = mode == 1 && L.digest_capacity != 0 && g_synth_mode != 3;
   int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
                                interval_offsets, ambig, ambig_capacity, ambig_offsets, status, ws + L.pair, L.pair_bytes,
-                               cuda_stream, 0, mode == 0 && (f.warp_tab || f.ov_spans) ? &f : nullptr, true, &fused);
+                               cuda_stream, 0, mode == 0 && (f.warp_tab || f.ov_spans) ? &f : nullptr, true, &fused,
+                               use_digest ? (uint64_t*)(ws + L.digest) : nullptr, L.digest_capacity);
   if (rc != ARGUS_OK) return rc;
   if (mode == 0 && !fused) mode = 2;  // the pairing front end chose a kernel without the hooks
 
@@ -106,7 +116,8 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
       rc = argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta,
                                            cta_sm, num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab,
                                            nullptr, nullptr, status, ws + L.agg, L.agg_bytes, cuda_stream, false,
-                                           mode == 1 && list ? &f : nullptr);
+                                           mode == 1 && list ? &f : nullptr,
+                                           use_digest ? (const uint64_t*)(ws + L.digest) : nullptr);
     }
     if (rc != ARGUS_OK) return rc;
   }

@@ -276,7 +276,7 @@ def _synthesize_matches(spec, ev, offs, **kw):
     return res, st
 
 
-@pytest.fixture(params=[-1, 0, 1, 2], ids=["auto", "in-pairing-kernel", "one-pass", "plain-calls"])
+@pytest.fixture(params=[-1, 0, 1, 2, 3], ids=["auto", "in-pairing-kernel", "one-pass-digests", "plain-calls", "one-pass-records"])
 def synth_mode(request):
     """Where argus_synthesize aggregates and selects overlap spans; results must not depend on it."""
     from paper_2609_12299_b200.binding import argus_set_synthesize_mode
@@ -316,6 +316,36 @@ def test_synthesize_wide_histogram_and_flags(synth_mode):
             rows.append((t_end, "E", r, i))
             t += d + int(rng.integers(0, 100))
         ev = make_events(rows)
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    _synthesize_matches(spec, np.concatenate(evs), np.array(offs, np.uint64))
+
+
+def test_synthesize_hot_regions_long_streams(synth_mode):
+    """Streams long enough for the digest pass to give the most frequent regions their per-lane copies: two regions
+    own most intervals; durations just below and above the digest's 23 bits, so that the 32-bit sums of the
+    copies carry, bins fall outside a region's window, and wide digests send lanes to the records."""
+    rng = np.random.default_rng(77)
+    spec = tg.TraceSpec(tg.GEMM, 1, 1)  # only for warps_per_cta / cta_sm / pairs
+    S = spec.num_streams
+    evs, offs = [], [0]
+    for s in range(S):
+        n = 120000 if s % 3 == 0 else 9000
+        region = rng.choice(5, size=n, p=[0.45, 0.4, 0.05, 0.05, 0.05]).astype(np.uint64)
+        kind = rng.random(n)
+        dur = np.where(kind < 0.6, rng.integers(1 << 21, 1 << 23, n),
+                       np.where(kind < 0.9, rng.integers(0, 300, n),
+                                np.where(kind < 0.97, rng.integers(1 << 23, 1 << 36, n), 2 ** rng.integers(0, 23, n)))).astype(np.uint64)
+        gap = rng.integers(0, 50, n).astype(np.uint64)
+        t_begin = (np.uint64(1) << np.uint64(33)) + np.concatenate([[0], np.cumsum(dur + gap)[:-1]]).astype(np.uint64)
+        ev = np.zeros(2 * n, argus.EVENT_DTYPE)
+        ev["ts"][0::2] = t_begin
+        ev["ts"][1::2] = t_begin + dur
+        ev["tag"][0::2] = (region << np.uint64(1)).astype(np.uint32)
+        ev["tag"][1::2] = ((region << np.uint64(1)) | np.uint64(1)).astype(np.uint32)
+        ctx = np.arange(n, dtype=np.uint32)
+        ev["ctx"][0::2] = ctx
+        ev["ctx"][1::2] = ctx + (rng.random(n) < 0.01)  # a few context mismatches: flagged intervals
         evs.append(ev)
         offs.append(offs[-1] + len(ev))
     _synthesize_matches(spec, np.concatenate(evs), np.array(offs, np.uint64))
