@@ -254,29 +254,44 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
 }
 
 // ---- the pass over the intervals' 8-byte digests (what argus_synthesize's pairing wrote beside the records) ----
-// One CTA per stream, no scope. The stream's row is gathered in shared memory as 32-bit words, one array per
-// field (field f of region r at word f * R + r, so the lanes of a warp that hold different regions hit different
-// banks). A few regions usually own most intervals of a stream, and 32 lanes adding to one address serialise;
-// so after a probe of the stream's first intervals the kDigestHot most frequent regions get 32 copies of their
-// cell, one per lane (field f of copy l at word f * 32 + l: bank = lane, never a conflict), which are folded into
-// the region's cell when the stream ends. One word per region (meta) holds what a lane needs to know about its
-// region: histogram window base, copy slot, whether the region appears in an overlap pair. A digest marked
-// wide (a duration of 2^23 ticks or more) sends its lane to the record and to 64-bit atomics on the global row.
-// Overlap candidates take their start time from the record.
+// One CTA per stream, no scope. The stream's row is gathered in shared memory in cells of kDgWords = 25 32-bit
+// words (an odd size: the cells of 32 different regions start in 32 different banks). A few regions usually own
+// most intervals of a stream, and 32 lanes adding to one address serialise; so after a probe of the stream's
+// first intervals the kDigestHot most frequent regions get 32 copies of their cell, one per lane (consecutive
+// cells: never a bank conflict), which are folded into the region's cell when the stream ends. The last word of
+// a region's cell (meta) holds what a lane needs to know about its region: histogram window base, copy slot,
+// whether the region appears in an overlap pair. A digest marked wide (a duration of 2^23 ticks or more) sends
+// its lane to the record and to 64-bit atomics on the global row. Overlap candidates take their start time from
+// the record. The table is addressed with 32-bit shared-memory addresses and the fields by constant offsets.
 constexpr u32 kDigestHot = 4;
 constexpr u32 kDgSumInclLo = 0, kDgSumInclHi = 1, kDgSumExclLo = 2, kDgSumExclHi = 3, kDgMin = 4, kDgMax = 5, kDgFlag = 6,
-              kDgCountOut = 7, kDgBins = 8, kDgMeta = kDgBins + kAggWindow, kDgFields = kDgMeta + 1;
-constexpr u32 kDgHotFields = kDgMeta;          // a copy has no meta word
+              kDgCountOut = 7, kDgBins = 8, kDgMeta = kDgBins + kAggWindow, kDgWords = kDgMeta + 1;
+static_assert(kDgWords % 2 == 1, "an odd cell size keeps the cells of different regions in different banks");
 constexpr u32 kDgNone = 0xffu;                 // meta: bits 0-7 window base, 8-15 copy slot (kDgNone = unset), bit 16 in a pair
-constexpr u32 kDigestProbe = 1024;             // intervals looked at before the hot regions are chosen
-constexpr u32 kDigestMinStream = 8192;         // shorter streams are gathered without copies
+constexpr u32 kDigestProbe = 512;              // intervals looked at before the hot regions are chosen
+constexpr u32 kDigestMinStream = 2048;         // shorter streams are gathered without copies
 
-__host__ __device__ constexpr size_t digest_table_words(u32 R) { return (size_t)kDgFields * R + (size_t)kDigestHot * kDgHotFields * 32; }
+__host__ __device__ constexpr size_t digest_table_words(u32 R) { return (size_t)kDgWords * (R + kDigestHot * 32); }
+
+template <u32 F> __device__ __forceinline__ u32 dg_add(u32 cell, u32 v) {  // returns the old value
+  u32 old;
+  asm volatile("atom.shared.add.u32 %0, [%1+%3], %2;" : "=r"(old) : "r"(cell), "r"(v), "n"(F * 4) : "memory");
+  return old;
+}
+template <u32 F> __device__ __forceinline__ void dg_inc(u32 cell, u32 v) {
+  asm volatile("red.shared.add.u32 [%0+%2], %1;" :: "r"(cell), "r"(v), "n"(F * 4) : "memory");
+}
+template <u32 F> __device__ __forceinline__ void dg_min(u32 cell, u32 v) {
+  asm volatile("red.shared.min.u32 [%0+%2], %1;" :: "r"(cell), "r"(v), "n"(F * 4) : "memory");
+}
+template <u32 F> __device__ __forceinline__ void dg_max(u32 cell, u32 v) {
+  asm volatile("red.shared.max.u32 [%0+%2], %1;" :: "r"(cell), "r"(v), "n"(F * 4) : "memory");
+}
 
 // The histogram bin of an interval whose bin is not inside the region's window as the lane saw it: the window
 // may not be chosen yet (then this lane tries to), or the bin really lies outside (then it is counted here).
 // Returns the bin's place in the window, or kAggWindow and beyond when it has been dealt with.
-__device__ __noinline__ u32 digest_bin_rare(u32* meta_word, u32 bin, u32* base, u32 stride, u64* row_bins) {
+__device__ __noinline__ u32 digest_bin_rare(u32* meta_word, u32 bin, u32 cell, u64* row_bins) {
   const u32 m = *reinterpret_cast<volatile u32*>(meta_word);
   u32 hb = m & 0xffu;
   if (hb == kDgNone) {
@@ -286,19 +301,20 @@ __device__ __noinline__ u32 digest_bin_rare(u32* meta_word, u32 bin, u32* base, 
   }
   const u32 rel = bin - hb;
   if (rel < kAggWindow) return rel;
-  atomicAdd(base + kDgCountOut * stride, 1u);
+  dg_inc<kDgCountOut>(cell, 1u);
   atomicAdd(row_bins + bin, 1ull);
   return 0xffffffffu;
 }
 
 __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
   extern __shared__ __align__(16) unsigned char sh_raw[];
-  u32* const cold = reinterpret_cast<u32*>(sh_raw);
+  u32* const tab = reinterpret_cast<u32*>(sh_raw);
   const u32 R = a.num_regions;
-  u32* const hot = cold + (size_t)kDgFields * R;
-  u32* const pairbits = hot + kDigestHot * kDgHotFields * 32;
+  const u32 num_cells = R + kDigestHot * 32;
+  u32* const pairbits = tab + (size_t)kDgWords * num_cells;
   u32* const pairs_sm = pairbits + (R + 31) / 32;
   __shared__ u32 hot_region[kDigestHot];
+  const u32 tab_addr = (u32)__cvta_generic_to_shared(tab);
   const u32 cells = R * kCell;
   const u32 lane = threadIdx.x & 31;
   const bool has_ov = a.ov.ov_spans != nullptr && a.ov.num_pairs != 0;
@@ -317,11 +333,12 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
   for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
     u64* row = a.warp_tab + (size_t)s * cells;
     for (u32 i = threadIdx.x; i < cells; i += blockDim.x) row[i] = (i % kCell == 2) ? ~0ull : 0ull;
-    for (u32 i = threadIdx.x; i < kDgMeta * R; i += blockDim.x) cold[i] = (i / R == kDgMin) ? 0xffffffffu : 0u;
-    for (u32 r = threadIdx.x; r < R; r += blockDim.x)
-      cold[kDgMeta * R + r] = kDgNone | (kDgNone << 8) | (((pairbits[r >> 5] >> (r & 31)) & 1u) << 16);
-    for (u32 i = threadIdx.x; i < kDigestHot * kDgHotFields * 32; i += blockDim.x)
-      hot[i] = ((i >> 5) % kDgHotFields == kDgMin) ? 0xffffffffu : 0u;
+    for (u32 i = threadIdx.x; i < kDgWords * num_cells; i += blockDim.x) {
+      const u32 f = i % kDgWords, c = i / kDgWords;
+      u32 v = f == kDgMin ? 0xffffffffu : 0u;
+      if (f == kDgMeta && c < R) v = kDgNone | (kDgNone << 8) | (((pairbits[c >> 5] >> (c & 31)) & 1u) << 16);
+      tab[i] = v;
+    }
     if (threadIdx.x < kDigestHot) hot_region[threadIdx.x] = 0xffffffffu;
     __threadfence();
     __syncthreads();
@@ -338,7 +355,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
       const u32 n = (u32)(hi - lo);
       const u64* const dgs = a.digest + lo;
       const argus_interval_t* const ivs = a.intervals + lo;
-      // two legs: the probe (every cell in the region arrays), then, hot regions chosen, the rest of the stream
+      // two legs: the probe (every interval into its region's cell), then, hot regions chosen, the rest of the stream
       const u32 probe_end = n >= kDigestMinStream ? kDigestProbe : n;
       for (int leg = 0; leg < 2; ++leg) {
         const u32 leg_lo = leg ? probe_end : 0u, leg_hi = leg ? n : probe_end;
@@ -348,16 +365,17 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
             for (u32 h = 0; h < kDigestHot; ++h) {
               u32 best = 0;
               for (u32 r = lane; r < R; r += 32) {
-                if (((cold[kDgMeta * R + r] >> 8) & 0xffu) != kDgNone) continue;
-                u32 cnt = cold[kDgCountOut * R + r];
+                const u32* c = tab + r * kDgWords;
+                if (((c[kDgMeta] >> 8) & 0xffu) != kDgNone) continue;
+                u32 cnt = c[kDgCountOut];
 #pragma unroll
-                for (u32 j = 0; j < kAggWindow; ++j) cnt += cold[(kDgBins + j) * R + r];
+                for (u32 j = 0; j < kAggWindow; ++j) cnt += c[kDgBins + j];
                 const u32 key = ((cnt > 0xffffu ? 0xffffu : cnt) << 16) | r;
                 best = key > best ? key : best;
               }
               const u32 top = __reduce_max_sync(0xffffffffu, best);
               if ((top >> 16) < kDigestProbe / 64) break;  // not worth a set of copies
-              if (lane == 0) { atomicAnd(&cold[kDgMeta * R + (top & 0xffffu)], ~0xff00u | (h << 8)); hot_region[h] = top & 0xffffu; }
+              if (lane == 0) { atomicAnd(&tab[(top & 0xffffu) * kDgWords + kDgMeta], ~0xff00u | (h << 8)); hot_region[h] = top & 0xffffu; }
               __syncwarp();
             }
           }
@@ -365,33 +383,35 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
         }
         // every lane of a warp runs the same number of rounds, so that spans can be appended a warp at a time
         u32 b = leg_lo + (threadIdx.x & ~31u);
+        // digests are asked for two rounds ahead (one round is shorter than a loaded DRAM access)
         u64 dg_next = b + lane < leg_hi ? __ldg(dgs + b + lane) : 0ull;
+        u64 dg_next2 = b + lane + kAggThreads < leg_hi ? __ldg(dgs + b + lane + kAggThreads) : 0ull;
         for (; b < leg_hi; b += kAggThreads) {
           const u32 i = b + lane;
           const u64 dg = dg_next;
-          dg_next = i + kAggThreads < leg_hi ? __ldg(dgs + i + kAggThreads) : 0ull;
+          dg_next = dg_next2;
+          dg_next2 = i + 2 * kAggThreads < leg_hi ? __ldg(dgs + i + 2 * kAggThreads) : 0ull;
           const u32 dlo = (u32)dg, dhi = (u32)(dg >> 32);
           const bool in = i < leg_hi;
           const u32 region = dlo & 0xffffu;
           const bool ok = in && region < R;
           const u32 rsafe = ok ? region : 0u;
           const u32 incl = (dlo >> 18) | ((dhi & 0x1ffu) << 14), excl = dhi >> 9;
-          const u32 meta = cold[kDgMeta * R + rsafe];
+          const u32 meta = tab[rsafe * kDgWords + kDgMeta];
           const u32 slot = (meta >> 8) & 0xffu;
-          u32* const base = slot != kDgNone ? hot + slot * (kDgHotFields * 32) + lane : cold + rsafe;
-          const u32 stride = slot != kDgNone ? 32u : R;
+          const u32 cell = tab_addr + (slot != kDgNone ? R + slot * 32 + lane : rsafe) * (kDgWords * 4);
           // the common case without a branch: a lane that does not take part (past the end, wide, bad region)
           // adds nothing; whatever is rare (a carry, a flag, a bin outside the window, ...) is settled in one place
           const bool take = ok && !(dlo & (1u << 17));
           const u32 vi = take ? incl : 0u, ve = take ? excl : 0u;
-          const u32 old_i = atomicAdd(base + kDgSumInclLo * stride, vi);
-          const u32 old_e = atomicAdd(base + kDgSumExclLo * stride, ve);
-          atomicMin(base + kDgMin * stride, take ? incl : 0xffffffffu);
-          atomicMax(base + kDgMax * stride, vi);
+          const u32 old_i = dg_add<kDgSumInclLo>(cell, vi);
+          const u32 old_e = dg_add<kDgSumExclLo>(cell, ve);
+          dg_min<kDgMin>(cell, take ? incl : 0xffffffffu);
+          dg_max<kDgMax>(cell, vi);
           const u32 bin = 31u - (u32)__clz((int)(incl | 1u));
           const u32 rel = bin - (meta & 0xffu);
           const bool in_win = take && rel < kAggWindow;
-          atomicAdd(base + (kDgBins + (in_win ? rel : 0u)) * stride, in_win ? 1u : 0u);
+          dg_inc<kDgBins>(cell + (in_win ? rel : 0u) * 4, in_win ? 1u : 0u);
           u64 span = vi;
           const bool rare = in && ((dlo & (3u << 16)) || !ok || old_i + vi < old_i || old_e + ve < old_e || !in_win);
           if (rare) {
@@ -410,12 +430,12 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
               if (dlo & (1u << 16)) atomicAdd(row_cell + 7, 1ull);
               atomicAdd(row_cell + 8 + log2_bin(span), 1ull);
             } else {
-              if (old_i + vi < old_i) atomicAdd(base + kDgSumInclHi * stride, 1u);
-              if (old_e + ve < old_e) atomicAdd(base + kDgSumExclHi * stride, 1u);
-              if (dlo & (1u << 16)) atomicAdd(base + kDgFlag * stride, 1u);
+              if (old_i + vi < old_i) dg_inc<kDgSumInclHi>(cell, 1u);
+              if (old_e + ve < old_e) dg_inc<kDgSumExclHi>(cell, 1u);
+              if (dlo & (1u << 16)) dg_inc<kDgFlag>(cell, 1u);
               if (!in_win) {
-                const u32 r2 = digest_bin_rare(cold + kDgMeta * R + region, bin, base, stride, row + (size_t)region * kCell + 8);
-                if (r2 < kAggWindow) atomicAdd(base + (kDgBins + r2) * stride, 1u);
+                const u32 r2 = digest_bin_rare(tab + region * kDgWords + kDgMeta, bin, cell, row + (size_t)region * kCell + 8);
+                if (r2 < kAggWindow) dg_inc<kDgBins>(cell + r2 * 4, 1u);
               }
             }
           }
@@ -435,10 +455,10 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
                 ovc_used = 0;
               }
               if (pick) {
-                const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
-                if (slot < a.ov.ov_capacity) {
-                  a.ov.ov_spans[slot] = make_ulonglong2(t0, t0 + span);
-                  a.ov.ov_seg[slot] = ((k >> 1) * a.num_sms + sm_index) * 2 + (k & 1u);
+                const u64 slot_o = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
+                if (slot_o < a.ov.ov_capacity) {
+                  a.ov.ov_spans[slot_o] = make_ulonglong2(t0, t0 + span);
+                  a.ov.ov_seg[slot_o] = ((k >> 1) * a.num_sms + sm_index) * 2 + (k & 1u);
                 }
               }
               ovc_used += c;
@@ -457,55 +477,53 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
       }
     }
     __syncthreads();
-    // fold the lanes' copies into their region's cell: one thread per (hot region, field), lanes taken in a
-    // rotated order so that the threads of a warp read different banks
-    if (threadIdx.x < kDigestHot * kDgHotFields) {
-      const u32 h = threadIdx.x / kDgHotFields, f = threadIdx.x % kDgHotFields;
+    // fold the lanes' copies into their region's cell: one thread per (hot region, field)
+    if (threadIdx.x < kDigestHot * kDgMeta) {
+      const u32 h = threadIdx.x / kDgMeta, f = threadIdx.x % kDgMeta;
       const u32 r = hot_region[h];
       if (r != 0xffffffffu && f != kDgSumInclHi && f != kDgSumExclHi) {
-        const u32* src = hot + (h * kDgHotFields + f) * 32;
+        const u32* src = tab + (R + h * 32) * kDgWords + f;
+        u32* dst = tab + r * kDgWords + f;
         if (f == kDgSumInclLo || f == kDgSumExclLo) {
-          u64 sum = (u64)cold[f * R + r] | ((u64)cold[(f + 1) * R + r] << 32);
-          for (u32 l = 0; l < 32; ++l) {
-            const u32 ll = (l + threadIdx.x) & 31u;
-            sum += (u64)src[ll] | ((u64)src[32 + ll] << 32);
-          }
-          cold[f * R + r] = (u32)sum;
-          cold[(f + 1) * R + r] = (u32)(sum >> 32);
+          u64 sum = (u64)dst[0] | ((u64)dst[1] << 32);
+          for (u32 l = 0; l < 32; ++l) sum += (u64)src[l * kDgWords] | ((u64)src[l * kDgWords + 1] << 32);
+          dst[0] = (u32)sum;
+          dst[1] = (u32)(sum >> 32);
         } else {
-          u32 acc = cold[f * R + r];
+          u32 acc = dst[0];
           for (u32 l = 0; l < 32; ++l) {
-            const u32 v = src[(l + threadIdx.x) & 31u];
+            const u32 v = src[l * kDgWords];
             acc = f == kDgMin ? (v < acc ? v : acc) : f == kDgMax ? (v > acc ? v : acc) : acc + v;
           }
-          cold[f * R + r] = acc;
+          dst[0] = acc;
         }
       }
     }
     __syncthreads();
-    // the region arrays into the global row, which already holds the wide intervals, the bins outside the
+    // the regions' cells into the global row, which already holds the wide intervals, the bins outside the
     // windows and the ambiguity counters: everything is combined, nothing overwritten
     constexpr u32 kItems = 6 + kAggWindow;
     for (u32 i = threadIdx.x; i < R * kItems; i += blockDim.x) {
       const u32 r = i % R, f = i / R;
+      const u32* c = tab + r * kDgWords;
       u64* cell = row + (size_t)r * kCell;
       switch (f) {
         case 0: {
-          u64 n = cold[kDgCountOut * R + r];
+          u64 cnt = c[kDgCountOut];
 #pragma unroll
-          for (u32 j = 0; j < kAggWindow; ++j) n += cold[(kDgBins + j) * R + r];
-          if (n) atomicAdd(cell + 0, n);
+          for (u32 j = 0; j < kAggWindow; ++j) cnt += c[kDgBins + j];
+          if (cnt) atomicAdd(cell + 0, cnt);
           break;
         }
-        case 1: { const u64 v = (u64)cold[kDgSumInclLo * R + r] | ((u64)cold[kDgSumInclHi * R + r] << 32); if (v) atomicAdd(cell + 1, v); break; }
-        case 2: { const u32 v = cold[kDgMin * R + r]; if (v != 0xffffffffu) atomicMin(cell + 2, (u64)v); break; }
-        case 3: { const u32 v = cold[kDgMax * R + r]; if (v) atomicMax(cell + 3, (u64)v); break; }
-        case 4: { const u64 v = (u64)cold[kDgSumExclLo * R + r] | ((u64)cold[kDgSumExclHi * R + r] << 32); if (v) atomicAdd(cell + 4, v); break; }
-        case 5: { const u32 v = cold[kDgFlag * R + r]; if (v) atomicAdd(cell + 7, (u64)v); break; }
+        case 1: { const u64 v = (u64)c[kDgSumInclLo] | ((u64)c[kDgSumInclHi] << 32); if (v) atomicAdd(cell + 1, v); break; }
+        case 2: { const u32 v = c[kDgMin]; if (v != 0xffffffffu) atomicMin(cell + 2, (u64)v); break; }
+        case 3: { const u32 v = c[kDgMax]; if (v) atomicMax(cell + 3, (u64)v); break; }
+        case 4: { const u64 v = (u64)c[kDgSumExclLo] | ((u64)c[kDgSumExclHi] << 32); if (v) atomicAdd(cell + 4, v); break; }
+        case 5: { const u32 v = c[kDgFlag]; if (v) atomicAdd(cell + 7, (u64)v); break; }
         default: {
           const u32 j = f - 6;
-          const u32 v = cold[(kDgBins + j) * R + r];
-          if (v) atomicAdd(cell + 8 + (cold[kDgMeta * R + r] & 0xffu) + j, (u64)v);
+          const u32 v = c[kDgBins + j];
+          if (v) atomicAdd(cell + 8 + (c[kDgMeta] & 0xffu) + j, (u64)v);
         }
       }
     }
