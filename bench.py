@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 METRIC = "marker events/sec (pair+aggregate, 1 B200) and % of HBM roofline"  # the step also runs the overlap stage
 UNIT = "events/s"
 ALG_BYTES_PER_EVENT = 40.0  # 16 B event read + 48 B interval written per 2 events
-NCU_DRAM_BYTES_PER_EVENT = (614.414848e6 + 867.210240e6) / 38380544  # pairing kernel, ncu capture summarised in profiles/
+NCU_DRAM_BYTES_PER_EVENT = (614.276352e6 + 1018.343e6) / 38380544  # pairing kernel, ncu capture summarised in profiles/
 
 
 def load_peaks():

@@ -453,8 +453,9 @@ int argus_ring_linearise(const argus_event_t* ring /*device [S][slot_capacity]*/
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *
  * Arguments have the meaning they have in argus_pair_intervals, argus_aggregate and
- * argus_overlap. Pairing is followed by one pass over the intervals that both aggregates
- * them and selects the overlap spans (up to 400 regions and 128 pairs; beyond that the three
+ * argus_overlap. Pairing also writes an 8-byte digest of every interval into the workspace
+ * (4 bytes per event), and one pass over the digests both aggregates the intervals and
+ * selects the overlap spans (up to 400 regions and 128 pairs; beyond that the three
  * operations run one after the other). Any of the four tables may be NULL; without tables
  * the pairing kernel selects the overlap spans itself. num_pairs may be 0. max_overlap_spans bounds
  * the spans selected for overlap over all pairs (an interval counts once per pair and role
