@@ -1,6 +1,9 @@
 // argus_aggregate.cu — argus_aggregate: intervals (+ ambiguity records) -> per-(scope, region) tables.
 //
-//   k_agg_streams_compact : one CTA per stream accumulates that stream's row of the warp-scope table in
+//   k_agg_streams_digest : argus_synthesize's pass: one CTA per stream reads the 8-byte digests the pairing
+//                   kernel wrote beside the interval records (not the records) and gathers the stream's row
+//                   in 100-byte shared-memory cells, with per-lane copies of the most frequent regions' cells;
+//   k_agg_streams_compact : the same over the 48-byte records, with an optional scope: that stream's row in
 //                   the compact shared-memory form the fused pairing kernel uses (112 B per region, so
 //                   several CTAs fit an SM), for up to kAggCompactRegions regions;
 //   k_agg_streams : the same with a full 576 B-per-region copy in shared memory when that fits, else on
