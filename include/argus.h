@@ -54,7 +54,7 @@ enum {
   ARGUS_ERR_CAPACITY = 4,    /* device: interval/ambiguity capacity too small; see *_required */
   ARGUS_ERR_DEPTH = 5,       /* device: a stream would hold more than ARGUS_MAX_DEPTH open frames */
   ARGUS_ERR_BAD_REGION = 6,  /* device: tag>>1 >= num_regions                             */
-  ARGUS_ERR_BAD_OFFSETS = 7, /* device: stream_offsets / interval_offsets not non-decreasing */
+  ARGUS_ERR_BAD_OFFSETS = 7, /* device: stream_offsets / interval_offsets decreasing or beyond the array */
   ARGUS_ERR_TIMEOUT = 8,     /* device: a bounded wait expired                            */
   ARGUS_ERR_STATIC_LIMIT = 9 /* host: input larger than the built-in scratch of a *_static call */
 };
@@ -267,8 +267,9 @@ int argus_aggregate(const argus_interval_t* intervals /*device*/,
  * whose CTA maps to m (all depths and contexts, flagged ones included, empty spans
  * dropped); U_P, U_C = their unions. out[k][m] = { |U_P ∩ U_C|, |U_P|, |U_C|, |U_P ∪ U_C| }.
  * max_intervals is an upper bound of interval_offsets[S] known on the host (for instance
- * the capacity given to argus_pair_intervals); it sizes the workspace. If more spans are
- * selected than the workspace holds, status->code = ARGUS_ERR_CAPACITY.
+ * the capacity given to argus_pair_intervals); it sizes the workspace, and a stream whose
+ * offsets reach beyond it is not read (status->code = ARGUS_ERR_BAD_OFFSETS). If more spans
+ * are selected than the workspace holds, status->code = ARGUS_ERR_CAPACITY.
  * ------------------------------------------------------------------------------------- */
 size_t argus_overlap_workspace_bytes(uint64_t max_intervals, uint32_t num_streams,
                                      uint32_t num_pairs, uint32_t num_sms);

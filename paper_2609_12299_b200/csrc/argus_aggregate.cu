@@ -54,6 +54,7 @@ struct AggArgs {
   // overlap span selection in the same pass over the intervals (argus_synthesize); ov.ov_spans null = off
   ArgusFuseArgs ov;
   const u64* digest;  // digests of the intervals (k_agg_streams_digest), null = read the records
+  u64 interval_limit; // records the interval array holds: a stream whose offsets reach beyond it is reported, not read
 };
 
 constexpr u32 kAggOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
@@ -117,7 +118,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams(AggArgs a) {
     const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
     const int sel = stream_in_scope(a, s);
     if (sel == 2 && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, a.cta_sm[s / a.warps_per_cta]);
-    if (hi < lo) {
+    if (hi < lo || hi > a.interval_limit) {
       if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
     } else if (sel == 1) {
       for (u64 i = lo + threadIdx.x; i < hi; i += blockDim.x) {
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
       if (m >= a.num_sms && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
       sm_index = m < a.num_sms ? m : 0;
     }
-    if (hi < lo) {
+    if (hi < lo || hi > a.interval_limit) {
       if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
     } else if (sel == 1) {
       // every lane of a warp runs the same number of rounds, so that spans can be appended a warp at a time
@@ -352,7 +353,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
       if (m >= a.num_sms && threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
       sm_index = m < a.num_sms ? m : 0;
     }
-    if (hi < lo || ((hi - lo) >> 32)) {
+    if (hi < lo || hi > a.interval_limit || ((hi - lo) >> 32)) {
       if (threadIdx.x == 0) argus_set_error(a.status, ARGUS_ERR_BAD_OFFSETS, s, 0);
     } else {
       const u32 n = (u32)(hi - lo);
@@ -610,7 +611,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_iter(AggArgs a) {
   for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
     if (stream_in_scope(a, s) != 1) continue;  // a bad cta_sm entry is reported by k_agg_streams
     const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
-    for (u64 i = lo + threadIdx.x; i < hi && hi >= lo; i += blockDim.x) {
+    for (u64 i = lo + threadIdx.x; i < hi && hi >= lo && hi <= a.interval_limit; i += blockDim.x) {
       const uint4* p = reinterpret_cast<const uint4*>(a.intervals + i);
       const uint4 q1 = __ldg(p + 1);
       const u32 region = q1.z, ctx = q1.w;
@@ -726,7 +727,7 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
   a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
   a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0; a.iter_copies = nullptr; a.num_copies = 0;
   a.iter_inline = 0;
-  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.digest = nullptr;
+  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.digest = nullptr; a.interval_limit = ~0ull;
   if (ambig && ambig_offsets) {
     k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
     ARGUS_CHECK_LAUNCH();
@@ -745,7 +746,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
                                     argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
                                     argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
                                     size_t workspace_bytes, void* cuda_stream, bool reset_status,
-                                    const ArgusFuseArgs* ov_select, const uint64_t* digest) {
+                                    const ArgusFuseArgs* ov_select, const uint64_t* digest, uint64_t interval_limit) {
   if (!interval_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if (ov_select && (num_regions > kAggCompactRegions || ov_select->num_pairs > kFuseMaxPairs)) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
@@ -782,6 +783,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   a.role_tab = (u64*)role_tab; a.iter_tab = (u64*)iter_tab; a.num_iters = num_iters;
   if (ov_select) { a.ov = *ov_select; } else { a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; }
   a.digest = !scope && !role_tab && !iter_tab && num_regions <= kAggCompactRegions ? (const u64*)digest : nullptr;
+  a.interval_limit = interval_limit;
   const size_t smem = (size_t)num_regions * sizeof(argus_agg_t);
   a.use_smem = smem <= kAggSmemLimit;
   const size_t iter_bytes = (size_t)num_iters * smem;
@@ -855,10 +857,11 @@ int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* 
                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
                              argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
                              argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
-                             bool reset_status) {
+                             bool reset_status, uint64_t interval_limit) {
   return argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm,
                                          num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab, nullptr,
-                                         nullptr, status, workspace, workspace_bytes, cuda_stream, reset_status, nullptr);
+                                         nullptr, status, workspace, workspace_bytes, cuda_stream, reset_status, nullptr,
+                                         nullptr, interval_limit);
 }
 
 bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs) {

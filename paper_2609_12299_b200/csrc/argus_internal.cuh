@@ -24,9 +24,10 @@ int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* 
                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
                              argus_agg_t* warp_tab, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab,
                              argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
-                             bool reset_status);
+                             bool reset_status, uint64_t interval_limit = ~0ull);
 // scope, role_tab, iter_tab nullable; ov_select (nullable): also append the overlap spans of the selected intervals;
-// digest (nullable; needs no scope, no role or iteration table, at most 400 regions): the intervals' digests, read instead of the records
+// digest (nullable; needs no scope, no role or iteration table, at most 400 regions): the intervals' digests, read instead of the records;
+// interval_limit: records the interval array holds (a stream whose offsets reach beyond it is reported as ARGUS_ERR_BAD_OFFSETS, not read)
 int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uint64_t* interval_offsets,
                                     const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
                                     uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
@@ -34,7 +35,8 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
                                     argus_agg_t* sm_tab, argus_agg_t* kernel_tab, argus_agg_t* role_tab,
                                     argus_agg_t* iter_tab, argus_status_t* status, void* workspace,
                                     size_t workspace_bytes, void* cuda_stream, bool reset_status,
-                                    const ArgusFuseArgs* ov_select, const uint64_t* digest = nullptr);
+                                    const ArgusFuseArgs* ov_select, const uint64_t* digest = nullptr,
+                                    uint64_t interval_limit = ~0ull);
 // second half of aggregation when the pairing kernel already filled the interval statistics of warp_tab
 int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
                               uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,

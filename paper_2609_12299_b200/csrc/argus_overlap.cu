@@ -20,6 +20,7 @@ constexpr u32 kMaxPairs = 256;
 struct OvArgs {
   const argus_interval_t* intervals;
   const u64* interval_offsets;
+  u64 max_intervals;  // records the interval array holds
   u32 num_streams, warps_per_cta, num_sms, num_pairs;
   const u32* cta_sm;
   const u32* pairs;
@@ -69,7 +70,7 @@ __global__ void __launch_bounds__(256) k_ov_select(OvArgs a, OvSelectOut o) {
   for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
     const u32 m = a.cta_sm[s / a.warps_per_cta];
     const u64 lo = a.interval_offsets[s], hi = a.interval_offsets[s + 1];
-    if (m >= a.num_sms || hi < lo) {
+    if (m >= a.num_sms || hi < lo || hi > a.max_intervals) {  // offsets beyond the interval array are reported, not read
       if (threadIdx.x == 0) argus_set_error(a.status, m >= a.num_sms ? ARGUS_ERR_INVALID_ARG : ARGUS_ERR_BAD_OFFSETS, s, m);
       continue;
     }
@@ -401,7 +402,7 @@ static int ov_setup(OvArgs& a, uint32_t num_streams, uint32_t warps_per_cta, con
   if (workspace_bytes < L.total_fixed + 256 + own_list_bytes) return ARGUS_ERR_WORKSPACE;
   workspace_bytes -= own_list_bytes;  // the caller keeps its list behind the part laid out here
   char* ws = (char*)workspace;
-  a.intervals = nullptr; a.interval_offsets = nullptr; a.num_streams = num_streams;
+  a.intervals = nullptr; a.interval_offsets = nullptr; a.max_intervals = 0; a.num_streams = num_streams;
   a.warps_per_cta = warps_per_cta; a.num_sms = num_sms; a.num_pairs = num_pairs; a.cta_sm = cta_sm; a.pairs = pairs;
   a.out = out; a.status = status;
   a.seg_count = (u64*)(ws + L.seg_count); a.seg_cursor = (u64*)(ws + L.seg_cursor); a.seg_base = (u64*)(ws + L.seg_base);
@@ -455,7 +456,7 @@ static int overlap_scoped(const argus_interval_t* intervals, uint64_t max_interv
   const int rc = ov_setup(a, num_streams, warps_per_cta, cta_sm, num_sms, pairs, num_pairs, out, status, workspace,
                           workspace_bytes, stream, list_bytes);
   if (rc != ARGUS_OK) return rc;
-  a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets;
+  a.intervals = intervals; a.interval_offsets = (const u64*)interval_offsets; a.max_intervals = max_intervals;
   if (scope) {
     a.scoped = 1; a.ctx_lo = scope->ctx_lo; a.ctx_hi = scope->ctx_hi; a.warp_mask = scope->warp_mask;
     a.sm_mask = scope->sm_mask; a.region_mask = scope->region_mask;

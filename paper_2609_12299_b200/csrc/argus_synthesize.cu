@@ -117,7 +117,7 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
                                            cta_sm, num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab,
                                            nullptr, nullptr, status, ws + L.agg, L.agg_bytes, cuda_stream, false,
                                            mode == 1 && list ? &f : nullptr,
-                                           use_digest ? (const uint64_t*)(ws + L.digest) : nullptr);
+                                           use_digest ? (const uint64_t*)(ws + L.digest) : nullptr, interval_capacity);
     }
     if (rc != ARGUS_OK) return rc;
   }

@@ -382,6 +382,34 @@ def test_synthesize_overlap_span_capacity():
     assert int(st["code"]) == 4 and int(st["intervals_required"]) > 512
 
 
+def test_synthesize_interval_capacity_too_small(synth_mode):
+    """Fewer interval slots than the trace needs: the call reports ARGUS_ERR_CAPACITY with the required count, the
+    later stages read nothing beyond the array, and the same buffers work again with enough room."""
+    spec = tg.config(1).scaled(2, 40)
+    ev, offs = tg.generate_host(spec)
+    d_ev, d_off = to_dev(ev, offs)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(DEV)
+    need = len(ev) // 2
+    res = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, pairs,
+                                 interval_capacity=need // 3)
+    st = res.fetch_status()
+    assert int(st["code"]) == 4 and int(st["intervals_required"]) == need
+    _synthesize_matches(spec, ev, offs)
+
+
+def test_overlap_offsets_beyond_the_interval_array_are_reported():
+    spec = tg.config(1).scaled(2, 40)
+    ev, offs = tg.generate_host(spec)
+    d_ev, d_off = to_dev(ev, offs)
+    pr = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(DEV)
+    n_iv = int(pr.interval_offsets[-1].item())
+    _, st = argus.argus_overlap(pr.intervals, n_iv // 2, pr.interval_offsets, spec.warps_per_cta, cta_sm, spec.num_sms, pairs)
+    assert int(argus.argus_status_fetch(st)["code"]) == 7  # ARGUS_ERR_BAD_OFFSETS
+
+
 def test_maximum_region_count():
     """num_regions at its upper bound (65536): pairing, the global-row aggregation path and the one-call
     pipeline (which cannot host such a table in shared memory and runs the three plain calls)."""
