@@ -266,7 +266,7 @@ def _synthesize_matches(spec, ev, offs, **kw):
     assert np.array_equal(res.pair.ambig_offsets.cpu().numpy().view(np.uint64), o_aoffs)
     _, o_tabs, _ = oracle.aggregate(o_iv, o_ioffs, o_am, o_aoffs, spec.warps_per_cta, spec.cta_sm, spec.num_sms,
                                     spec.num_regions)
-    for lv in ("warp", "cta", "sm", "kernel"):
+    for lv in kw.get("levels", ("warp", "cta", "sm", "kernel")):
         got, want = res.agg.table_numpy(lv), o_tabs[lv]
         if got.tobytes() != want.tobytes():
             bad = np.argwhere(got != want)
@@ -293,6 +293,14 @@ def test_synthesize_fused_matches_oracle(idx, ctas, iters, synth_mode):
     res, st = _synthesize_matches(spec, ev, offs)
     if spec.well_formed:
         assert int(st["n_sequential_tiles"]) == 0
+
+
+@pytest.mark.parametrize("levels", [("kernel",), ("sm",), ("cta", "kernel"), ("warp",), ()])
+def test_synthesize_table_subsets(levels, synth_mode):
+    """Any subset of the four tables may be asked for (none: intervals and overlap only)."""
+    spec = tg.config(3).scaled(2, 5)
+    ev, offs = tg.generate_host(spec)
+    _synthesize_matches(spec, ev, offs, levels=levels)
 
 
 def test_synthesize_wide_histogram_and_flags(synth_mode):
