@@ -450,6 +450,28 @@ int argus_ring_linearise(const argus_event_t* ring /*device [S][slot_capacity]*/
                          argus_status_t* status /*device*/, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------
+ * argus_pair_intervals_ring — pairing straight from the ring container above, without the
+ * packed copy: the pairing kernel fetches every tile of a stream from its slot with one bulk
+ * copy, or two where the tile straddles the slot's end. Results (intervals, ambiguity
+ * records, offsets, status) are those of argus_ring_linearise followed by
+ * argus_pair_intervals; event indices (begin_idx, event_idx) count the surviving records of
+ * the stream, oldest first. stream_offsets[S + 1] (out) receives the offsets the packed form
+ * would have, dropped[S] (out, nullable) the records lost to the wrap. Workspace:
+ * argus_pair_workspace_bytes(S * slot_capacity, S, ambig_capacity) bytes, 256-byte aligned.
+ * ------------------------------------------------------------------------------------- */
+int argus_pair_intervals_ring(const argus_event_t* ring /*device [S][slot_capacity]*/,
+                              uint32_t slot_capacity, const uint64_t* written /*device [S]*/,
+                              uint32_t num_streams, uint32_t num_regions,
+                              uint64_t* stream_offsets /*device [S+1] out*/,
+                              uint64_t* dropped /*device [S] out, nullable*/,
+                              argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
+                              uint64_t* interval_offsets /*device [S+1] out*/,
+                              argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
+                              uint64_t* ambig_offsets /*device [S+1] out*/,
+                              argus_status_t* status /*device*/, void* workspace /*device*/,
+                              size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
  * argus_synthesize — the three operations above in one call, with identical results
  * (Section 3.2 for intervals and scopes; the Synthesize task of Section 3.4).
  *

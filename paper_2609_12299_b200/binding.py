@@ -80,6 +80,8 @@ def load_library():
     lib.argus_join_samples.restype = ci
     lib.argus_ring_linearise.argtypes = [vp, u32, vp, u32, vp, u64, vp, vp, vp, vp]
     lib.argus_ring_linearise.restype = ci
+    lib.argus_pair_intervals_ring.argtypes = [vp, u32, vp, u32, u32, vp, vp, vp, u64, vp, vp, u64, vp, vp, vp, sz, vp]
+    lib.argus_pair_intervals_ring.restype = ci
     lib.argus_status_fetch.argtypes = [vp, vp, vp]
     lib.argus_status_fetch.restype = ci
     lib.argus_strerror.argtypes = [ci]
@@ -470,6 +472,30 @@ def argus_ring_linearise(ring: torch.Tensor, slot_capacity: int, written: torch.
     if rc != 0:
         raise ArgusError(rc, "argus_ring_linearise")
     return events, offsets, dropped[:S], status
+
+
+def argus_pair_intervals_ring(ring: torch.Tensor, slot_capacity: int, written: torch.Tensor, num_regions: int,
+                              interval_capacity: int | None = None, ambig_capacity: int | None = None):
+    """Pairing straight from a ring container (see argus_ring_linearise for the layout), without the packed copy.
+    Returns (PairResult, stream_offsets int64 [S + 1] of the packed form, dropped int64 [S])."""
+    lib = load_library()
+    dev = ring.device
+    S = written.numel()
+    bound = S * slot_capacity
+    icap = bound // 2 if interval_capacity is None else int(interval_capacity)
+    acap = bound if ambig_capacity is None else int(ambig_capacity)
+    out = PairResult(_bytes(icap * 48, dev), torch.empty(S + 1, dtype=torch.int64, device=dev),
+                     _bytes(acap * 32, dev), torch.empty(S + 1, dtype=torch.int64, device=dev),
+                     _bytes(64, dev), icap, acap, _bytes(lib.argus_pair_workspace_bytes(bound, S, acap), dev))
+    offsets = torch.empty(S + 1, dtype=torch.int64, device=dev)
+    dropped = torch.empty(max(S, 1), dtype=torch.int64, device=dev)
+    rc = lib.argus_pair_intervals_ring(_ptr(ring), slot_capacity, _ptr(written), S, num_regions, _ptr(offsets), _ptr(dropped),
+                                       _ptr(out.intervals), out.interval_capacity, _ptr(out.interval_offsets), _ptr(out.ambig),
+                                       out.ambig_capacity, _ptr(out.ambig_offsets), _ptr(out.status), _ptr(out.workspace),
+                                       out.workspace.numel(), _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_pair_intervals_ring")
+    return out, offsets, dropped[:S]
 
 
 @dataclass

@@ -7,12 +7,15 @@
 // argus_pair.cu — the whole pairing pipeline. kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled.
 // `fuse` (nullable) asks the tiled kernel to feed aggregation / overlap selection; *fused_out tells whether it did.
 // `digest` (nullable): one 8-byte digest per interval record, at the record's position (see argus_fuse.cuh).
+// `ring_written` (nullable): `events` is a ring container (one slot of ring_capacity records per stream, written[s] records
+// ever written); stream_offsets describe the packed survivors and num_events bounds them. Tiled kernel only.
 int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
                         uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
                         uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
                         uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
                         size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out, uint64_t* digest = nullptr, uint64_t digest_capacity = 0);
+                        bool reset_status, bool* fused_out, uint64_t* digest = nullptr, uint64_t digest_capacity = 0,
+                        const uint64_t* ring_written = nullptr, uint32_t ring_capacity = 0);
 
 // argus_pair_tiled.cu
 bool argus_pair_tiled_can_fuse(uint32_t num_regions);

@@ -157,7 +157,13 @@ __global__ void __launch_bounds__(256) k_ambig_scatter(AmbigArgs g) {
       const u32 mid = lo + ((hi - lo) >> 1);
       if (g.p.stream_offsets[mid] <= x) lo = mid; else hi = mid;
     }
-    const argus_event_t e = g.p.events[x];
+    u64 at = x;  // where the record lies: packed input, or its slot position in a ring container
+    if (g.p.ring_written) {
+      u64 pos = argus_ring_first(g.p, lo) + (x - g.p.stream_offsets[lo]);
+      if (pos >= g.p.ring_capacity) pos -= g.p.ring_capacity;
+      at = (u64)lo * g.p.ring_capacity + pos;
+    }
+    const argus_event_t e = g.p.events[at];
     argus_ambiguity_t rec;
     rec.ts = e.ts; rec.tag = e.tag; rec.ctx = e.ctx; rec.stream = lo;
     rec.event_idx = (u32)(x - g.p.stream_offsets[lo]);
@@ -220,7 +226,8 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
                         uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
                         uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
                         size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out, uint64_t* digest, uint64_t digest_capacity) {
+                        bool reset_status, bool* fused_out, uint64_t* digest, uint64_t digest_capacity,
+                        const uint64_t* ring_written, uint32_t ring_capacity) {
   if (!stream_offsets || !interval_offsets || !ambig_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if ((num_events && !events) || (interval_capacity && !intervals) || (ambig_capacity && !ambig)) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
@@ -247,6 +254,8 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   a.queue = (u32*)(ws + L.queue); a.queue_capacity = L.queue_capacity;
   a.records = (ArgusStreamRecord*)(ws + L.records); a.record_capacity = L.record_capacity;
   memset(&a.fuse, 0, sizeof(a.fuse));
+  a.ring_written = (const u64*)ring_written; a.ring_capacity = ring_capacity;
+  if (ring_written && (ring_capacity == 0 || kernel_choice == 1)) return ARGUS_ERR_INVALID_ARG;  // only the tiled kernel reads rings
   // a stream's intervals start at half its first event's position at the latest, so positions stay below num_events / 2 + 1
   a.digest = digest_capacity >= (interval_capacity < num_events / 2 + 1 ? interval_capacity : num_events / 2 + 1) ? (u64*)digest : nullptr;
 
@@ -254,7 +263,7 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   // control block, counts and bitmap are contiguous at the start of the workspace
   ARGUS_CUDA_TRY(cudaMemsetAsync(ws, 0, L.word_prefix, stream));
 
-  const bool tiled = kernel_choice != 1 && argus_pair_tiled_usable(a);
+  const bool tiled = (kernel_choice != 1 && argus_pair_tiled_usable(a)) || ring_written != nullptr;
   const bool fused = tiled && fuse && argus_pair_tiled_can_fuse(num_regions);
   if (fused) a.fuse = *fuse;
   if (fused_out) *fused_out = fused;
@@ -314,4 +323,27 @@ extern "C" int argus_pair_intervals(const argus_event_t* events, uint64_t num_ev
   return argus_pair_intervals_ex(events, num_events, stream_offsets, num_streams, num_regions, intervals,
                                  interval_capacity, interval_offsets, ambig, ambig_capacity, ambig_offsets, status,
                                  workspace, workspace_bytes, cuda_stream, 0);
+}
+
+// implemented in argus_ring.cu
+int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
+                                uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream);
+
+extern "C" int argus_pair_intervals_ring(const argus_event_t* ring, uint32_t slot_capacity, const uint64_t* written,
+                                         uint32_t num_streams, uint32_t num_regions, uint64_t* stream_offsets,
+                                         uint64_t* dropped, argus_interval_t* intervals, uint64_t interval_capacity,
+                                         uint64_t* interval_offsets, argus_ambiguity_t* ambig, uint64_t ambig_capacity,
+                                         uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
+  if (!status || !stream_offsets || slot_capacity == 0) return ARGUS_ERR_INVALID_ARG;
+  if (num_streams && (!ring || !written)) return ARGUS_ERR_INVALID_ARG;
+  if (((uintptr_t)written & 7) || ((uintptr_t)dropped & 7)) return ARGUS_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), stream));
+  const uint64_t bound = (uint64_t)num_streams * slot_capacity;  // what the slots can hold: sizes the workspace
+  int rc = argus_internal_ring_offsets(written, slot_capacity, num_streams, bound, stream_offsets, dropped, status, cuda_stream);
+  if (rc != ARGUS_OK) return rc;
+  return argus_internal_pair(ring, bound, stream_offsets, num_streams, num_regions, intervals, interval_capacity, interval_offsets,
+                             ambig, ambig_capacity, ambig_offsets, status, workspace, workspace_bytes, cuda_stream, 2, nullptr,
+                             false, nullptr, nullptr, 0, written, slot_capacity);
 }

@@ -76,10 +76,18 @@ struct ArgusPairArgs {
   u32 record_capacity;
   u64* digest;            // one digest per interval record, same positions (null = none); holds every position below
                           // min(interval_capacity, num_events / 2 + 1), which is all a stream can reach
+  const u64* ring_written; // non-null: `events` is a ring container, one slot of ring_capacity records per stream, record i of
+  u32 ring_capacity;       // a stream at slot position i mod capacity; stream_offsets then describe the packed survivors
   ArgusFuseArgs fuse;     // optional aggregation / overlap selection fed from the pairing kernel (first pass only)
 };
 
 #define ARGUS_NOTE_POS_BITS 48
+
+// Ring container: slot position of the oldest surviving record of stream s.
+__device__ __forceinline__ u32 argus_ring_first(const ArgusPairArgs& a, u32 s) {
+  const u64 w = a.ring_written[s];
+  return w > a.ring_capacity ? (u32)(w % a.ring_capacity) : 0u;
+}
 
 __device__ __forceinline__ void argus_note_ambiguity(const ArgusPairArgs& a, u64 gpos, u32 kind, u32 depth) {
   const u64 slot = atomicAdd(&a.ctl->n_notes, 1ull);

@@ -168,7 +168,25 @@ __device__ __forceinline__ int tile_latest_begin(const TileSmem<NT, E>& sm, int 
 
 constexpr u32 kOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
 
-template <int NT, int E, int MINB, bool FUSE>
+// One tile of a stream into shared memory: a bulk copy, or two when the stream lives in a ring slot and the
+// tile straddles the slot's end. `src` is the stream's first record (packed input) or its slot (ring).
+template <bool RING>
+__device__ __forceinline__ void tile_fetch(const ArgusPairArgs& a, uint4* dst, const argus_event_t* src, u32 ring_first,
+                                           u32 start, u32 count, u64* bar) {
+  mbar_expect_tx(bar, count * 16u);
+  if (!RING) {
+    tma_load_1d(dst, src + start, count * 16u, bar);
+  } else {
+    u32 p = ring_first + start;  // both below the capacity
+    if (p >= a.ring_capacity) p -= a.ring_capacity;
+    const u32 room = a.ring_capacity - p;
+    const u32 head = count < room ? count : room;
+    tma_load_1d(dst, src + p, head * 16u, bar);
+    if (count > head) tma_load_1d(dst + head, src, (count - head) * 16u, bar);
+  }
+}
+
+template <int NT, int E, int MINB, bool FUSE, bool RING = false>
 __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   using SM = TileSmem<NT, E>;
   constexpr int T = SM::T, NW = SM::NW, NWORDS = SM::NWORDS, MAXI = SM::MAXI, NI = SM::NI;
@@ -242,7 +260,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     const u32 n = (u32)(hi - lo);
     const u64 gpos0 = lo - off0;
     const u64 out_base = a.redo ? a.interval_offsets[s] : (gpos0 >> 1);
-    const argus_event_t* src = a.events + lo;
+    const argus_event_t* src = RING ? a.events + (u64)s * a.ring_capacity : a.events + lo;
+    const u32 ring_first = RING ? argus_ring_first(a, s) : 0u;
     const u32 ntiles = (n + T - 1) / T;
     int ch = 0;          // carried stack height (uniform)
     u64 n_int = 0;       // intervals of this stream so far (uniform)
@@ -289,9 +308,8 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     }
     if (tid == 0 && ti0 < ti_end) {  // first tile of this chunk, into the buffer its index selects
       const u32 start = ti0 * (u32)T;
-      const u32 bytes = ((n - start) < (u32)T ? (n - start) : (u32)T) * 16u;
-      mbar_expect_tx(&sm.bar[ti0 & 1], bytes);
-      tma_load_1d((ti0 & 1) ? sm.evall + T + 2 * kCar : sm.evall, src + start, bytes, &sm.bar[ti0 & 1]);
+      tile_fetch<RING>(a, (ti0 & 1) ? sm.evall + T + 2 * kCar : sm.evall, src, ring_first, start,
+                       (n - start) < (u32)T ? (n - start) : (u32)T, &sm.bar[ti0 & 1]);
     }
 
     int cpar = 0;        // which carried-frame block holds the current stack
@@ -306,9 +324,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       const int carlo = b ? -2 * kCar : T;               // reference of slot 0 of carried block 0, seen from this buffer
       if (tid == 0 && ti + 1 < ti_end) {  // prefetch the next tile into the other buffer
         const u32 nstart = tile_start + T;
-        const u32 bytes = ((n - nstart) < (u32)T ? (n - nstart) : (u32)T) * 16u;
-        mbar_expect_tx(&sm.bar[b ^ 1], bytes);
-        tma_load_1d(b ? ev0 : ev1, src + nstart, bytes, &sm.bar[b ^ 1]);
+        tile_fetch<RING>(a, b ? ev0 : ev1, src, ring_first, nstart, (n - nstart) < (u32)T ? (n - nstart) : (u32)T, &sm.bar[b ^ 1]);
       }
       TT_MARK(0);
       {
@@ -660,7 +676,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   }
 }
 
-template <int NT, int E, int MINB, bool FUSE>
+template <int NT, int E, int MINB, bool FUSE, bool RING = false>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   // the shared-memory opt-in and the occupancy belong to one device: cached per device, redone when the size changes
   constexpr int kMaxDevices = 64;
@@ -672,10 +688,10 @@ int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   ARGUS_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return ARGUS_ERR_INVALID_ARG;
   if (!grid_of[dev] || smem_of[dev] != smem) {
-    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int sms = 0, per_sm = 0;
     ARGUS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB, FUSE>, NT, smem));
+    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB, FUSE, RING>, NT, smem));
     if (per_sm < 1) return ARGUS_ERR_CUDA;
     if (per_sm > MINB) per_sm = MINB;
     grid_of[dev] = sms * per_sm;
@@ -683,7 +699,7 @@ int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   }
   const int grid_cache = grid_of[dev];
   const u32 grid = a.num_streams < (u32)grid_cache ? a.num_streams : (u32)grid_cache;
-  k_pair_tiled<NT, E, MINB, FUSE><<<grid, NT, smem, stream>>>(a);
+  k_pair_tiled<NT, E, MINB, FUSE, RING><<<grid, NT, smem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   return ARGUS_OK;
 }
@@ -718,6 +734,7 @@ extern "C" int argus_debug_tile_timing(unsigned long long* out8) {
 extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
+  if (a.ring_written) return launch_tiled<128, 5, 6, false, true>(a, stream);  // ring container: plain pairing, one shape
   switch (g_variant) {
     case 1: return launch_tiled_any<192, 5, 4>(a, stream);
     case 2: return launch_tiled_any<320, 5, 2>(a, stream);

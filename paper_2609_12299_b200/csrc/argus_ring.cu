@@ -53,6 +53,16 @@ __global__ void __launch_bounds__(256) k_ring_copy(const uint4* ring, u32 slot_c
 
 }  // namespace
 
+// stream_offsets (and dropped) of the records that survive in the slots; status->code = ARGUS_ERR_CAPACITY if they
+// exceed event_capacity. The status block is not cleared here.
+int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
+                                uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream) {
+  k_ring_offsets<<<1, kRingScanThreads, 0, (cudaStream_t)cuda_stream>>>((const u64*)written, slot_capacity, num_streams, event_capacity,
+                                                                        (u64*)stream_offsets, (u64*)dropped, status);
+  ARGUS_CHECK_LAUNCH();
+  return ARGUS_OK;
+}
+
 extern "C" int argus_ring_linearise(const argus_event_t* ring, uint32_t slot_capacity, const uint64_t* written,
                                     uint32_t num_streams, argus_event_t* events, uint64_t event_capacity,
                                     uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream) {

@@ -2,6 +2,7 @@
 
     python -m paper_2609_12299_b200.measure scoped   # argus_aggregate_scoped / argus_overlap_scoped on trace 3
     python -m paper_2609_12299_b200.measure pcmap    # PC-to-region mapping and attribution on a mapping run
+    python -m paper_2609_12299_b200.measure ring     # pairing from a ring container: packed copy first, or directly
 
 Each line printed is one JSON object: what ran, its time (best of the repetitions after warm-up), the
 algorithmic bytes it has to move and the fraction of the measured HBM copy bandwidth that amounts to.
@@ -119,9 +120,46 @@ def run_pcmap(iters: int, num_pcs: int, execs_per_begin: int):
     _line("argus_attribute without alpha output", ms_attr2, (R + 1) * num_pcs * 8 + num_pcs * 16, rows=R + 1, pcs=num_pcs)
 
 
+def run_ring(iters: int, shift_tokens: int):
+    """Trace 3 held in a ring container (one slot per stream, exactly as long as the stream): pairing after
+    argus_ring_linearise against argus_pair_intervals_ring, which reads the slots directly."""
+    spec = tg.config(3).scaled(iters=iters) if iters else tg.config(3)
+    dev = torch.device("cuda", 0)
+    d_ev, d_off = tg.generate_cuda(spec, dev)
+    n = d_ev.numel() // 16
+    S = spec.num_streams
+    cap = n // S                                      # every stream of this trace has the same length
+    shift = (cap // spec.iters) * shift_tokens        # records written before the survivors: a whole number of tokens
+    written = torch.full((S,), cap + shift, dtype=torch.int64, device=dev)
+    R = spec.num_regions
+    state = {}
+
+    def two_steps():
+        ev, offs, _, st = argus.argus_ring_linearise(d_ev, cap, written)
+        state["p"] = argus.argus_pair_intervals(ev, offs, R, interval_capacity=n // 2, ambig_capacity=max(n // 64, 4096),
+                                                out=state.get("p"))
+        return ev
+
+    ms2 = _time(two_steps, reps=3, warmup=1)
+    st = state["p"].fetch_status()
+    assert int(st["code"]) == 0, st
+    _line("argus_ring_linearise + argus_pair_intervals", ms2, 72.0 * n, events=n, workload=spec.name, shift_records=shift,
+          sequential_tiles=int(st["n_sequential_tiles"]), note="algorithmic bytes: 32 B/event for the copy + 40 B/event for pairing")
+    del state["p"]
+    torch.cuda.empty_cache()
+    ms1 = _time(lambda: argus.argus_pair_intervals_ring(d_ev, cap, written, R, interval_capacity=n // 2,
+                                                         ambig_capacity=max(n // 64, 4096)), reps=3, warmup=1)
+    pr, _, _ = argus.argus_pair_intervals_ring(d_ev, cap, written, R, interval_capacity=n // 2, ambig_capacity=max(n // 64, 4096))
+    st = pr.fetch_status()
+    assert int(st["code"]) == 0, st
+    _line("argus_pair_intervals_ring (allocations included)", ms1, 40.0 * n, events=n, workload=spec.name, shift_records=shift,
+          sequential_tiles=int(st["n_sequential_tiles"]))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["scoped", "pcmap"])
+    ap.add_argument("what", choices=["scoped", "pcmap", "ring"])
+    ap.add_argument("--shift-tokens", type=int, default=100, help="`ring`: tokens written before the surviving records (0: no wrap)")
     ap.add_argument("--iters", type=int, default=0, help="tokens per stream of the decode trace (0: full size for `scoped`, 24 for `pcmap`)")
     ap.add_argument("--pcs", type=int, default=70_560)
     ap.add_argument("--execs-per-begin", type=int, default=2)
@@ -129,6 +167,8 @@ def main():
     argus.load_library()
     if a.what == "scoped":
         run_scoped(a.iters)
+    elif a.what == "ring":
+        run_ring(a.iters, a.shift_tokens)
     else:
         run_pcmap(a.iters or 24, a.pcs, a.execs_per_begin)
 

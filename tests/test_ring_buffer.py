@@ -92,3 +92,26 @@ def test_gpu_ring_linearise_matches_the_oracle(S, cap):
         ev2, _, _, status2 = argus.argus_ring_linearise(d_ring, cap, d_written, event_capacity=max(n - 1, 0))
         st2 = argus.argus_status_fetch(status2)
         assert (int(st2["code"]) == 4 and int(st2["intervals_required"]) == n) if n else int(st2["code"]) == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("S,cap", [(9, 64), (40, 1000), (3, 1), (0, 8), (6, 5000)])
+def test_gpu_pairing_straight_from_the_ring(S, cap):
+    """argus_pair_intervals_ring = linearise + pair, without the copy: tiles that straddle the slot's end are fetched
+    in two pieces (slot sizes below, around and above the 640-record tile; streams that wrapped and streams that did not)."""
+    import torch
+    import paper_2609_12299_b200 as argus
+    rng = np.random.default_rng(S * 77 + cap)
+    streams, (ring, written) = _random_case(rng, S, cap)
+    rc, want, offs, dropped, st = oracle.ring_linearise(ring, cap, written)
+    rc, iv, ioffs, am, aoffs, o_st = oracle.pair(want, offs, 5)
+    d_ring = torch.from_numpy(ring.view(np.uint8).reshape(-1).copy()).to("cuda:0")
+    d_written = torch.from_numpy(written.view(np.int64).copy()).to("cuda:0")
+    pr, d_offs, d_dropped = argus.argus_pair_intervals_ring(d_ring, cap, d_written, 5)
+    assert int(pr.fetch_status()["code"]) == 0
+    assert np.array_equal(d_offs.cpu().numpy().view(np.uint64), offs)
+    assert np.array_equal(d_dropped.cpu().numpy().view(np.uint64), dropped)
+    assert pr.intervals_numpy().tobytes() == iv.tobytes()
+    assert pr.ambig_numpy().tobytes() == am.tobytes()
+    assert np.array_equal(pr.interval_offsets.cpu().numpy().view(np.uint64), ioffs)
+    assert np.array_equal(pr.ambig_offsets.cpu().numpy().view(np.uint64), aoffs)
