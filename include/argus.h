@@ -504,6 +504,26 @@ int argus_synthesize(const argus_event_t* events /*device*/, uint64_t num_events
                      argus_status_t* status /*device*/, void* workspace /*device*/,
                      size_t workspace_bytes, void* cuda_stream);
 
+/* The same from the ring container: argus_pair_intervals_ring's pairing inside the one-call
+ * pipeline. stream_offsets[S + 1] and dropped[S] (nullable) are outputs as there. Workspace:
+ * argus_synthesize_workspace_bytes(S * slot_capacity, ...) bytes. */
+int argus_synthesize_ring(const argus_event_t* ring /*device [S][slot_capacity]*/,
+                          uint32_t slot_capacity, const uint64_t* written /*device [S]*/,
+                          uint32_t num_streams, uint32_t num_regions,
+                          uint64_t* stream_offsets /*device [S+1] out*/,
+                          uint64_t* dropped /*device [S] out, nullable*/,
+                          argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
+                          uint64_t* interval_offsets /*device [S+1] out*/,
+                          argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
+                          uint64_t* ambig_offsets /*device [S+1] out*/, uint32_t warps_per_cta,
+                          const uint32_t* cta_sm /*device [C]*/, uint32_t num_sms,
+                          argus_agg_t* warp_tab /*device, nullable*/, argus_agg_t* cta_tab /*device, nullable*/,
+                          argus_agg_t* sm_tab /*device, nullable*/, argus_agg_t* kernel_tab /*device, nullable*/,
+                          const uint32_t* pairs /*device [K][2]*/, uint32_t num_pairs,
+                          argus_overlap_t* overlap_out /*device [K][M]*/, uint64_t max_overlap_spans,
+                          argus_status_t* status /*device*/, void* workspace /*device*/,
+                          size_t workspace_bytes, void* cuda_stream);
+
 /* Copies the device status block to host memory and synchronises `cuda_stream`.
  * Returns ARGUS_OK or ARGUS_ERR_CUDA; the device-side code is in host_copy->code. */
 int argus_status_fetch(const argus_status_t* dev_status, argus_status_t* host_copy,

@@ -101,6 +101,9 @@ def load_library():
     lib.argus_synthesize.argtypes = [vp, u64, vp, u32, u32, vp, u64, vp, vp, u64, vp, u32, vp, u32, vp, vp, vp, vp, vp, u32,
                                      vp, u64, vp, vp, sz, vp]
     lib.argus_synthesize.restype = ci
+    lib.argus_synthesize_ring.argtypes = [vp, u32, vp, u32, u32, vp, vp, vp, u64, vp, vp, u64, vp, u32, vp, u32, vp, vp, vp, vp, vp,
+                                          u32, vp, u64, vp, vp, sz, vp]
+    lib.argus_synthesize_ring.restype = ci
     _lib = lib
     return lib
 
@@ -521,6 +524,50 @@ def argus_synthesize_workspace_bytes(num_events: int, num_streams: int, num_regi
                                                 max_overlap_spans)
 
 
+def _synthesize_buffers(dev, n, S, K, num_regions, warps_per_cta, num_sms, interval_capacity, ambig_capacity, max_overlap_spans,
+                        levels) -> SynthesizeResult:
+    """Output tensors and workspace of the one-call pipeline for a trace of at most n events."""
+    icap = n // 2 if interval_capacity is None else int(interval_capacity)
+    acap = n if ambig_capacity is None else int(ambig_capacity)
+    mos = (2 * K * icap if max_overlap_spans is None else int(max_overlap_spans)) if K else 0
+    C = S // warps_per_cta if warps_per_cta else 0
+    keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1}
+    tabs = {lv: (_bytes(keys[lv] * num_regions * 576, dev) if lv in levels else None) for lv in keys}
+    status = _bytes(64, dev)
+    pr = PairResult(_bytes(icap * 48, dev), torch.empty(S + 1, dtype=torch.int64, device=dev), _bytes(acap * 32, dev),
+                    torch.empty(S + 1, dtype=torch.int64, device=dev), status, icap, acap, _bytes(1, dev))
+    ag = AggregateResult(tabs["warp"], tabs["cta"], tabs["sm"], tabs["kernel"], status, _bytes(1, dev),
+                         {lv: (keys[lv], num_regions) for lv in keys})
+    ws = _bytes(argus_synthesize_workspace_bytes(n, S, num_regions, acap, K, num_sms, mos), dev)
+    return SynthesizeResult(pr, ag, _bytes(K * num_sms * 32, dev) if K else None, status, ws, mos)
+
+
+def argus_synthesize_ring(ring: torch.Tensor, slot_capacity: int, written: torch.Tensor, num_regions: int, warps_per_cta: int,
+                          cta_sm: torch.Tensor, num_sms: int, pairs: torch.Tensor | None = None,
+                          interval_capacity: int | None = None, ambig_capacity: int | None = None,
+                          max_overlap_spans: int | None = None, levels=("warp", "cta", "sm", "kernel")):
+    """The one-call pipeline on a ring container (see argus_ring_linearise for the layout).
+    Returns (SynthesizeResult, stream_offsets int64 [S + 1] of the packed form, dropped int64 [S])."""
+    lib = load_library()
+    dev = ring.device
+    S = written.numel()
+    K = 0 if pairs is None else pairs.numel() // 2
+    out = _synthesize_buffers(dev, S * slot_capacity, S, K, num_regions, warps_per_cta, num_sms, interval_capacity,
+                              ambig_capacity, max_overlap_spans, levels)
+    offsets = torch.empty(S + 1, dtype=torch.int64, device=dev)
+    dropped = torch.empty(max(S, 1), dtype=torch.int64, device=dev)
+    p, a = out.pair, out.agg
+    rc = lib.argus_synthesize_ring(_ptr(ring), slot_capacity, _ptr(written), S, num_regions, _ptr(offsets), _ptr(dropped),
+                                   _ptr(p.intervals), p.interval_capacity, _ptr(p.interval_offsets), _ptr(p.ambig),
+                                   p.ambig_capacity, _ptr(p.ambig_offsets), warps_per_cta, _ptr(cta_sm), num_sms, _ptr(a.warp),
+                                   _ptr(a.cta), _ptr(a.sm), _ptr(a.kernel), _ptr(pairs), K, _ptr(out.overlap),
+                                   out.max_overlap_spans, _ptr(out.status), _ptr(out.workspace), out.workspace.numel(),
+                                   _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_synthesize_ring")
+    return out, offsets, dropped[:S]
+
+
 def argus_synthesize(events: torch.Tensor, stream_offsets: torch.Tensor, num_regions: int, warps_per_cta: int,
                      cta_sm: torch.Tensor, num_sms: int, pairs: torch.Tensor | None = None,
                      interval_capacity: int | None = None, ambig_capacity: int | None = None,
@@ -533,19 +580,8 @@ def argus_synthesize(events: torch.Tensor, stream_offsets: torch.Tensor, num_reg
     S = stream_offsets.numel() - 1
     K = 0 if pairs is None else pairs.numel() // 2
     if out is None:
-        icap = n // 2 if interval_capacity is None else int(interval_capacity)
-        acap = n if ambig_capacity is None else int(ambig_capacity)
-        mos = (2 * K * icap if max_overlap_spans is None else int(max_overlap_spans)) if K else 0
-        C = S // warps_per_cta if warps_per_cta else 0
-        keys = {"warp": S, "cta": C, "sm": num_sms, "kernel": 1}
-        tabs = {lv: (_bytes(keys[lv] * num_regions * 576, dev) if lv in levels else None) for lv in keys}
-        status = _bytes(64, dev)
-        pr = PairResult(_bytes(icap * 48, dev), torch.empty(S + 1, dtype=torch.int64, device=dev), _bytes(acap * 32, dev),
-                        torch.empty(S + 1, dtype=torch.int64, device=dev), status, icap, acap, _bytes(1, dev))
-        ag = AggregateResult(tabs["warp"], tabs["cta"], tabs["sm"], tabs["kernel"], status, _bytes(1, dev),
-                             {lv: (keys[lv], num_regions) for lv in keys})
-        ws = _bytes(argus_synthesize_workspace_bytes(n, S, num_regions, acap, K, num_sms, mos), dev)
-        out = SynthesizeResult(pr, ag, _bytes(K * num_sms * 32, dev) if K else None, status, ws, mos)
+        out = _synthesize_buffers(dev, n, S, K, num_regions, warps_per_cta, num_sms, interval_capacity, ambig_capacity,
+                                  max_overlap_spans, levels)
     p, a = out.pair, out.agg
     rc = lib.argus_synthesize(_ptr(events), n, _ptr(stream_offsets), S, num_regions, _ptr(p.intervals), p.interval_capacity,
                               _ptr(p.interval_offsets), _ptr(p.ambig), p.ambig_capacity, _ptr(p.ambig_offsets), warps_per_cta,

@@ -50,14 +50,21 @@ extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t
   return syn_layout(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms, max_overlap_spans).total;
 }
 
-extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
-                                uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
-                                uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
-                                uint64_t ambig_capacity, uint64_t* ambig_offsets, uint32_t warps_per_cta,
-                                const uint32_t* cta_sm, uint32_t num_sms, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
-                                argus_agg_t* sm_tab, argus_agg_t* kernel_tab, const uint32_t* pairs, uint32_t num_pairs,
-                                argus_overlap_t* overlap_out, uint64_t max_overlap_spans, argus_status_t* status,
-                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+// implemented in argus_ring.cu
+int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
+                                uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream);
+
+// ring_written non-null: `events` is a ring container whose packed offsets are already in stream_offsets (device);
+// num_events then bounds the surviving records and the status block has been cleared by the caller.
+static int synthesize_impl(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                           uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                           uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                           uint64_t ambig_capacity, uint64_t* ambig_offsets, uint32_t warps_per_cta,
+                           const uint32_t* cta_sm, uint32_t num_sms, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                           argus_agg_t* sm_tab, argus_agg_t* kernel_tab, const uint32_t* pairs, uint32_t num_pairs,
+                           argus_overlap_t* overlap_out, uint64_t max_overlap_spans, argus_status_t* status,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream, const uint64_t* ring_written,
+                           uint32_t ring_capacity) {
   if (!status || !workspace || ((uintptr_t)workspace & 255)) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
@@ -77,7 +84,8 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
   f.pairs = pairs; f.num_pairs = num_pairs; f.ov_spans = nullptr; f.ov_seg = nullptr; f.ov_capacity = 0; f.ov_count = nullptr;
   // where aggregation and overlap selection happen: 0 = in the pairing kernel, 1 = in one pass over the
   // intervals after plain pairing, 2 = the plain calls
-  const bool can_fuse = num_streams > 0 && argus_pair_tiled_can_fuse(num_regions) && argus_pair_tiled_can_fuse_overlap(num_pairs);
+  const bool can_fuse = num_streams > 0 && !ring_written &&  // the kernel that reads rings has no hooks
+                        argus_pair_tiled_can_fuse(num_regions) && argus_pair_tiled_can_fuse_overlap(num_pairs);
   int mode = 2;
   if (num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs)) mode = 1;
   else if (can_fuse) mode = 0;
@@ -103,8 +111,9 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
   const bool use_digest = mode == 1 && L.digest_capacity != 0 && g_synth_mode != 3;
   int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
                                interval_offsets, ambig, ambig_capacity, ambig_offsets, status, ws + L.pair, L.pair_bytes,
-                               cuda_stream, 0, mode == 0 && (f.warp_tab || f.ov_spans) ? &f : nullptr, true, &fused,
-                               use_digest ? (uint64_t*)(ws + L.digest) : nullptr, L.digest_capacity);
+                               cuda_stream, ring_written ? 2 : 0, mode == 0 && (f.warp_tab || f.ov_spans) ? &f : nullptr,
+                               ring_written == nullptr, &fused, use_digest ? (uint64_t*)(ws + L.digest) : nullptr,
+                               L.digest_capacity, ring_written, ring_capacity);
   if (rc != ARGUS_OK) return rc;
   if (mode == 0 && !fused) mode = 2;  // the pairing front end chose a kernel without the hooks
 
@@ -132,4 +141,40 @@ extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events
     if (rc != ARGUS_OK) return rc;
   }
   return ARGUS_OK;
+}
+
+extern "C" int argus_synthesize(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
+                                uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
+                                uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
+                                uint64_t ambig_capacity, uint64_t* ambig_offsets, uint32_t warps_per_cta,
+                                const uint32_t* cta_sm, uint32_t num_sms, argus_agg_t* warp_tab, argus_agg_t* cta_tab,
+                                argus_agg_t* sm_tab, argus_agg_t* kernel_tab, const uint32_t* pairs, uint32_t num_pairs,
+                                argus_overlap_t* overlap_out, uint64_t max_overlap_spans, argus_status_t* status,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return synthesize_impl(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
+                         interval_offsets, ambig, ambig_capacity, ambig_offsets, warps_per_cta, cta_sm, num_sms, warp_tab, cta_tab,
+                         sm_tab, kernel_tab, pairs, num_pairs, overlap_out, max_overlap_spans, status, workspace, workspace_bytes,
+                         cuda_stream, nullptr, 0);
+}
+
+extern "C" int argus_synthesize_ring(const argus_event_t* ring, uint32_t slot_capacity, const uint64_t* written,
+                                     uint32_t num_streams, uint32_t num_regions, uint64_t* stream_offsets, uint64_t* dropped,
+                                     argus_interval_t* intervals, uint64_t interval_capacity, uint64_t* interval_offsets,
+                                     argus_ambiguity_t* ambig, uint64_t ambig_capacity, uint64_t* ambig_offsets,
+                                     uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, argus_agg_t* warp_tab,
+                                     argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab, const uint32_t* pairs,
+                                     uint32_t num_pairs, argus_overlap_t* overlap_out, uint64_t max_overlap_spans,
+                                     argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!status || !stream_offsets || slot_capacity == 0) return ARGUS_ERR_INVALID_ARG;
+  if (num_streams && (!ring || !written)) return ARGUS_ERR_INVALID_ARG;
+  if (((uintptr_t)written & 7) || ((uintptr_t)dropped & 7) || ((uintptr_t)stream_offsets & 7)) return ARGUS_ERR_INVALID_ARG;
+  ARGUS_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(argus_status_t), (cudaStream_t)cuda_stream));
+  const uint64_t bound = (uint64_t)num_streams * slot_capacity;  // what the slots can hold: sizes the workspace
+  const int rc = argus_internal_ring_offsets(written, slot_capacity, num_streams, bound, stream_offsets, dropped, status, cuda_stream);
+  if (rc != ARGUS_OK) return rc;
+  // without streams there is nothing to read from a ring: the plain path writes the empty results
+  return synthesize_impl(ring, bound, stream_offsets, num_streams, num_regions, intervals, interval_capacity, interval_offsets,
+                         ambig, ambig_capacity, ambig_offsets, warps_per_cta, cta_sm, num_sms, warp_tab, cta_tab, sm_tab,
+                         kernel_tab, pairs, num_pairs, overlap_out, max_overlap_spans, status, workspace, workspace_bytes,
+                         cuda_stream, num_streams ? written : nullptr, slot_capacity);
 }

@@ -115,3 +115,40 @@ def test_gpu_pairing_straight_from_the_ring(S, cap):
     assert pr.ambig_numpy().tobytes() == am.tobytes()
     assert np.array_equal(pr.interval_offsets.cpu().numpy().view(np.uint64), ioffs)
     assert np.array_equal(pr.ambig_offsets.cpu().numpy().view(np.uint64), aoffs)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode", [-1, 2, 3])
+def test_gpu_synthesize_straight_from_the_ring(mode):
+    """argus_synthesize_ring = linearise + argus_synthesize, in the modes that exist for a ring (digests, plain calls,
+    pass over the records)."""
+    import torch
+    import paper_2609_12299_b200 as argus
+    from paper_2609_12299_b200.binding import argus_set_synthesize_mode
+    rng = np.random.default_rng(99)
+    S, cap, R, W, M = 12, 3000, 5, 4, 3
+    streams = [random_wellformed(rng, int(rng.integers(0, 2 * cap)), R, max_height=5) for _ in range(S)]
+    ring, written = make_ring(streams, cap)
+    cta_sm = np.array([0, 2, 1], np.uint32)
+    pairs_np = np.array([(0, 1), (2, 2), (4, 3)], np.uint32)
+    rc, want, offs, dropped, st = oracle.ring_linearise(ring, cap, written)
+    rc, iv, ioffs, am, aoffs, o_st = oracle.pair(want, offs, R)
+    _, o_tabs, _ = oracle.aggregate(iv, ioffs, am, aoffs, W, cta_sm, M, R)
+    _, o_ov, _ = oracle.overlap(iv, ioffs, W, cta_sm, M, pairs_np)
+    d_ring = torch.from_numpy(ring.view(np.uint8).reshape(-1).copy()).to("cuda:0")
+    d_written = torch.from_numpy(written.view(np.int64).copy()).to("cuda:0")
+    d_cta_sm = torch.from_numpy(cta_sm.view(np.int32)).to("cuda:0")
+    d_pairs = torch.from_numpy(pairs_np.view(np.int32)).to("cuda:0")
+    argus_set_synthesize_mode(mode)
+    try:
+        res, d_offs, d_dropped = argus.argus_synthesize_ring(d_ring, cap, d_written, R, W, d_cta_sm, M, d_pairs)
+        assert int(res.fetch_status()["code"]) == 0
+    finally:
+        argus_set_synthesize_mode(-1)
+    assert np.array_equal(d_offs.cpu().numpy().view(np.uint64), offs)
+    assert np.array_equal(d_dropped.cpu().numpy().view(np.uint64), dropped)
+    assert res.pair.intervals_numpy().tobytes() == iv.tobytes()
+    assert res.pair.ambig_numpy().tobytes() == am.tobytes()
+    for lv in ("warp", "cta", "sm", "kernel"):
+        assert res.agg.table_numpy(lv).tobytes() == o_tabs[lv].tobytes(), lv
+    assert res.overlap_numpy(M).tobytes() == o_ov.tobytes()
