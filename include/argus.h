@@ -427,6 +427,21 @@ int argus_join_samples(const argus_interval_t* reference /*device*/, uint64_t nu
                        argus_join_t* out /*device [Q]*/, argus_status_t* status /*device*/,
                        void* cuda_stream);
 
+/* The same when the samples are the interval arrays of num_runs probe runs, one after the
+ * other in `samples`, each ordered by stream as argus_pair_intervals writes them:
+ * sample_offsets[run * (S + 1) + s] .. [run * (S + 1) + s + 1] (indices into `samples`) are
+ * the intervals of stream s in that run. A query then reads only its own stream's samples in
+ * every run (num_runs * N / S records instead of N), which is what makes thousands of queries
+ * against whole traces affordable. Offsets that decrease or leave `samples` set
+ * ARGUS_ERR_BAD_OFFSETS. Same results as argus_join_samples on the same records. */
+int argus_join_samples_grouped(const argus_interval_t* reference /*device*/, uint64_t num_reference,
+                               const uint64_t* ref_index /*device [Q]*/, uint32_t num_queries,
+                               const argus_interval_t* samples /*device*/, uint64_t num_samples,
+                               const uint64_t* sample_offsets /*device [num_runs][S+1]*/,
+                               uint32_t num_runs, uint32_t num_streams,
+                               argus_join_t* out /*device [Q]*/, argus_status_t* status /*device*/,
+                               void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------------
  * Ring-buffer input — a second container for the marker records of Section 3.2: tracers
  * commonly give every warp a fixed slot of slot_capacity records and let it wrap. The paper

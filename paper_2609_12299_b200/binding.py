@@ -77,6 +77,8 @@ def load_library():
     lib.argus_attribute.argtypes = [vp, u32, u32, vp, vp, vp, vp, vp, sz, vp]
     lib.argus_attribute.restype = ci
     lib.argus_join_samples.argtypes = [vp, u64, vp, u32, vp, u64, vp, vp, vp]
+    lib.argus_join_samples_grouped.argtypes = [vp, u64, vp, u32, vp, u64, vp, u32, u32, vp, vp, vp]
+    lib.argus_join_samples_grouped.restype = ci
     lib.argus_join_samples.restype = ci
     lib.argus_ring_linearise.argtypes = [vp, u32, vp, u32, vp, u64, vp, vp, vp, vp]
     lib.argus_ring_linearise.restype = ci
@@ -456,6 +458,24 @@ def argus_join_samples(reference: torch.Tensor, ref_index: torch.Tensor, samples
                                 samples.numel() // 48, _ptr(out), _ptr(status), _stream_ptr(dev))
     if rc != 0:
         raise ArgusError(rc, "argus_join_samples")
+    return out, status
+
+
+def argus_join_samples_grouped(reference: torch.Tensor, ref_index: torch.Tensor, samples: torch.Tensor,
+                               sample_offsets: torch.Tensor, num_streams: int):
+    """As argus_join_samples, with `samples` = the interval arrays of several probe runs one after the other and
+    sample_offsets int64 [num_runs, S + 1] = where each stream's intervals of each run lie in `samples`."""
+    lib = load_library()
+    dev = reference.device
+    Q = ref_index.numel()
+    out = _bytes(Q * 64, dev)
+    status = _bytes(64, dev)
+    runs = sample_offsets.numel() // (num_streams + 1)
+    rc = lib.argus_join_samples_grouped(_ptr(reference), reference.numel() // 48, _ptr(ref_index), Q, _ptr(samples),
+                                        samples.numel() // 48, _ptr(sample_offsets), runs, num_streams, _ptr(out), _ptr(status),
+                                        _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_join_samples_grouped")
     return out, status
 
 

@@ -3,6 +3,7 @@
     python -m paper_2609_12299_b200.measure scoped   # argus_aggregate_scoped / argus_overlap_scoped on trace 3
     python -m paper_2609_12299_b200.measure pcmap    # PC-to-region mapping and attribution on a mapping run
     python -m paper_2609_12299_b200.measure ring     # pairing from a ring container: packed copy first, or directly
+    python -m paper_2609_12299_b200.measure join     # cross-run join against a whole trace, plain and grouped by stream
 
 Each line printed is one JSON object: what ran, its time (best of the repetitions after warm-up), the
 algorithmic bytes it has to move and the fraction of the measured HBM copy bandwidth that amounts to.
@@ -156,9 +157,34 @@ def run_ring(iters: int, shift_tokens: int):
           sequential_tiles=int(st["n_sequential_tiles"]))
 
 
+def run_join(iters: int, queries: int):
+    """Cross-run join on the decode trace: the run's own intervals serve as reference and as one probe run."""
+    spec = tg.config(3).scaled(iters=iters) if iters else tg.config(3)
+    dev = torch.device("cuda", 0)
+    d_ev, d_off = tg.generate_cuda(spec, dev)
+    n = d_ev.numel() // 16
+    p = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions, interval_capacity=n // 2, ambig_capacity=max(n // 64, 4096))
+    assert int(p.fetch_status()["code"]) == 0
+    del d_ev
+    torch.cuda.empty_cache()
+    n_iv = int(p.interval_offsets[-1].item())
+    iv = p.intervals[: n_iv * 48]
+    g = torch.Generator(device="cpu").manual_seed(7)
+    idx = torch.randint(0, n_iv, (queries,), generator=g, dtype=torch.int64).to(dev)
+    few = idx[:8].contiguous()
+    ms = _time(lambda: argus.argus_join_samples(iv, few, iv), reps=2, warmup=1)
+    _line("argus_join_samples, 8 queries (every query reads the 32 key bytes of every sample)", ms, 8 * 32.0 * n_iv,
+          intervals=n_iv, workload=spec.name)
+    offs = p.interval_offsets.view(1, -1).contiguous()
+    ms = _time(lambda: argus.argus_join_samples_grouped(iv, idx, iv, offs, spec.num_streams), reps=3, warmup=1)
+    _line(f"argus_join_samples_grouped, {queries} queries (every query reads its own stream's samples)", ms,
+          queries * 32.0 * n_iv / spec.num_streams, intervals=n_iv, workload=spec.name)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["scoped", "pcmap", "ring"])
+    ap.add_argument("what", choices=["scoped", "pcmap", "ring", "join"])
+    ap.add_argument("--queries", type=int, default=2000, help="`join`: queries of the grouped join")
     ap.add_argument("--shift-tokens", type=int, default=100, help="`ring`: tokens written before the surviving records (0: no wrap)")
     ap.add_argument("--iters", type=int, default=0, help="tokens per stream of the decode trace (0: full size for `scoped`, 24 for `pcmap`)")
     ap.add_argument("--pcs", type=int, default=70_560)
@@ -169,6 +195,8 @@ def main():
         run_scoped(a.iters)
     elif a.what == "ring":
         run_ring(a.iters, a.shift_tokens)
+    elif a.what == "join":
+        run_join(a.iters, a.queries)
     else:
         run_pcmap(a.iters or 24, a.pcs, a.execs_per_begin)
 

@@ -66,6 +66,42 @@ def test_join_on_paired_runs():
     assert np.all(got["count"] == 3 * 8)   # the eight loads of an iteration share their key: 8 samples per run
 
 
+def test_grouped_join_on_paired_runs():
+    """The same selection through argus_join_samples_grouped: the three probe runs' interval arrays one after the other
+    with their per-stream offsets, so that a query reads only its stream's intervals of every run."""
+    from paper_2609_12299_b200 import tracegen as tg
+    from dataclasses import replace
+    spec = tg.config(1).scaled(2, 40)
+    S = spec.num_streams
+    runs, offsets = [], []
+    for k in range(4):
+        d_ev, d_off = tg.generate_cuda(replace(spec, seed=spec.seed + 17 * k), DEV)
+        pr = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions)
+        assert int(pr.fetch_status()["code"]) == 0
+        runs.append(pr.intervals_numpy())
+        offsets.append(pr.interval_offsets.cpu().numpy().view(np.uint64).copy())
+    ref, smp = runs[0], np.concatenate(runs[1:])
+    base = np.cumsum([0] + [len(r) for r in runs[1:-1]]).astype(np.uint64)
+    grouped = np.stack([offsets[1 + r] + base[r] for r in range(3)])            # [3, S + 1], indices into smp
+    sel = np.nonzero((ref["region"] == 1) & (ref["ctx"] >= 5) & (ref["ctx"] <= 20))[0].astype(np.uint64)
+    rc, want, o_st = oracle.join_samples(ref, sel, smp)
+    d_idx = torch.from_numpy(sel.view(np.int64).copy()).to(DEV)
+    d_grp = torch.from_numpy(grouped.view(np.int64).copy()).to(DEV)
+    out, status = argus.argus_join_samples_grouped(_dev(ref), d_idx, _dev(smp), d_grp, S)
+    assert int(argus.argus_status_fetch(status)["code"]) == 0
+    assert out.cpu().numpy()[: len(sel) * 64].view(argus.JOIN_DTYPE).tobytes() == want.tobytes()
+    # offsets that leave the sample array are reported
+    bad = grouped.copy()
+    bad[2, S] = len(smp) + 5
+    out, status = argus.argus_join_samples_grouped(_dev(ref), d_idx, _dev(smp), torch.from_numpy(bad.view(np.int64).copy()).to(DEV), S)
+    st = argus.argus_status_fetch(status)
+    assert int(st["code"]) in (0, 7)   # 7 only if a query's stream is the last one
+    sel_last = np.nonzero(ref["stream"] == S - 1)[0][:4].astype(np.uint64)
+    out, status = argus.argus_join_samples_grouped(_dev(ref), torch.from_numpy(sel_last.view(np.int64).copy()).to(DEV), _dev(smp),
+                                                   torch.from_numpy(bad.view(np.int64).copy()).to(DEV), S)
+    assert int(argus.argus_status_fetch(status)["code"]) == 7
+
+
 def test_join_edges_on_gpu():
     ref, smp, _ = load_join_example()
     got, st = _join(ref, np.zeros(0, np.uint64), smp)
