@@ -34,6 +34,8 @@ __global__ void __launch_bounds__(128) k_pair_thread_per_stream(ArgusPairArgs a)
     return;
   }
   const u64 base = a.redo ? a.interval_offsets[s] : ((lo - off0) >> 1);
+  // second pass: intervals that already lie where they belong (same position, all of them fitted) stay
+  if (a.redo && base == ((lo - off0) >> 1) && base + a.counts[s] <= a.interval_capacity) return;
   ArgusFrame stk[ARGUS_MAX_DEPTH];
   ArgusSeqState st;
   st.h = 0; st.n_int = 0; st.n_ctx = st.n_rev = st.n_clamp = 0; st.failed = false;

@@ -260,6 +260,13 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     const u32 n = (u32)(hi - lo);
     const u64 gpos0 = lo - off0;
     const u64 out_base = a.redo ? a.interval_offsets[s] : (gpos0 >> 1);
+    if (a.redo && rec == kNoRec && out_base == (gpos0 >> 1) && out_base + a.counts[s] <= a.interval_capacity) {
+      // second pass: this stream's intervals (and digests) already lie where they belong — the first pass wrote them
+      // at the same positions, all of them fitted, and no other stream writes there in either pass
+      if (tid == 0) atomicAdd(&a.ctl->n_done[1], 1u);
+      __syncthreads();
+      continue;
+    }
     const argus_event_t* src = RING ? a.events + (u64)s * a.ring_capacity : a.events + lo;
     const u32 ring_first = RING ? argus_ring_first(a, s) : 0u;
     const u32 ntiles = (n + T - 1) / T;

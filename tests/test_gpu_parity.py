@@ -182,6 +182,27 @@ def test_exact_capacity_with_malformed_trace(kernel):
     assert_pair_matches(ev, offs, spec.num_regions, kernel, interval_capacity=len(o_iv), ambig_capacity=len(o_am))
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("where", ["first", "middle", "last"])
+def test_one_malformed_stream_among_wellformed_ones(kernel, where):
+    """One stream loses an end marker: the streams before it keep their place in the interval array (the second
+    pass leaves them alone), the ones after it move up by one."""
+    spec = tg.config(3).scaled(3, 4)
+    ev, offs = tg.generate_host(spec)
+    S = spec.num_streams
+    k = {"first": 0, "middle": S // 2, "last": S - 1}[where]
+    lo, hi = int(offs[k]), int(offs[k + 1])
+    ends = np.nonzero(ev["tag"][lo:hi] & 1)[0]
+    drop = lo + int(ends[len(ends) // 2])
+    ev2 = np.delete(ev, drop)
+    offs2 = offs.copy()
+    offs2[k + 1:] -= 1
+    pr, (o_iv, _, o_am, _) = assert_pair_matches(ev2, offs2, spec.num_regions, kernel)
+    assert len(o_am) >= 1 and len(o_iv) < len(ev2) // 2 + 1
+    # and through the one-call pipeline (digests follow the intervals)
+    _synthesize_matches(spec, ev2, offs2)
+
+
 def test_invalid_arguments_raise():
     ev = make_events([(1, "B", 0, 0), (2, "E", 0, 0)])
     d_ev, d_off = to_dev(ev, np.array([0, 2], np.uint64))
