@@ -59,6 +59,13 @@ struct AggArgs {
 
 constexpr u32 kAggOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
 
+// The slots of a reserved chunk that the warp leaves unused are tagged, so that the list needs no clearing
+// (a warp that holds no chunk has used == kAggOvChunk: nothing to tag).
+__device__ __forceinline__ void agg_ov_retire(const ArgusFuseArgs& ov, u64 base, u32 used, u32 lane) {
+  for (u32 i = used + lane; i < kAggOvChunk; i += 32)
+    if (base + i < ov.ov_capacity) ov.ov_seg[base + i] = 0xffffffffu;
+}
+
 __device__ __forceinline__ bool mask_bit(const u32* mask, u32 i) { return !mask || ((mask[i >> 5] >> (i & 31)) & 1u); }
 
 // Warp-role and SM tests of a scope: one answer per stream. 2 = bad cta_sm entry.
@@ -223,6 +230,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
             if (!bal) continue;
             const u32 c = __popc(bal);
             if (ovc_used + c > kAggOvChunk) {
+              agg_ov_retire(a.ov, ovc_base, ovc_used, lane);
               u64 nb64 = 0;
               if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)kAggOvChunk);
               ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
@@ -255,6 +263,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
     argus_fuse_flush(ctab, row, R, threadIdx.x, blockDim.x);
     __syncthreads();
   }
+  if (has_ov) agg_ov_retire(a.ov, ovc_base, ovc_used, lane);
 }
 
 // ---- the pass over the intervals' 8-byte digests (what argus_synthesize's pairing wrote beside the records) ----
@@ -453,6 +462,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
               if (!bal) continue;
               const u32 c = __popc(bal);
               if (ovc_used + c > kAggOvChunk) {
+                agg_ov_retire(a.ov, ovc_base, ovc_used, lane);
                 u64 nb64 = 0;
                 if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)kAggOvChunk);
                 ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
@@ -533,6 +543,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
     }
     __syncthreads();
   }
+  if (has_ov) agg_ov_retire(a.ov, ovc_base, ovc_used, lane);
 }
 
 __device__ __forceinline__ u64 combine(u32 field, u64 x, u64 y) {

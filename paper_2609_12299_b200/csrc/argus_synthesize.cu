@@ -105,7 +105,9 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
     f.ov_capacity = max_overlap_spans;
     f.ov_count = (u64*)(ws + L.list_count);
     ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_count, 0, 256, stream));
-    ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)max_overlap_spans * 4 + 4, stream));
+    // the pairing kernel's hooks leave unused slots of their chunks untouched: those must read as "no span"; the
+    // aggregation passes tag them themselves
+    if (mode == 0) ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)max_overlap_spans * 4 + 4, stream));
   }
   bool fused = false;
   const bool use_digest = mode == 1 && L.digest_capacity != 0 && g_synth_mode != 3;
