@@ -57,12 +57,11 @@ struct AggArgs {
   u64 interval_limit; // records the interval array holds: a stream whose offsets reach beyond it is reported, not read
 };
 
-constexpr u32 kAggOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
 
 // The slots of a reserved chunk that the warp leaves unused are tagged, so that the list needs no clearing
-// (a warp that holds no chunk has used == kAggOvChunk: nothing to tag).
+// (a warp that holds no chunk has used == the chunk size: nothing to tag).
 __device__ __forceinline__ void agg_ov_retire(const ArgusFuseArgs& ov, u64 base, u32 used, u32 lane) {
-  for (u32 i = used + lane; i < kAggOvChunk; i += 32)
+  for (u32 i = used + lane; i < ov.ov_chunk; i += 32)
     if (base + i < ov.ov_capacity) ov.ov_seg[base + i] = 0xffffffffu;
 }
 
@@ -170,7 +169,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
   u64* const iter_base = !a.iter_inline ? nullptr
                          : a.iter_copies ? a.iter_copies + (u64)(blockIdx.x % a.num_copies) * a.num_iters * cells : a.iter_tab;
   u64 ovc_base = 0;             // warp-uniform: current chunk of the global span list
-  u32 ovc_used = kAggOvChunk;
+  u32 ovc_used = a.ov.ov_chunk;  // none held yet
   if (has_ov) {
     for (u32 i = threadIdx.x; i < (R + 31) / 32; i += blockDim.x) pairbits[i] = 0;
     __syncthreads();
@@ -229,10 +228,10 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_compact(AggArgs a) 
             const u32 bal = __ballot_sync(0xffffffffu, pick);
             if (!bal) continue;
             const u32 c = __popc(bal);
-            if (ovc_used + c > kAggOvChunk) {
+            if (ovc_used + c > a.ov.ov_chunk) {
               agg_ov_retire(a.ov, ovc_base, ovc_used, lane);
               u64 nb64 = 0;
-              if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)kAggOvChunk);
+              if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)a.ov.ov_chunk);
               ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
               ovc_used = 0;
             }
@@ -332,7 +331,7 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
   const u32 lane = threadIdx.x & 31;
   const bool has_ov = a.ov.ov_spans != nullptr && a.ov.num_pairs != 0;
   u64 ovc_base = 0;
-  u32 ovc_used = kAggOvChunk;
+  u32 ovc_used = a.ov.ov_chunk;  // none held yet
   for (u32 i = threadIdx.x; i < (R + 31) / 32; i += blockDim.x) pairbits[i] = 0;
   __syncthreads();
   if (has_ov) {
@@ -461,10 +460,10 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
               const u32 bal = __ballot_sync(0xffffffffu, pick);
               if (!bal) continue;
               const u32 c = __popc(bal);
-              if (ovc_used + c > kAggOvChunk) {
+              if (ovc_used + c > a.ov.ov_chunk) {
                 agg_ov_retire(a.ov, ovc_base, ovc_used, lane);
                 u64 nb64 = 0;
-                if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)kAggOvChunk);
+                if (lane == 0) nb64 = atomicAdd(a.ov.ov_count, (u64)a.ov.ov_chunk);
                 ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
                 ovc_used = 0;
               }
@@ -738,7 +737,7 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
   a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
   a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0; a.iter_copies = nullptr; a.num_copies = 0;
   a.iter_inline = 0;
-  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.digest = nullptr; a.interval_limit = ~0ull;
+  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.ov.ov_chunk = 256; a.digest = nullptr; a.interval_limit = ~0ull;
   if (ambig && ambig_offsets) {
     k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
     ARGUS_CHECK_LAUNCH();
@@ -792,7 +791,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   a.warp_mask = scope ? scope->warp_mask : ~0ull;
   a.sm_mask = scope ? scope->sm_mask : nullptr; a.region_mask = scope ? scope->region_mask : nullptr;
   a.role_tab = (u64*)role_tab; a.iter_tab = (u64*)iter_tab; a.num_iters = num_iters;
-  if (ov_select) { a.ov = *ov_select; } else { a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; }
+  if (ov_select) { a.ov = *ov_select; } else { a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.ov.ov_chunk = 256; }
   a.digest = !scope && !role_tab && !iter_tab && num_regions <= kAggCompactRegions ? (const u64*)digest : nullptr;
   a.interval_limit = interval_limit;
   const size_t smem = (size_t)num_regions * sizeof(argus_agg_t);

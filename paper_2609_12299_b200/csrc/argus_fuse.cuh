@@ -33,6 +33,7 @@ struct ArgusFuseArgs {
   ulonglong2* ov_spans;   // appended (start, end); null = no fused overlap selection
   u32* ov_seg;            // segment of each appended span: (pair * num_sms + sm) * 2 + role
   u64 ov_capacity;
+  u32 ov_chunk;           // list slots a warp reserves at a time: a power of two from 32 to 256
   u64* ov_count;          // spans appended so far (may exceed the capacity)
 };
 

@@ -166,7 +166,6 @@ __device__ __forceinline__ int tile_latest_begin(const TileSmem<NT, E>& sm, int 
   return valid ? r : -1;
 }
 
-constexpr u32 kOvChunk = 256;  // overlap spans a warp reserves from the global list at a time
 
 // One tile of a stream into shared memory: a bulk copy, or two when the stream lives in a ring slot and the
 // tile straddles the slot's end. `src` is the stream's first record (packed input) or its slot (ring).
@@ -216,7 +215,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   u64* row = nullptr;      // global row of the current stream in the warp-scope table
   u32 sm_index = 0;        // SM of the current stream's CTA
   u64 ovc_base = 0;        // warp-uniform: current chunk of the global overlap span list
-  u32 ovc_used = kOvChunk;
+  u32 ovc_used = a.fuse.ov_chunk;  // list slots a warp reserves at a time; none held yet
   u32 hot0 = 0xffffffffu, hot1 = 0xffffffffu;  // hot regions of the current stream, private partial sums
   u64 hsi0 = 0, hsi1 = 0, hse0 = 0, hse1 = 0;
   if (has_pairs) {
@@ -523,9 +522,9 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
                 const u32 bal = __ballot_sync(0xffffffffu, sel);
                 if (!bal) continue;
                 const u32 c = __popc(bal);
-                if (ovc_used + c > kOvChunk) {
+                if (ovc_used + c > a.fuse.ov_chunk) {
                   u64 nb64 = 0;
-                  if (lane == 0) nb64 = atomicAdd(a.fuse.ov_count, (u64)kOvChunk);
+                  if (lane == 0) nb64 = atomicAdd(a.fuse.ov_count, (u64)a.fuse.ov_chunk);
                   ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
                   ovc_used = 0;
                 }

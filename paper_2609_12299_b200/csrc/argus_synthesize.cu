@@ -15,7 +15,8 @@ int g_synth_mode = -1;  // -1 = automatic
 
 struct SynLayout {
   size_t pair, pair_bytes, agg, agg_bytes, list_count, list_seg, list_spans, ov, ov_bytes, digest, total;
-  uint64_t digest_capacity;
+  uint64_t digest_capacity, list_capacity, list_slack;
+  uint32_t list_chunk;
 };
 
 SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_regions, uint64_t ambig_capacity,
@@ -24,9 +25,17 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
   size_t o = 0;
   L.pair = o; L.pair_bytes = argus_pair_workspace_bytes(num_events, num_streams, ambig_capacity); o += argus_align_up(L.pair_bytes, 256);
   L.agg = o; L.agg_bytes = argus_aggregate_workspace_bytes(num_events / 2, num_streams, num_regions); o += argus_align_up(L.agg_bytes, 256);
+  // The span list: warps reserve slots in chunks and leave some unused, so the list is longer than the spans it
+  // may hold, by a quarter or by one smallest chunk for every warp that can append, whichever is more
+  // (one block of 8 warps per stream in the aggregation passes; at most 148 x 8 blocks of 10 in the pairing kernel).
+  const uint64_t warps = (uint64_t)num_streams * 8 > 148ull * 8 * 10 ? (uint64_t)num_streams * 8 : 148ull * 8 * 10;
+  L.list_slack = num_pairs ? (max_overlap_spans / 4 > warps * 32 ? max_overlap_spans / 4 : warps * 32) : 0;
+  L.list_chunk = 256;
+  while (L.list_chunk > 32 && warps * L.list_chunk > L.list_slack) L.list_chunk >>= 1;
+  L.list_capacity = max_overlap_spans + L.list_slack;
   L.list_count = o; o += 256;
-  L.list_seg = o; o += argus_align_up((size_t)max_overlap_spans * 4 + 4, 256);
-  L.list_spans = o; o += argus_align_up((size_t)max_overlap_spans * 16 + 16, 256);
+  L.list_seg = o; o += argus_align_up((size_t)L.list_capacity * 4 + 4, 256);
+  L.list_spans = o; o += argus_align_up((size_t)L.list_capacity * 16 + 16, 256);
   L.ov = o;
   L.ov_bytes = argus_align_up((size_t)num_pairs * num_sms * 2 * 8 * 3 + 1024 + (size_t)max_overlap_spans * 24 + 256, 256);
   o += L.ov_bytes;
@@ -81,7 +90,7 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
 
   ArgusFuseArgs f;
   f.warp_tab = nullptr; f.cta_sm = cta_sm; f.warps_per_cta = warps_per_cta; f.num_sms = num_sms;
-  f.pairs = pairs; f.num_pairs = num_pairs; f.ov_spans = nullptr; f.ov_seg = nullptr; f.ov_capacity = 0; f.ov_count = nullptr;
+  f.pairs = pairs; f.num_pairs = num_pairs; f.ov_spans = nullptr; f.ov_seg = nullptr; f.ov_capacity = 0; f.ov_count = nullptr; f.ov_chunk = L.list_chunk;
   // where aggregation and overlap selection happen: 0 = in the pairing kernel, 1 = in one pass over the
   // intervals after plain pairing, 2 = the plain calls
   const bool can_fuse = num_streams > 0 && !ring_written &&  // the kernel that reads rings has no hooks
@@ -102,12 +111,12 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
   if (list) {
     f.ov_spans = (ulonglong2*)(ws + L.list_spans);
     f.ov_seg = (u32*)(ws + L.list_seg);
-    f.ov_capacity = max_overlap_spans;
+    f.ov_capacity = L.list_capacity;
     f.ov_count = (u64*)(ws + L.list_count);
     ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_count, 0, 256, stream));
     // the pairing kernel's hooks leave unused slots of their chunks untouched: those must read as "no span"; the
     // aggregation passes tag them themselves
-    if (mode == 0) ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)max_overlap_spans * 4 + 4, stream));
+    if (mode == 0) ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)L.list_capacity * 4 + 4, stream));
   }
   bool fused = false;
   const bool use_digest = mode == 1 && L.digest_capacity != 0 && g_synth_mode != 3;

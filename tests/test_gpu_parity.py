@@ -411,6 +411,26 @@ def test_synthesize_overlap_span_capacity():
     assert int(st["code"]) == 4 and int(st["intervals_required"]) > 512
 
 
+@pytest.mark.parametrize("idx,ctas,iters", [(0, 4, 626), (1, 7, 300), (2, 3, 3), (3, 3, 9), (4, 9, 400)])
+def test_outputs_repeat_byte_for_byte(idx, ctas, iters):
+    """The same call twice on fresh buffers: every output byte is the same (all device-side accumulation is integer
+    atomics, ranks come from prefix sums, spans are sorted before they are measured)."""
+    spec = tg.config(idx).scaled(ctas, iters)
+    ev, offs = tg.generate_host(spec)
+    d_ev, d_off = to_dev(ev, offs)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(DEV)
+    runs = []
+    for _ in range(2):
+        res = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, pairs)
+        assert int(res.fetch_status()["code"]) == 0
+        runs.append([res.pair.intervals_numpy().tobytes(), res.pair.ambig_numpy().tobytes(),
+                     res.pair.interval_offsets.cpu().numpy().tobytes(), res.pair.ambig_offsets.cpu().numpy().tobytes(),
+                     res.overlap.cpu().numpy().tobytes(), res.status.cpu().numpy().tobytes()] +
+                    [res.agg.table_numpy(lv).tobytes() for lv in ("warp", "cta", "sm", "kernel")])
+    assert runs[0] == runs[1]
+
+
 def test_synthesize_interval_capacity_too_small(synth_mode):
     """Fewer interval slots than the trace needs: the call reports ARGUS_ERR_CAPACITY with the required count, the
     later stages read nothing beyond the array, and the same buffers work again with enough room."""
