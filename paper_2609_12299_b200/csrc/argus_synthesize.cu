@@ -37,7 +37,9 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
   L.list_seg = o; o += argus_align_up((size_t)L.list_capacity * 4 + 4, 256);
   L.list_spans = o; o += argus_align_up((size_t)L.list_capacity * 16 + 16, 256);
   L.ov = o;
-  L.ov_bytes = argus_align_up((size_t)num_pairs * num_sms * 2 * 8 * 3 + 1024 + (size_t)max_overlap_spans * 24 + 256, 256);
+  // segment counters and the sorted spans (24 B each); a little more, so that the plain overlap call, which gets the
+  // list's room and this as one workspace and splits it itself (50.7 B a span), also holds max_overlap_spans
+  L.ov_bytes = argus_align_up((size_t)num_pairs * num_sms * 2 * 8 * 3 + 1024 + (size_t)max_overlap_spans * 27 + 4096, 256);
   o += L.ov_bytes;
   // one digest per interval (a stream's intervals start at half its first event's position at the latest)
   L.digest_capacity = argus_aggregate_can_select_overlap(num_regions, num_pairs) ? num_events / 2 + 1 : 0;
@@ -147,7 +149,8 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
                                             status, ws + L.ov, L.ov_bytes, cuda_stream);
     } else {
       rc = argus_internal_overlap(intervals, interval_capacity, interval_offsets, num_streams, warps_per_cta, cta_sm, num_sms,
-                                  pairs, num_pairs, overlap_out, status, ws + L.ov, L.ov_bytes, cuda_stream, false);
+                                  pairs, num_pairs, overlap_out, status, ws + L.list_count, L.ov + L.ov_bytes - L.list_count,
+                                  cuda_stream, false);
     }
     if (rc != ARGUS_OK) return rc;
   }

@@ -431,6 +431,57 @@ def test_outputs_repeat_byte_for_byte(idx, ctas, iters):
     assert runs[0] == runs[1]
 
 
+def _fuzz_case(seed):
+    """A random trace shape: stream count, region count, SM map, pairs; streams of random length, some empty, some
+    corrupted (dropped and duplicated markers, flipped kinds, changed regions, time running backwards, huge gaps)."""
+    rng = np.random.default_rng(1000 + seed)
+    W = int(rng.choice([1, 2, 4, 8, 16]))
+    C = int(rng.integers(1, 7))
+    S = W * C
+    R = int(rng.choice([1, 2, 5, 37, 300, 500]))
+    M = int(rng.integers(1, 5))
+    evs, offs = [], [0]
+    for s in range(S):
+        kind = rng.random()
+        n_pairs = 0 if kind < 0.1 else int(rng.integers(1, 1500 if kind < 0.9 else 12000))
+        ev = random_wellformed(rng, n_pairs, R, max_height=int(rng.integers(1, 9)), t0=int(rng.integers(0, 1 << 45)))
+        if len(ev) and rng.random() < 0.5:      # corrupt it
+            n = len(ev)
+            keep = rng.random(n) > 0.003
+            ev = ev[keep]
+            n = len(ev)
+            if n:
+                flip = rng.random(n) < 0.002
+                ev["tag"][flip] ^= 1
+                chg = rng.random(n) < 0.002
+                ev["tag"][chg] = (rng.integers(0, R, int(chg.sum())).astype(np.uint32) << 1) | (ev["tag"][chg] & 1)
+                back = rng.random(n) < 0.002
+                ev["ts"][back] -= np.minimum(ev["ts"][back], rng.integers(1, 1000, int(back.sum())).astype(np.uint64))
+                jump = rng.random(n) < 0.001
+                ev["ts"] += np.cumsum(np.where(jump, rng.integers(1 << 30, 1 << 40, n), 0)).astype(np.uint64)
+                dup = np.nonzero(rng.random(n) < 0.002)[0]
+                ev = np.insert(ev, dup, ev[dup])
+        evs.append(ev)
+        offs.append(offs[-1] + len(ev))
+    K = int(rng.integers(0, 5))
+
+    class Spec:
+        num_regions, warps_per_cta, num_sms = R, W, M
+        cta_sm = rng.integers(0, M, C).astype(np.uint32)
+        overlap_pairs = rng.integers(0, R, (K, 2)).astype(np.uint32)
+    ev = np.concatenate(evs) if evs else np.zeros(0, argus.EVENT_DTYPE)
+    return Spec, ev.astype(argus.EVENT_DTYPE), np.array(offs, np.uint64)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_synthesize_random_shapes(seed, synth_mode):
+    spec, ev, offs = _fuzz_case(seed)
+    rc, _, _, _, _, o_st = oracle.pair(ev, offs, spec.num_regions)
+    if int(o_st["code"]) != 0:
+        pytest.skip("the random corruption opened more than 64 frames")
+    _synthesize_matches(spec, ev, offs)
+
+
 def test_synthesize_interval_capacity_too_small(synth_mode):
     """Fewer interval slots than the trace needs: the call reports ARGUS_ERR_CAPACITY with the required count, the
     later stages read nothing beyond the array, and the same buffers work again with enough room."""
