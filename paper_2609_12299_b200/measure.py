@@ -155,6 +155,16 @@ def run_ring(iters: int, shift_tokens: int):
     assert int(st["code"]) == 0, st
     _line("argus_pair_intervals_ring (allocations included)", ms1, 40.0 * n, events=n, workload=spec.name, shift_records=shift,
           sequential_tiles=int(st["n_sequential_tiles"]))
+    del pr
+    torch.cuda.empty_cache()
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(dev)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(dev)
+    kw = dict(interval_capacity=n // 2, ambig_capacity=max(n // 64, 4096), max_overlap_spans=n // 8)
+    ms3 = _time(lambda: argus.argus_synthesize_ring(d_ev, cap, written, R, spec.warps_per_cta, cta_sm, spec.num_sms, pairs, **kw),
+                reps=3, warmup=1)
+    res, _, _ = argus.argus_synthesize_ring(d_ev, cap, written, R, spec.warps_per_cta, cta_sm, spec.num_sms, pairs, **kw)
+    assert int(res.fetch_status()["code"]) == 0
+    _line("argus_synthesize_ring (allocations included)", ms3, 40.0 * n, events=n, workload=spec.name, shift_records=shift)
 
 
 def run_join(iters: int, queries: int):
