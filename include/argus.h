@@ -561,6 +561,15 @@ unsigned long long argus_launch_count(void);
 void argus_profile_enable(int on);
 int argus_profile_read(double* ms_total /*host [4]*/, unsigned long long* launches /*host [4]*/);
 
+/* Tuning and test aids (process-wide; results never depend on them).
+ * argus_set_synthesize_mode: where argus_synthesize aggregates and selects overlap spans: -1 automatic,
+ * 0 inside the pairing kernel, 1 in one pass over the intervals' digests, 2 the three plain operations,
+ * 3 in one pass over the interval records. A mode the inputs do not allow falls back to the automatic choice.
+ * argus_set_tile_variant: shape of the tiled pairing kernel, 0 = automatic, 1..5 = the other compiled
+ * shapes <threads, events per thread, blocks per SM>: <192,5,4>, <320,5,2>, <64,5,8>, <256,7,2>, <160,5,5>. */
+void argus_set_synthesize_mode(int mode);
+void argus_set_tile_variant(int variant);
+
 #ifdef __cplusplus
 }
 #endif
