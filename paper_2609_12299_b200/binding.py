@@ -268,7 +268,8 @@ class AggregateResult:
 
     def table_numpy(self, level: str) -> np.ndarray:
         t = getattr(self, level)
-        return t.cpu().numpy().view(AGG_DTYPE).reshape(self.shape[level])
+        keys, regions = self.shape[level]
+        return t[: keys * regions * 576].cpu().numpy().view(AGG_DTYPE).reshape(self.shape[level])  # (a table without keys is empty)
 
 
 def argus_aggregate(intervals: torch.Tensor, interval_offsets: torch.Tensor, ambig: torch.Tensor | None,

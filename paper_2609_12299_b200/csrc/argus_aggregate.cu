@@ -761,7 +761,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
   if (ov_select && (num_regions > kAggCompactRegions || ov_select->num_pairs > kFuseMaxPairs)) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
-  if ((sm_tab || (scope && scope->sm_mask)) && (!cta_sm || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
+  if ((sm_tab || (scope && scope->sm_mask)) && ((!cta_sm && num_streams) || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
   if (scope && scope->ctx_hi < scope->ctx_lo) return ARGUS_ERR_INVALID_ARG;
   if (iter_tab && (!scope || scope->ctx_hi - scope->ctx_lo >= ARGUS_MAX_ITER_ROWS)) return ARGUS_ERR_INVALID_ARG;
   if (((uintptr_t)intervals & 15) || ((uintptr_t)workspace & 255) || ((uintptr_t)warp_tab & 7) || ((uintptr_t)cta_tab & 7) ||

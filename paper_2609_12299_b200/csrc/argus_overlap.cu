@@ -435,7 +435,7 @@ static int overlap_scoped(const argus_interval_t* intervals, uint64_t max_interv
                           const uint32_t* pairs, uint32_t num_pairs, const argus_scope_t* scope, argus_overlap_t* out,
                           argus_status_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream,
                           bool reset_status) {
-  if (!interval_offsets || !cta_sm || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
+  if (!interval_offsets || (!cta_sm && num_streams) || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if (scope && scope->ctx_hi < scope->ctx_lo) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0 || num_sms == 0) return ARGUS_ERR_INVALID_ARG;
   if (num_pairs > kMaxPairs || (num_pairs && (!pairs || !out))) return ARGUS_ERR_INVALID_ARG;

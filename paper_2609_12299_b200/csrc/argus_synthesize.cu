@@ -79,7 +79,7 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
   if (!status || !workspace || ((uintptr_t)workspace & 255)) return ARGUS_ERR_INVALID_ARG;
   if (warps_per_cta == 0 || num_streams % warps_per_cta != 0) return ARGUS_ERR_INVALID_ARG;
   if (num_regions == 0 || num_regions > ARGUS_MAX_REGIONS) return ARGUS_ERR_INVALID_ARG;
-  if ((sm_tab || num_pairs) && (!cta_sm || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
+  if ((sm_tab || num_pairs) && ((!cta_sm && num_streams) || num_sms == 0)) return ARGUS_ERR_INVALID_ARG;
   if (num_pairs && (!pairs || !overlap_out)) return ARGUS_ERR_INVALID_ARG;
   const SynLayout L = syn_layout(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms, max_overlap_spans);
   if (workspace_bytes < L.total) return ARGUS_ERR_WORKSPACE;

@@ -482,6 +482,19 @@ def test_synthesize_random_shapes(seed, synth_mode):
     _synthesize_matches(spec, ev, offs)
 
 
+def test_synthesize_empty_inputs(synth_mode):
+    """Streams without events, and no streams at all: empty outputs, zeroed tables, status clean."""
+    spec = tg.TraceSpec(tg.TINY, 2, 1)   # 8 streams, 4 warps per CTA
+    ev = make_events([])
+    _synthesize_matches(spec, ev, np.zeros(spec.num_streams + 1, np.uint64))
+
+    class NoStreams:
+        num_regions, warps_per_cta, num_sms = 3, 4, 2
+        cta_sm = np.zeros(0, np.uint32)
+        overlap_pairs = np.array([(0, 1)], np.uint32)
+    _synthesize_matches(NoStreams, ev, np.zeros(1, np.uint64))
+
+
 def test_synthesize_interval_capacity_too_small(synth_mode):
     """Fewer interval slots than the trace needs: the call reports ARGUS_ERR_CAPACITY with the required count, the
     later stages read nothing beyond the array, and the same buffers work again with enough room."""
