@@ -44,6 +44,7 @@ extern "C" {
 #define ARGUS_MAX_DEPTH   64          /* max simultaneously open frames per stream */
 #define ARGUS_MAX_REGIONS 65536       /* upper bound of num_regions */
 #define ARGUS_HIST_BINS   64
+#define ARGUS_MAX_PAIRS   256         /* (producer, consumer) pairs of one overlap call */
 
 /* return / status codes */
 enum {
@@ -266,6 +267,7 @@ int argus_aggregate(const argus_interval_t* intervals /*device*/,
  * spans [t_begin, t_begin + inclusive) of all intervals of region P (resp. Cn) in streams
  * whose CTA maps to m (all depths and contexts, flagged ones included, empty spans
  * dropped); U_P, U_C = their unions. out[k][m] = { |U_P ∩ U_C|, |U_P|, |U_C|, |U_P ∪ U_C| }.
+ * At most ARGUS_MAX_PAIRS pairs per call (more: ARGUS_ERR_INVALID_ARG).
  * max_intervals is an upper bound of interval_offsets[S] known on the host (for instance
  * the capacity given to argus_pair_intervals); it sizes the workspace, and a stream whose
  * offsets reach beyond it is not read (status->code = ARGUS_ERR_BAD_OFFSETS). If more spans

@@ -15,7 +15,7 @@
 namespace {
 
 constexpr int kOvThreads = 1024;
-constexpr u32 kMaxPairs = 256;
+constexpr u32 kMaxPairs = ARGUS_MAX_PAIRS;
 
 struct OvArgs {
   const argus_interval_t* intervals;
