@@ -220,7 +220,30 @@ __device__ __forceinline__ void cmp_swap(ulonglong2* d, u64 i, u64 l) {
   if (span_less(y, x)) { d[i] = y; d[l] = x; }
 }
 
+constexpr u32 kOvSortTile = 4096;  // spans of a segment sorted in shared memory at a time (64 KB)
+
+// Stages of the network whose partners lie inside one tile, on the tile in shared memory: the flip of block size k
+// (if `flip`) and then the distances j_top, j_top / 2, ..., 1. `tbase` is the tile's first index in the segment.
+__device__ __forceinline__ void ov_sort_tile_stages(ulonglong2* t, u64 tbase, u64 n, u32 k, bool flip, u32 j_top) {
+  if (flip) {
+    for (u32 i = threadIdx.x; i < kOvSortTile; i += blockDim.x) {
+      const u32 l = i ^ (k - 1);
+      if (l > i && tbase + l < n) cmp_swap(t, i, l);
+    }
+    __syncthreads();
+  }
+  for (u32 j = j_top; j > 0; j >>= 1) {
+    for (u32 i = threadIdx.x; i < kOvSortTile; i += blockDim.x) {
+      const u32 l = i ^ j;
+      if (l > i && tbase + l < n) cmp_swap(t, i, l);
+    }
+    __syncthreads();
+  }
+}
+
 __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
+  extern __shared__ __align__(16) unsigned char sort_raw[];
+  ulonglong2* const tile = reinterpret_cast<ulonglong2*>(sort_raw);
   __shared__ u64 sh[33];
   __shared__ u64 sh_carry_e, sh_carry_len;
   if (a.status->code != 0) return;
@@ -231,18 +254,41 @@ __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
   ulonglong2* d = a.spans + base;
   u64 p = 1;
   while (p < n) p <<= 1;
-  // bitonic network whose comparators all sort ascending; slots >= n act as +infinity and never move
-  for (u64 k = 2; k <= p; k <<= 1) {
-    for (u64 i = threadIdx.x; i < p; i += blockDim.x) {
+  // Bitonic network whose comparators all sort ascending; slots >= n act as +infinity and never move. A stage is a
+  // barrier apart from the next, and a segment larger than the L1 pays an L2 round trip per stage in global memory:
+  // so every run of stages whose partners lie within kOvSortTile spans is done on tiles in shared memory (one load
+  // and one store of the segment per run), and only the stages that reach across tiles work on global memory.
+  const u64 ntiles = (n + kOvSortTile - 1) / kOvSortTile;
+  for (u64 tI = 0; tI < ntiles; ++tI) {  // all block sizes up to a tile
+    const u64 tbase = tI * kOvSortTile;
+    const u32 cnt = (u32)(n - tbase < kOvSortTile ? n - tbase : kOvSortTile);
+    for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) tile[i] = d[tbase + i];
+    __syncthreads();
+    for (u32 k = 2; k <= kOvSortTile && k <= p; k <<= 1) ov_sort_tile_stages(tile, tbase, n, k, true, k >> 2);
+    for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) d[tbase + i] = tile[i];
+    __syncthreads();
+  }
+  for (u64 k = 2ull * kOvSortTile; k <= p; k <<= 1) {
+    for (u64 i = threadIdx.x; i < p; i += blockDim.x) {  // the flip and the long distances: across tiles
       const u64 l = i ^ (k - 1);
       if (l > i && l < n) cmp_swap(d, i, l);
     }
     __syncthreads();
-    for (u64 j = k >> 2; j > 0; j >>= 1) {
+    u64 j = k >> 2;
+    for (; j >= kOvSortTile; j >>= 1) {
       for (u64 i = threadIdx.x; i < p; i += blockDim.x) {
         const u64 l = i ^ j;
         if (l > i && l < n) cmp_swap(d, i, l);
       }
+      __syncthreads();
+    }
+    for (u64 tI = 0; tI < ntiles; ++tI) {  // the distances below a tile
+      const u64 tbase = tI * kOvSortTile;
+      const u32 cnt = (u32)(n - tbase < kOvSortTile ? n - tbase : kOvSortTile);
+      for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) tile[i] = d[tbase + i];
+      __syncthreads();
+      ov_sort_tile_stages(tile, tbase, n, 0, false, (u32)j);
+      for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) d[tbase + i] = tile[i];
       __syncthreads();
     }
   }
@@ -386,7 +432,17 @@ static int ov_run(OvArgs& a, const OvList* list, cudaStream_t stream) {
     }
   }
   argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 0);
-  k_ov_sort<<<a.nseg, kOvThreads, 0, stream>>>(a);
+  {
+    static bool opted_in[64];  // the shared-memory opt-in belongs to a device
+    int dev = 0;
+    ARGUS_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ARGUS_ERR_INVALID_ARG;
+    if (!opted_in[dev]) {
+      ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_ov_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kOvSortTile * sizeof(ulonglong2))));
+      opted_in[dev] = true;
+    }
+  }
+  k_ov_sort<<<a.nseg, kOvThreads, kOvSortTile * sizeof(ulonglong2), stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 1);
   k_ov_measure<<<a.nseg / 2, 256, 0, stream>>>(a);
