@@ -224,18 +224,21 @@ constexpr u32 kOvSortTile = 4096;  // spans of a segment sorted in shared memory
 
 // Stages of the network whose partners lie inside one tile, on the tile in shared memory: the flip of block size k
 // (if `flip`) and then the distances j_top, j_top / 2, ..., 1. `tbase` is the tile's first index in the segment.
+// (every thread takes whole comparators: comparator c of a stage with distance bit h joins i = c with a zero
+// inserted at bit h, and its partner)
 __device__ __forceinline__ void ov_sort_tile_stages(ulonglong2* t, u64 tbase, u64 n, u32 k, bool flip, u32 j_top) {
   if (flip) {
-    for (u32 i = threadIdx.x; i < kOvSortTile; i += blockDim.x) {
-      const u32 l = i ^ (k - 1);
-      if (l > i && tbase + l < n) cmp_swap(t, i, l);
+    const u32 h = k >> 1;
+    for (u32 c = threadIdx.x; c < kOvSortTile / 2; c += blockDim.x) {
+      const u32 i = ((c & ~(h - 1)) << 1) | (c & (h - 1)), l = i ^ (k - 1);
+      if (tbase + l < n) cmp_swap(t, i, l);
     }
     __syncthreads();
   }
   for (u32 j = j_top; j > 0; j >>= 1) {
-    for (u32 i = threadIdx.x; i < kOvSortTile; i += blockDim.x) {
-      const u32 l = i ^ j;
-      if (l > i && tbase + l < n) cmp_swap(t, i, l);
+    for (u32 c = threadIdx.x; c < kOvSortTile / 2; c += blockDim.x) {
+      const u32 i = ((c & ~(j - 1)) << 1) | (c & (j - 1)), l = i | j;
+      if (tbase + l < n) cmp_swap(t, i, l);
     }
     __syncthreads();
   }
@@ -269,16 +272,17 @@ __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
     __syncthreads();
   }
   for (u64 k = 2ull * kOvSortTile; k <= p; k <<= 1) {
-    for (u64 i = threadIdx.x; i < p; i += blockDim.x) {  // the flip and the long distances: across tiles
-      const u64 l = i ^ (k - 1);
-      if (l > i && l < n) cmp_swap(d, i, l);
+    const u64 h = k >> 1;
+    for (u64 c = threadIdx.x; c < p / 2; c += blockDim.x) {  // the flip and the long distances: across tiles
+      const u64 i = ((c & ~(h - 1)) << 1) | (c & (h - 1)), l = i ^ (k - 1);
+      if (l < n) cmp_swap(d, i, l);
     }
     __syncthreads();
     u64 j = k >> 2;
     for (; j >= kOvSortTile; j >>= 1) {
-      for (u64 i = threadIdx.x; i < p; i += blockDim.x) {
-        const u64 l = i ^ j;
-        if (l > i && l < n) cmp_swap(d, i, l);
+      for (u64 c = threadIdx.x; c < p / 2; c += blockDim.x) {
+        const u64 i = ((c & ~(j - 1)) << 1) | (c & (j - 1)), l = i | j;
+        if (l < n) cmp_swap(d, i, l);
       }
       __syncthreads();
     }
