@@ -30,6 +30,8 @@ struct OvArgs {
   u64* seg_cursor;  // [nseg]     (zeroed)
   u64* seg_base;    // [nseg + 1]
   ulonglong2* spans;  // [capacity] (start, end) -> after k_ov_sort (piece begin, piece end)
+  ulonglong2* scratch;  // room k_ov_sort may use (the span list, which is dead by then); null = none
+  u64 scratch_capacity;
   u64* cum;           // [capacity] covered length before piece i within its segment
   u64 capacity;
   u32 nseg;
@@ -244,6 +246,108 @@ __device__ __forceinline__ void ov_sort_tile_stages(ulonglong2* t, u64 tbase, u6
   }
 }
 
+// Sort of a large segment in expected linear time: spans are spread over buckets of equal width in start time (about 32
+// a bucket for starts spread evenly), copied to `scratch` bucket by bucket, and every bucket is sorted by one warp with a
+// small bitonic network in shared memory and written back in place. Returns false, with `d` untouched, when some bucket
+// would hold more than kOvBucketMax spans (starts crowded in time): the caller then runs the full network.
+// Shared memory (kOvSortSmem bytes at `raw`): bucket offsets, bucket cursors, one slice of kOvBucketMax spans per warp.
+constexpr u32 kOvBucketMax = 128;
+constexpr u32 kOvBuckets = 4096;
+constexpr size_t kOvSortSmem = 2 * (kOvBuckets + 1) * 4 + 32 + (size_t)(kOvThreads / 32) * kOvBucketMax * sizeof(ulonglong2);
+
+__device__ bool ov_bucket_sort(ulonglong2* d, ulonglong2* scratch, u64 n, unsigned char* raw) {
+  u32* const off = reinterpret_cast<u32*>(raw);                 // [kOvBuckets + 1]
+  u32* const cur = off + kOvBuckets + 1;                        // [kOvBuckets + 1]
+  ulonglong2* const slices = reinterpret_cast<ulonglong2*>(raw + ((2 * (kOvBuckets + 1) * 4 + 15) & ~(size_t)15));
+  __shared__ u64 red[2][32];
+  __shared__ u32 sh_scan[33];
+  __shared__ u32 crowded;
+  const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (n >> 31) return false;
+  // range of the start times
+  u64 mn = ~0ull, mx = 0;
+  for (u64 i = threadIdx.x; i < n; i += blockDim.x) {
+    const u64 s = d[i].x;
+    mn = s < mn ? s : mn;
+    mx = s > mx ? s : mx;
+  }
+#pragma unroll
+  for (int dd = 16; dd > 0; dd >>= 1) {
+    const u64 a = __shfl_xor_sync(0xffffffffu, mn, dd), b = __shfl_xor_sync(0xffffffffu, mx, dd);
+    mn = a < mn ? a : mn;
+    mx = b > mx ? b : mx;
+  }
+  if (lane == 0) { red[0][warp] = mn; red[1][warp] = mx; }
+  if (threadIdx.x == 0) crowded = 0;
+  __syncthreads();
+  mn = red[0][0]; mx = red[1][0];
+  for (u32 w = 1; w < blockDim.x / 32; ++w) {
+    mn = red[0][w] < mn ? red[0][w] : mn;
+    mx = red[1][w] > mx ? red[1][w] : mx;
+  }
+  // buckets: a power of two of them, about 32 spans each; equal width, a power of two of ticks
+  u32 nb = 1;
+  while (nb < kOvBuckets && (u64)nb * 32 < n) nb <<= 1;
+  u32 shift = 0;
+  while (((mx - mn) >> shift) >= nb) ++shift;
+  for (u32 b = threadIdx.x; b <= nb; b += blockDim.x) { off[b] = 0; cur[b] = 0; }
+  __syncthreads();
+  for (u64 i = threadIdx.x; i < n; i += blockDim.x) atomicAdd(&off[(u32)((d[i].x - mn) >> shift)], 1u);
+  __syncthreads();
+  for (u32 b = threadIdx.x; b < nb; b += blockDim.x)
+    if (off[b] > kOvBucketMax) crowded = 1;
+  __syncthreads();
+  if (crowded) return false;  // uniform: every thread read the same word after the barrier
+  // exclusive prefix of the counts (nb <= 4 x 1024)
+  u32 carry = 0;
+  for (u32 b0 = 0; b0 < nb; b0 += blockDim.x) {
+    const u32 b = b0 + threadIdx.x;
+    const u32 c = b < nb ? off[b] : 0u;
+    u32 total;
+    const u32 ex = argus_block_exclusive_scan<u32>(c, sh_scan, &total);
+    if (b < nb) off[b] = carry + ex;
+    carry += total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) off[nb] = (u32)n;
+  __syncthreads();
+  for (u64 i = threadIdx.x; i < n; i += blockDim.x) {
+    const ulonglong2 sp = d[i];
+    const u32 b = (u32)((sp.x - mn) >> shift);
+    scratch[off[b] + atomicAdd(&cur[b], 1u)] = sp;
+  }
+  __syncthreads();
+  // one warp per bucket: small network in the warp's slice, then back in place (buckets are in time order)
+  ulonglong2* const sl = slices + (size_t)warp * kOvBucketMax;
+  for (u32 b = warp; b < nb; b += blockDim.x / 32) {
+    const u32 lo = off[b], c = off[b + 1] - lo;
+    if (c == 0) continue;
+    u32 m = 1;
+    while (m < c) m <<= 1;
+    for (u32 t = lane; t < m; t += 32) sl[t] = t < c ? scratch[lo + t] : make_ulonglong2(~0ull, ~0ull);
+    __syncwarp();
+    for (u32 k = 2; k <= m; k <<= 1) {
+      const u32 h = k >> 1;
+      for (u32 q = lane; q < m / 2; q += 32) {
+        const u32 i = ((q & ~(h - 1)) << 1) | (q & (h - 1));
+        cmp_swap(sl, i, i ^ (k - 1));
+      }
+      __syncwarp();
+      for (u32 j = k >> 2; j > 0; j >>= 1) {
+        for (u32 q = lane; q < m / 2; q += 32) {
+          const u32 i = ((q & ~(j - 1)) << 1) | (q & (j - 1));
+          cmp_swap(sl, i, i | j);
+        }
+        __syncwarp();
+      }
+    }
+    for (u32 t = lane; t < c; t += 32) d[lo + t] = sl[t];
+    __syncwarp();
+  }
+  __syncthreads();
+  return true;
+}
+
 __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
   extern __shared__ __align__(16) unsigned char sort_raw[];
   ulonglong2* const tile = reinterpret_cast<ulonglong2*>(sort_raw);
@@ -255,6 +359,9 @@ __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
   const u64 n = a.seg_base[seg + 1] - base;
   if (n == 0) return;
   ulonglong2* d = a.spans + base;
+  if (a.scratch && base + n <= a.scratch_capacity && n > kOvBucketMax && ov_bucket_sort(d, a.scratch + base, n, sort_raw)) {
+    // sorted by buckets of start time
+  } else {
   u64 p = 1;
   while (p < n) p <<= 1;
   // Bitonic network whose comparators all sort ascending; slots >= n act as +infinity and never move. A stage is a
@@ -295,6 +402,7 @@ __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
       for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) d[tbase + i] = tile[i];
       __syncthreads();
     }
+  }
   }
   // pieces of the union and running covered length
   if (threadIdx.x == 0) { sh_carry_e = 0; sh_carry_len = 0; }
@@ -442,11 +550,13 @@ static int ov_run(OvArgs& a, const OvList* list, cudaStream_t stream) {
     ARGUS_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return ARGUS_ERR_INVALID_ARG;
     if (!opted_in[dev]) {
-      ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_ov_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kOvSortTile * sizeof(ulonglong2))));
+      ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_ov_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kOvSortSmem));
       opted_in[dev] = true;
     }
   }
-  k_ov_sort<<<a.nseg, kOvThreads, kOvSortTile * sizeof(ulonglong2), stream>>>(a);
+  a.scratch = const_cast<ulonglong2*>(list->spans);  // every listed span has been copied into its segment
+  a.scratch_capacity = list->capacity;
+  k_ov_sort<<<a.nseg, kOvThreads, kOvSortSmem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 1);
   k_ov_measure<<<a.nseg / 2, 256, 0, stream>>>(a);
@@ -468,6 +578,7 @@ static int ov_setup(OvArgs& a, uint32_t num_streams, uint32_t warps_per_cta, con
   a.seg_count = (u64*)(ws + L.seg_count); a.seg_cursor = (u64*)(ws + L.seg_cursor); a.seg_base = (u64*)(ws + L.seg_base);
   a.capacity = (workspace_bytes - L.total_fixed) / 24;
   a.spans = (ulonglong2*)(ws + L.spans);
+  a.scratch = nullptr; a.scratch_capacity = 0;
   a.cum = (u64*)(ws + L.spans + argus_align_up((size_t)a.capacity * 16, 16));
   a.nseg = nseg;
   a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;

@@ -272,6 +272,47 @@ def test_overlap_random_spans_and_capacity():
     assert int(argus.argus_status_fetch(st)["code"]) == 4
 
 
+@pytest.mark.parametrize("shape", ["even", "same-start", "crowded-with-outliers", "huge-range", "one-bucket-over"])
+def test_overlap_segment_sort_paths(shape):
+    """Large segments are sorted by buckets of start time, or by the full network when the starts crowd:
+    starts spread evenly; thousands of equal starts; nearly all starts in a narrow window with a few far outliers;
+    starts over the whole 64-bit range; one bucket just over its capacity."""
+    rng = np.random.default_rng(len(shape))
+    S, W, M, R = 4, 2, 2, 2
+    n = 20000
+    cta_sm_np = np.array([0, 1], np.uint32)
+    iv = np.zeros(S * n, argus.INTERVAL_DTYPE)
+    for s in range(S):
+        if shape == "even":
+            t = (1 << 50) + np.sort(rng.integers(0, 1 << 34, n)).astype(np.uint64)
+        elif shape == "same-start":
+            t = np.full(n, 777, np.uint64)
+            t[: n // 2] += rng.integers(0, 3, n // 2).astype(np.uint64)
+        elif shape == "crowded-with-outliers":
+            t = (1 << 40) + rng.integers(0, 5000, n).astype(np.uint64)
+            t[:5] = (1 << 62) + rng.integers(0, 100, 5).astype(np.uint64)
+        elif shape == "huge-range":
+            t = rng.integers(0, 1 << 63, n).astype(np.uint64) * np.uint64(2) + rng.integers(0, 2, n).astype(np.uint64)
+            t = np.minimum(t, np.uint64((1 << 64) - (1 << 33)))
+        else:
+            t = np.arange(n, dtype=np.uint64) * np.uint64(1000)
+            t[100:230] = t[100]          # 130 equal starts: more than a bucket holds
+        sl = slice(s * n, (s + 1) * n)
+        iv["stream"][sl] = s
+        iv["region"][sl] = rng.integers(0, R, n)
+        iv["t_begin"][sl] = t
+        iv["inclusive"][sl] = rng.integers(0, 1 << 20, n)
+    ioffs = (np.arange(S + 1) * n).astype(np.uint64)
+    pairs_np = np.array([(0, 1), (1, 1)], np.uint32)
+    _, o_ov, _ = oracle.overlap(iv, ioffs, W, cta_sm_np, M, pairs_np)
+    d_iv = torch.from_numpy(iv.view(np.uint8).reshape(-1).copy()).to(DEV)
+    d_off = torch.from_numpy(ioffs.view(np.int64).copy()).to(DEV)
+    ov, st = argus.argus_overlap(d_iv, len(iv), d_off, W, torch.from_numpy(cta_sm_np.view(np.int32)).to(DEV), M,
+                                 torch.from_numpy(pairs_np.view(np.int32)).to(DEV))
+    assert int(argus.argus_status_fetch(st)["code"]) == 0
+    assert ov.cpu().numpy().view(argus.OVERLAP_DTYPE).reshape(o_ov.shape).tobytes() == o_ov.tobytes()
+
+
 def _synthesize_matches(spec, ev, offs, **kw):
     d_ev, d_off = to_dev(ev, offs)
     cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
