@@ -459,22 +459,32 @@ __global__ void __launch_bounds__(kOvThreads) k_ov_sort(OvArgs a) {
   }
 }
 
-// covered length of the pieces [pc, cum) of one segment strictly before time t
-__device__ __forceinline__ u64 covered_before(const ulonglong2* pc, const u64* cum, u64 n, u64 t) {
-  // number of pieces whose begin is < t
-  u64 lo = 0, hi = n;
+constexpr int kOvMeasureThreads = 1024;
+
+// covered length of the consumer pieces before time t, given pos = number of pieces whose begin is < t
+__device__ __forceinline__ u64 covered_at(const ulonglong2* pc, const u64* cum, u64 pos, u64 t) {
+  if (pos == 0) return 0;
+  const ulonglong2 last = pc[pos - 1];
+  return cum[pos - 1] + ((t < last.y ? t : last.y) - last.x);
+}
+
+// pos = number of consumer pieces whose begin is < t, reached from an earlier boundary's pos (never past it): steps
+// of doubling length, then a binary search inside the last step, so a far boundary costs a logarithm of its distance
+__device__ __forceinline__ u64 advance_to(const ulonglong2* pc, u64 nc, u64 pos, u64 t) {
+  if (pos >= nc || !(pc[pos].x < t)) return pos;
+  u64 lo = pos, step = 1;  // pc[lo].x < t
+  while (lo + step < nc && pc[lo + step].x < t) { lo += step; step <<= 1; }
+  u64 hi = lo + step < nc ? lo + step : nc;  // the first piece with begin >= t lies in (lo, hi]
+  ++lo;
   while (lo < hi) {
     const u64 mid = lo + ((hi - lo) >> 1);
     if (pc[mid].x < t) lo = mid + 1; else hi = mid;
   }
-  if (lo == 0) return 0;
-  const ulonglong2 last = pc[lo - 1];
-  const u64 upto = t < last.y ? t : last.y;
-  return cum[lo - 1] + (upto - last.x);
+  return lo;
 }
 
-__global__ void __launch_bounds__(256) k_ov_measure(OvArgs a) {
-  __shared__ u64 sh[8];
+__global__ void __launch_bounds__(kOvMeasureThreads) k_ov_measure(OvArgs a) {
+  __shared__ u64 sh[kOvMeasureThreads / 32];
   if (a.status->code != 0) return;
   const u32 km = blockIdx.x;  // k * M + m
   const u64 bp = a.seg_base[2 * km], bc = a.seg_base[2 * km + 1], be = a.seg_base[2 * km + 2];
@@ -484,9 +494,29 @@ __global__ void __launch_bounds__(256) k_ov_measure(OvArgs a) {
   const u64* cum_c = a.cum + bc;
   u64 acc = 0;
   if (nc) {
-    for (u64 i = threadIdx.x; i < np; i += blockDim.x) {
-      const ulonglong2 piece = pp[i];
-      if (piece.y > piece.x) acc += covered_before(pc, cum_c, nc, piece.y) - covered_before(pc, cum_c, nc, piece.x);
+    // Every thread takes a run of consecutive producer pieces. Pieces are disjoint and in time order, so the
+    // boundaries a thread asks about never decrease: one binary search places the first, the rest are reached from
+    // the one before (usually the next consumer piece or two).
+    const u64 per = (np + blockDim.x - 1) / blockDim.x;
+    const u64 i0 = (u64)threadIdx.x * per, i1 = i0 + per < np ? i0 + per : np;
+    if (i0 < i1) {
+      u64 pos;  // number of consumer pieces whose begin is < the boundary at hand
+      {
+        const u64 t = pp[i0].x;
+        u64 lo = 0, hi = nc;
+        while (lo < hi) {
+          const u64 mid = lo + ((hi - lo) >> 1);
+          if (pc[mid].x < t) lo = mid + 1; else hi = mid;
+        }
+        pos = lo;
+      }
+      for (u64 i = i0; i < i1; ++i) {
+        const ulonglong2 piece = pp[i];
+        pos = advance_to(pc, nc, pos, piece.x);
+        const u64 before = covered_at(pc, cum_c, pos, piece.x);
+        pos = advance_to(pc, nc, pos, piece.y);
+        if (piece.y > piece.x) acc += covered_at(pc, cum_c, pos, piece.y) - before;
+      }
     }
   }
 #pragma unroll
@@ -559,7 +589,7 @@ static int ov_run(OvArgs& a, const OvList* list, cudaStream_t stream) {
   k_ov_sort<<<a.nseg, kOvThreads, kOvSortSmem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   argus_prof_mark(ARGUS_PROF_OVERLAP, stream, 1);
-  k_ov_measure<<<a.nseg / 2, 256, 0, stream>>>(a);
+  k_ov_measure<<<a.nseg / 2, kOvMeasureThreads, 0, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   return ARGUS_OK;
 }
