@@ -514,12 +514,16 @@ def _fuzz_case(seed):
     return Spec, ev.astype(argus.EVENT_DTYPE), np.array(offs, np.uint64)
 
 
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", list(range(16)) + [305])   # 305: a stream that opens a 65th frame
 def test_synthesize_random_shapes(seed, synth_mode):
     spec, ev, offs = _fuzz_case(seed)
     rc, _, _, _, _, o_st = oracle.pair(ev, offs, spec.num_regions)
-    if int(o_st["code"]) != 0:
-        pytest.skip("the random corruption opened more than 64 frames")
+    if int(o_st["code"]) != 0:   # the random corruption opened more than 64 frames: the same error is reported
+        d_ev, d_off = to_dev(ev, offs)
+        cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+        st = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, None).fetch_status()
+        assert int(st["code"]) == int(o_st["code"])
+        return
     _synthesize_matches(spec, ev, offs)
 
 

@@ -15,14 +15,19 @@ from test_ring_buffer import make_ring
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("seed", range(100, 112))
+@pytest.mark.parametrize("seed", list(range(100, 112)) + [328])   # 328: a stream that opens a 65th frame
 def test_random_shape_through_pairing_scopes_and_ring(seed):
     spec, ev, offs = _fuzz_case(seed)
     rng = np.random.default_rng(seed)
     R, W, M = spec.num_regions, spec.warps_per_cta, spec.num_sms
     rc, iv, ioffs, am, aoffs, o_st = oracle.pair(ev, offs, R)
-    if int(o_st["code"]) != 0:
-        pytest.skip("the random corruption opened more than 64 frames")
+    if int(o_st["code"]) != 0:   # the random corruption opened more than 64 frames: both kernels report it alike
+        from test_gpu_parity import run_pair
+        for kernel in (KERNEL_THREAD_PER_STREAM, KERNEL_TILED):
+            _, st = run_pair(ev, offs, R, kernel)
+            assert (int(st["code"]), int(st["bad_stream"]), int(st["bad_event"])) == \
+                   (int(o_st["code"]), int(o_st["bad_stream"]), int(o_st["bad_event"]))
+        return
     for kernel in (KERNEL_THREAD_PER_STREAM, KERNEL_TILED):
         assert_pair_matches(ev, offs, R, kernel)
     scope = {}
