@@ -47,6 +47,11 @@ int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* am
                               argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream);
 bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs);
 
+// argus_ring.cu — stream_offsets (and dropped) of the records that survive in the slots of a ring container;
+// status->code = ARGUS_ERR_CAPACITY if they exceed event_capacity. The status block is not cleared.
+int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
+                                uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream);
+
 // argus_overlap.cu
 int argus_internal_overlap(const argus_interval_t* intervals, uint64_t max_intervals, const uint64_t* interval_offsets,
                            uint32_t num_streams, uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms,

@@ -327,10 +327,6 @@ extern "C" int argus_pair_intervals(const argus_event_t* events, uint64_t num_ev
                                  workspace, workspace_bytes, cuda_stream, 0);
 }
 
-// implemented in argus_ring.cu
-int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
-                                uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream);
-
 extern "C" int argus_pair_intervals_ring(const argus_event_t* ring, uint32_t slot_capacity, const uint64_t* written,
                                          uint32_t num_streams, uint32_t num_regions, uint64_t* stream_offsets,
                                          uint64_t* dropped, argus_interval_t* intervals, uint64_t interval_capacity,

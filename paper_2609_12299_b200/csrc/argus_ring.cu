@@ -3,7 +3,7 @@
 //
 //   k_ring_offsets : single-block scan of min(written, slot_capacity) over the streams; capacity check
 //   k_ring_copy    : one block per stream copies the surviving records, oldest first (16-byte loads and stores)
-#include "argus_common.cuh"
+#include "argus_internal.cuh"
 
 namespace {
 
@@ -53,8 +53,6 @@ __global__ void __launch_bounds__(256) k_ring_copy(const uint4* ring, u32 slot_c
 
 }  // namespace
 
-// stream_offsets (and dropped) of the records that survive in the slots; status->code = ARGUS_ERR_CAPACITY if they
-// exceed event_capacity. The status block is not cleared here.
 int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
                                 uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream) {
   k_ring_offsets<<<1, kRingScanThreads, 0, (cudaStream_t)cuda_stream>>>((const u64*)written, slot_capacity, num_streams, event_capacity,

@@ -3,10 +3,11 @@
 // Pairing runs plain and writes, beside every 48-byte interval record, an 8-byte digest (region, both
 // durations, a flag bit); then ONE pass over the digests both aggregates the intervals and selects the overlap
 // spans. Hosting the table in the pairing kernel (which is bound by instruction issue and occupancy, not by
-// HBM) measured slower on every trace shape, and so did a pass over the records themselves (six times the bytes). The pairing kernel's own hooks
-// (aggregate and select while the interval is in registers: the interval array is never read back) remain
-// for calls that ask for overlap without tables and as a tuning choice (argus_set_synthesize_mode). More than 400
-// regions or 128 pairs: the three plain calls. Results are identical in every mode.
+// HBM) measured slower on every trace shape, and so did a pass over the records themselves (six times the
+// bytes). The pairing kernel's own hooks (aggregate and select while the interval is in registers: the interval
+// array is never read back) remain for calls that ask for overlap without tables and as a tuning choice
+// (argus_set_synthesize_mode). More than 400 regions or 128 pairs: the three plain calls. Results are identical
+// in every mode. argus_synthesize_ring is the same pipeline on a ring container.
 #include "argus_internal.cuh"
 
 namespace {
@@ -60,10 +61,6 @@ extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t
                                                    uint64_t max_overlap_spans) {
   return syn_layout(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms, max_overlap_spans).total;
 }
-
-// implemented in argus_ring.cu
-int argus_internal_ring_offsets(const uint64_t* written, uint32_t slot_capacity, uint32_t num_streams, uint64_t event_capacity,
-                                uint64_t* stream_offsets, uint64_t* dropped, argus_status_t* status, void* cuda_stream);
 
 // ring_written non-null: `events` is a ring container whose packed offsets are already in stream_offsets (device);
 // num_events then bounds the surviving records and the status block has been cleared by the caller.
