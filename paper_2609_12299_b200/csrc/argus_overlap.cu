@@ -5,11 +5,13 @@
 //                  (argus_synthesize gets the same list from the aggregation pass or the pairing kernel instead)
 //   k_ov_list_count_or_scatter : spans counted per segment, then copied into their segment (order irrelevant)
 //   k_ov_scan    : segment bases; capacity check
-//   k_ov_sort    : one CTA per segment: sort by (start, end); then turn the sorted spans into the
+//   k_ov_sort    : one CTA per segment: sort by (start, end) — by buckets of start time with one warp per bucket,
+//                  or by a bitonic network on shared-memory tiles when the starts crowd; then turn the sorted spans into the
 //                  disjoint pieces of their union, piece i = [max(start_i, E_{i-1}), E_i) with
 //                  E_i = max end of spans 0..i, and the running length before each piece
 //   k_ov_measure : one CTA per (k, m): |U_P|, |U_C|, and |U_P ∩ U_C| = sum over producer pieces of
-//                  F_C(b) - F_C(a), F_C(t) = covered length of U_C before t (binary search in C pieces)
+//                  F_C(b) - F_C(a), F_C(t) = covered length of U_C before t (threads walk runs of producer pieces
+//                  and find each boundary among the C pieces from the one before)
 #include "argus_internal.cuh"
 
 namespace {
