@@ -52,6 +52,45 @@ __global__ void __launch_bounds__(128) k_pair_thread_per_stream(ArgusPairArgs a)
 }
 
 // ---------------------------------------------------------------------------------------------
+// order: streams sorted by length class (floor(log2(events))), longest first. A stream is a chain of chunks that
+// one CTA at a time walks, so when lengths differ (producer and consumer warps of one kernel) the long chains must
+// start first or they end last, alone. Counting sort in one block; the order inside a class does not matter.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kScanThreads) k_pair_order(ArgusPairArgs a, u32* order) {
+  __shared__ u32 cnt[64], cur[64];
+  __shared__ u32 one_class;
+  if (threadIdx.x < 64) { cnt[threadIdx.x] = 0; cur[threadIdx.x] = 0; }
+  __syncthreads();
+  for (u32 s = threadIdx.x; s < a.num_streams; s += blockDim.x) {
+    const u64 lo = a.stream_offsets[s], hi = a.stream_offsets[s + 1];
+    const u64 n = hi > lo ? hi - lo : 0;
+    atomicAdd(&cnt[n ? 63 - __clzll((long long)n) : 0], 1u);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {  // bases, classes in descending order
+    u32 base = 0;
+    one_class = 0;
+    for (int c = 63; c >= 0; --c) {
+      const u32 k = cnt[c];
+      if (k == a.num_streams) one_class = 1;
+      cnt[c] = base;
+      base += k;
+    }
+  }
+  __syncthreads();
+  if (one_class) {  // streams of one length class start in index order, as without this kernel
+    for (u32 s = threadIdx.x; s < a.num_streams; s += blockDim.x) order[s] = s;
+    return;
+  }
+  for (u32 s = threadIdx.x; s < a.num_streams; s += blockDim.x) {
+    const u64 lo = a.stream_offsets[s], hi = a.stream_offsets[s + 1];
+    const u64 n = hi > lo ? hi - lo : 0;
+    const u32 c = n ? 63 - __clzll((long long)n) : 0;
+    order[cnt[c] + atomicAdd(&cur[c], 1u)] = s;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // offsets: exclusive scan of per-stream counts; decides whether the second pass is needed.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kScanThreads) k_pair_offsets(ArgusPairArgs a) {
@@ -185,7 +224,7 @@ __global__ void __launch_bounds__(256) k_ambig_offsets(AmbigArgs g) {
 }
 
 struct Layout {
-  size_t ctl, counts, queue, bits, word_prefix, block_prefix, notes, records, total;
+  size_t ctl, counts, queue, bits, word_prefix, block_prefix, notes, records, order, total;
   u64 num_words, num_blocks, queue_capacity;
   u32 record_capacity;
 };
@@ -206,6 +245,7 @@ Layout make_layout(uint64_t num_events, uint32_t num_streams, uint64_t ambig_cap
   L.block_prefix = o; o += argus_align_up(((size_t)L.num_blocks + 1) * 8, 256);
   L.notes = o; o += argus_align_up((size_t)ambig_capacity * 8 + 8, 256);
   L.records = o; o += argus_align_up((size_t)L.record_capacity * sizeof(ArgusStreamRecord), 256);
+  L.order = o; o += argus_align_up((size_t)num_streams * 4 + 4, 256);
   L.total = o;
   return L;
 }
@@ -266,6 +306,12 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   ARGUS_CUDA_TRY(cudaMemsetAsync(ws, 0, L.word_prefix, stream));
 
   const bool tiled = (kernel_choice != 1 && argus_pair_tiled_usable(a)) || ring_written != nullptr;
+  a.order = nullptr;
+  if (tiled && num_streams > 1) {
+    k_pair_order<<<1, kScanThreads, 0, stream>>>(a, (u32*)(ws + L.order));
+    ARGUS_CHECK_LAUNCH();
+    a.order = (const u32*)(ws + L.order);
+  }
   const bool fused = tiled && fuse && argus_pair_tiled_can_fuse(num_regions);
   if (fused) a.fuse = *fuse;
   if (fused_out) *fused_out = fused;

@@ -74,6 +74,7 @@ struct ArgusPairArgs {
   u64 queue_capacity;
   ArgusStreamRecord* records;
   u32 record_capacity;
+  const u32* order;       // streams in the order in which the tiled kernel starts them: longest first (null = by index)
   u64* digest;            // one digest per interval record, same positions (null = none); holds every position below
                           // min(interval_capacity, num_events / 2 + 1), which is all a stream can reach
   const u64* ring_written; // non-null: `events` is a ring container, one slot of ring_capacity records per stream, record i of

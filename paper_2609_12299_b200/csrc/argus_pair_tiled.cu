@@ -72,7 +72,7 @@ constexpr u32 kNoRec = 0xffffffffu;
 // hand-over from the queue. Returns false when every stream is done (or on a timeout). One thread per CTA.
 __device__ __forceinline__ bool tile_pop_work(const ArgusPairArgs& a, int p, u64* stream, u32* rec) {
   const u64 h = atomicAdd(reinterpret_cast<unsigned long long*>(&a.ctl->q_head[p]), 1ull);
-  if (h < a.num_streams) { *stream = h; *rec = kNoRec; return true; }
+  if (h < a.num_streams) { *stream = a.order ? a.order[h] : h; *rec = kNoRec; return true; }
   const u64 slot = h - a.num_streams;
   if (!a.queue || slot >= a.queue_capacity) return false;  // more positions than hand-overs can ever be published
   volatile u32* q = a.queue + slot;
