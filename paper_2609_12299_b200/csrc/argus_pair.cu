@@ -142,15 +142,19 @@ struct AmbigArgs {
   u64* ambig_offsets;
 };
 
+// (a fixed grid walks the blocks of words: a trace without ambiguous markers, the usual case, costs one small launch)
 __global__ void __launch_bounds__(kWordsPerBlock) k_ambig_word_prefix(AmbigArgs g) {
   __shared__ u32 sh[33];
   if (g.p.ctl->n_notes == 0) return;
-  const u64 w = (u64)blockIdx.x * kWordsPerBlock + threadIdx.x;
-  const u32 c = w < g.num_words ? __popc(g.p.bits[w]) : 0u;
-  u32 total;
-  const u32 ex = argus_block_exclusive_scan<u32>(c, sh, &total);
-  if (w < g.num_words) g.word_prefix[w] = ex;
-  if (threadIdx.x == 0) g.block_prefix[blockIdx.x] = total;
+  for (u64 blk = blockIdx.x; blk < g.num_blocks; blk += gridDim.x) {
+    const u64 w = blk * kWordsPerBlock + threadIdx.x;
+    const u32 c = w < g.num_words ? __popc(g.p.bits[w]) : 0u;
+    u32 total;
+    const u32 ex = argus_block_exclusive_scan<u32>(c, sh, &total);
+    if (w < g.num_words) g.word_prefix[w] = ex;
+    if (threadIdx.x == 0) g.block_prefix[blk] = total;
+    __syncthreads();
+  }
 }
 
 __global__ void __launch_bounds__(kScanThreads) k_ambig_block_scan(AmbigArgs g) {
@@ -339,7 +343,7 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   g.word_prefix = (u32*)(ws + L.word_prefix); g.block_prefix = (u64*)(ws + L.block_prefix);
   g.num_blocks = L.num_blocks; g.ambig = ambig; g.ambig_capacity = ambig_capacity; g.ambig_offsets = (u64*)ambig_offsets;
   if (L.num_blocks) {
-    k_ambig_word_prefix<<<(unsigned)L.num_blocks, kWordsPerBlock, 0, stream>>>(g);
+    k_ambig_word_prefix<<<(unsigned)(L.num_blocks < 2368 ? L.num_blocks : 2368), kWordsPerBlock, 0, stream>>>(g);
     ARGUS_CHECK_LAUNCH();
   }
   k_ambig_block_scan<<<1, kScanThreads, 0, stream>>>(g);
