@@ -117,6 +117,7 @@ def oracle_step(oracle, ev, offs, spec, cta_sm, num_sms):
 def oracle_sample(tg, spec, num_ctas):
     """Host copy of the first `num_ctas` CTAs of the workload (bit-identical to the device trace)."""
     offs = tg.host_offsets(spec)
+    num_ctas = min(num_ctas, spec.num_ctas)
     S = num_ctas * spec.warps_per_cta
     ev = tg.host_streams(spec, offs, 0, S)
     sub = (offs[: S + 1] - offs[0]).astype(np.uint64)
@@ -341,7 +342,7 @@ def main():
         dt = time.perf_counter() - t0
         cpu_baseline = {"value": len(ev) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "host_cores": os.cpu_count(),
                         "seconds": dt,
-                        "sample": f"first {args.cpu_ctas} CTAs = {args.cpu_ctas * spec.warps_per_cta} streams, {len(ev)} events, one pass"}
+                        "sample": f"first {len(csm)} CTAs = {len(offs) - 1} streams, {len(ev)} events, one pass"}
         # the same oracle as independent instances, one CTA of the trace each, on all host cores
         # (the C++ oracle runs outside the interpreter lock; each instance is still single-threaded)
         from concurrent.futures import ThreadPoolExecutor
