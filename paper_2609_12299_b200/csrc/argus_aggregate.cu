@@ -678,19 +678,6 @@ __global__ void __launch_bounds__(256) k_agg_iter_reduce(AggArgs a) {
   }
 }
 
-// ambiguity counters into the warp-scope table (used when the intervals were aggregated by the pairing kernel)
-__global__ void __launch_bounds__(256) k_agg_ambig(AggArgs a) {
-  for (u32 s = blockIdx.x; s < a.num_streams; s += gridDim.x) {
-    const u64 alo = a.ambig_offsets[s], ahi = a.ambig_offsets[s + 1];
-    u64* row = a.warp_tab + (size_t)s * a.num_regions * kCell;
-    for (u64 i = alo + threadIdx.x; i < ahi && ahi >= alo; i += blockDim.x) {
-      const u32 region = a.ambig[i].tag >> 1;
-      if (region >= a.num_regions) { argus_set_error(a.status, ARGUS_ERR_BAD_REGION, s, i); continue; }
-      atomicAdd(row + (size_t)region * kCell + (a.ambig[i].kind == ARGUS_AMBIG_UNMATCHED_END ? 6 : 5), 1ull);
-    }
-  }
-}
-
 struct AggLayout { size_t warp, cta, iter, total; };
 
 AggLayout agg_layout(uint32_t num_streams, uint32_t num_regions) {
@@ -704,46 +691,6 @@ AggLayout agg_layout(uint32_t num_streams, uint32_t num_regions) {
 }
 
 }  // namespace
-
-// Roll-up of a filled warp-scope table into the CTA, SM and kernel scopes.
-static int agg_rollup(AggArgs& a, argus_agg_t* cta_tab, argus_agg_t* sm_tab, argus_agg_t* kernel_tab, cudaStream_t stream) {
-  if (cta_tab || sm_tab || kernel_tab) {
-    k_agg_cta<<<1184, 256, 0, stream>>>(a);
-    ARGUS_CHECK_LAUNCH();
-  }
-  if (sm_tab || kernel_tab) {
-    if (sm_tab) { k_agg_init<<<296, 256, 0, stream>>>(a.sm_tab, (u64)a.num_sms * a.num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
-    if (kernel_tab) { k_agg_init<<<16, 256, 0, stream>>>(a.kernel_tab, (u64)a.num_regions * kCell); ARGUS_CHECK_LAUNCH(); }
-    k_agg_scatter<<<1184, 256, 0, stream>>>(a);
-    ARGUS_CHECK_LAUNCH();
-  }
-  return ARGUS_OK;
-}
-
-// Second half of aggregation when the pairing kernel already filled the interval statistics of
-// warp_tab: ambiguity counters, then the roll-up. warp_tab and cta_work must be non-null.
-int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                              argus_agg_t* warp_tab, argus_agg_t* cta_work, bool want_cta, argus_agg_t* sm_tab,
-                              argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream) {
-  cudaStream_t stream = (cudaStream_t)cuda_stream;
-  if (num_streams == 0) return ARGUS_OK;
-  AggArgs a;
-  a.intervals = nullptr; a.interval_offsets = nullptr; a.ambig = ambig; a.ambig_offsets = (const u64*)ambig_offsets;
-  a.num_streams = num_streams; a.warps_per_cta = warps_per_cta; a.num_ctas = num_streams / warps_per_cta;
-  a.num_sms = num_sms; a.num_regions = num_regions; a.cta_sm = cta_sm;
-  a.warp_tab = (u64*)warp_tab; a.cta_tab = (u64*)cta_work; a.sm_tab = (u64*)sm_tab; a.kernel_tab = (u64*)kernel_tab;
-  a.status = status; a.use_smem = 0;
-  a.scoped = 0; a.ctx_lo = 0; a.ctx_hi = 0xffffffffu; a.warp_mask = ~0ull; a.sm_mask = nullptr; a.region_mask = nullptr;
-  a.role_tab = nullptr; a.iter_tab = nullptr; a.num_iters = 0; a.iter_smem = 0; a.iter_copies = nullptr; a.num_copies = 0;
-  a.iter_inline = 0;
-  a.ov.ov_spans = nullptr; a.ov.num_pairs = 0; a.ov.ov_chunk = 256; a.digest = nullptr; a.interval_limit = ~0ull;
-  if (ambig && ambig_offsets) {
-    k_agg_ambig<<<num_streams < 1184 ? num_streams : 1184, 256, 0, stream>>>(a);
-    ARGUS_CHECK_LAUNCH();
-  }
-  return agg_rollup(a, want_cta || sm_tab || kernel_tab ? cta_work : nullptr, sm_tab, kernel_tab, stream);
-}
 
 extern "C" size_t argus_aggregate_workspace_bytes(uint64_t /*num_intervals*/, uint32_t num_streams, uint32_t num_regions) {
   return agg_layout(num_streams, num_regions).total + 256;

@@ -5,7 +5,6 @@
 #include "argus_fuse.cuh"
 
 // argus_pair.cu — the whole pairing pipeline. kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled.
-// `fuse` (nullable) asks the tiled kernel to feed aggregation / overlap selection; *fused_out tells whether it did.
 // `digest` (nullable): one 8-byte digest per interval record, at the record's position (see argus_fuse.cuh).
 // `ring_written` (nullable): `events` is a ring container (one slot of ring_capacity records per stream, written[s] records
 // ever written); stream_offsets describe the packed survivors and num_events bounds them. Tiled kernel only.
@@ -13,13 +12,9 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
                         uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
                         uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
                         uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
-                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out, uint64_t* digest = nullptr, uint64_t digest_capacity = 0,
+                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, bool reset_status,
+                        uint64_t* digest = nullptr, uint64_t digest_capacity = 0,
                         const uint64_t* ring_written = nullptr, uint32_t ring_capacity = 0);
-
-// argus_pair_tiled.cu
-bool argus_pair_tiled_can_fuse(uint32_t num_regions);
-bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs);
 
 // argus_aggregate.cu
 int argus_internal_aggregate(const argus_interval_t* intervals, const uint64_t* interval_offsets,
@@ -40,11 +35,6 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
                                     size_t workspace_bytes, void* cuda_stream, bool reset_status,
                                     const ArgusFuseArgs* ov_select, const uint64_t* digest = nullptr,
                                     uint64_t interval_limit = ~0ull);
-// second half of aggregation when the pairing kernel already filled the interval statistics of warp_tab
-int argus_internal_agg_finish(const argus_ambiguity_t* ambig, const uint64_t* ambig_offsets, uint32_t num_streams,
-                              uint32_t warps_per_cta, const uint32_t* cta_sm, uint32_t num_sms, uint32_t num_regions,
-                              argus_agg_t* warp_tab, argus_agg_t* cta_work, bool want_cta, argus_agg_t* sm_tab,
-                              argus_agg_t* kernel_tab, argus_status_t* status, void* cuda_stream);
 bool argus_aggregate_can_select_overlap(uint32_t num_regions, uint32_t num_pairs);
 
 // argus_ring.cu — stream_offsets (and dropped) of the records that survive in the slots of a ring container;

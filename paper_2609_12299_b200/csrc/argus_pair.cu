@@ -17,6 +17,7 @@ namespace {
 
 constexpr int kScanThreads = 1024;
 constexpr u32 kWordsPerBlock = 1024;  // bitmap words per prefix block (32768 events)
+u32 g_poll_limit = 1u << 19;          // see argus_testing_set_poll_limit
 
 // ---------------------------------------------------------------------------------------------
 // Reference-order kernel: one thread walks one stream with its stack in local memory.
@@ -265,14 +266,12 @@ extern "C" size_t argus_pair_workspace_bytes(uint64_t num_events, uint32_t num_s
 }
 
 // Whole pairing pipeline. kernel_choice: 0 = automatic, 1 = one thread per stream, 2 = tiled.
-// `fuse` (nullable) asks the tiled kernel to feed aggregation / overlap selection; *fused_out tells the
-// caller whether it did (only the tiled kernel can).
 int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
                         uint32_t num_streams, uint32_t num_regions, argus_interval_t* intervals,
                         uint64_t interval_capacity, uint64_t* interval_offsets, argus_ambiguity_t* ambig,
                         uint64_t ambig_capacity, uint64_t* ambig_offsets, argus_status_t* status, void* workspace,
-                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, const ArgusFuseArgs* fuse,
-                        bool reset_status, bool* fused_out, uint64_t* digest, uint64_t digest_capacity,
+                        size_t workspace_bytes, void* cuda_stream, int kernel_choice, bool reset_status,
+                        uint64_t* digest, uint64_t digest_capacity,
                         const uint64_t* ring_written, uint32_t ring_capacity) {
   if (!stream_offsets || !interval_offsets || !ambig_offsets || !status || !workspace) return ARGUS_ERR_INVALID_ARG;
   if ((num_events && !events) || (interval_capacity && !intervals) || (ambig_capacity && !ambig)) return ARGUS_ERR_INVALID_ARG;
@@ -299,7 +298,7 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   a.redo = 0;
   a.queue = (u32*)(ws + L.queue); a.queue_capacity = L.queue_capacity;
   a.records = (ArgusStreamRecord*)(ws + L.records); a.record_capacity = L.record_capacity;
-  memset(&a.fuse, 0, sizeof(a.fuse));
+  a.poll_limit = g_poll_limit;
   a.ring_written = (const u64*)ring_written; a.ring_capacity = ring_capacity;
   if (ring_written && (ring_capacity == 0 || kernel_choice == 1)) return ARGUS_ERR_INVALID_ARG;  // only the tiled kernel reads rings
   // a stream's intervals start at half its first event's position at the latest, so positions stay below num_events / 2 + 1
@@ -316,9 +315,6 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
     ARGUS_CHECK_LAUNCH();
     a.order = (const u32*)(ws + L.order);
   }
-  const bool fused = tiled && fuse && argus_pair_tiled_can_fuse(num_regions);
-  if (fused) a.fuse = *fuse;
-  if (fused_out) *fused_out = fused;
   for (int pass = 0; pass < 2; ++pass) {
     a.redo = pass;
     if (num_streams) {
@@ -364,7 +360,7 @@ extern "C" int argus_pair_intervals_ex(const argus_event_t* events, uint64_t num
                                        void* workspace, size_t workspace_bytes, void* cuda_stream, int kernel_choice) {
   return argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
                              interval_offsets, ambig, ambig_capacity, ambig_offsets, status, workspace, workspace_bytes,
-                             cuda_stream, kernel_choice, nullptr, true, nullptr);
+                             cuda_stream, kernel_choice, true);
 }
 
 extern "C" int argus_pair_intervals(const argus_event_t* events, uint64_t num_events, const uint64_t* stream_offsets,
@@ -392,6 +388,6 @@ extern "C" int argus_pair_intervals_ring(const argus_event_t* ring, uint32_t slo
   int rc = argus_internal_ring_offsets(written, slot_capacity, num_streams, bound, stream_offsets, dropped, status, cuda_stream);
   if (rc != ARGUS_OK) return rc;
   return argus_internal_pair(ring, bound, stream_offsets, num_streams, num_regions, intervals, interval_capacity, interval_offsets,
-                             ambig, ambig_capacity, ambig_offsets, status, workspace, workspace_bytes, cuda_stream, 2, nullptr,
-                             false, nullptr, nullptr, 0, written, slot_capacity);
+                             ambig, ambig_capacity, ambig_offsets, status, workspace, workspace_bytes, cuda_stream, 2, false,
+                             nullptr, 0, written, slot_capacity);
 }

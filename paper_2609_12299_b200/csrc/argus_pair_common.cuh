@@ -79,7 +79,7 @@ struct ArgusPairArgs {
                           // min(interval_capacity, num_events / 2 + 1), which is all a stream can reach
   const u64* ring_written; // non-null: `events` is a ring container, one slot of ring_capacity records per stream, record i of
   u32 ring_capacity;       // a stream at slot position i mod capacity; stream_offsets then describe the packed survivors
-  ArgusFuseArgs fuse;     // optional aggregation / overlap selection fed from the pairing kernel (first pass only)
+  u32 poll_limit;          // polls without any hand-over anywhere after which an idle CTA gives up (about a second)
 };
 
 #define ARGUS_NOTE_POS_BITS 48
@@ -115,8 +115,7 @@ struct ArgusSeqState {
 // Processes one event exactly as the definition states. `stk` holds ARGUS_MAX_DEPTH frames.
 // `out_base` is the position of this stream's first interval. Returns false on a device error.
 __device__ __forceinline__ bool argus_seq_step(const ArgusPairArgs& a, ArgusFrame* stk, ArgusSeqState& s, u32 stream,
-                                               u64 stream_gpos0, u64 out_base, u32 i, u64 ts, u32 tag, u32 ctx,
-                                               const ArgusFuseCtx* fx = nullptr) {
+                                               u64 stream_gpos0, u64 out_base, u32 i, u64 ts, u32 tag, u32 ctx) {
   const u32 region = tag >> 1;
   if (region >= a.num_regions) {
     argus_set_error(a.status, ARGUS_ERR_BAD_REGION, stream, i);
@@ -159,7 +158,6 @@ __device__ __forceinline__ bool argus_seq_step(const ArgusPairArgs& a, ArgusFram
     a.ctl->spec_overflow = 1;
   }
   s.n_int++;
-  if (fx && !a.redo) argus_fuse_emit(a.fuse, *fx, f.region, f.ts, incl, excl, flags);
   if (s.h > 0) stk[s.h - 1].child += incl;
   return true;
 }

@@ -14,11 +14,15 @@
 //   - every finished interval adds its inclusive time to its parent frame's accumulator (shared
 //     atomics), which gives exclusive time without ordering the threads.
 // This is exact when the tile is well nested (every end meets the frame on top with the same region
-// id). Any doubt (region mismatch, negative height, bad region id, depth overflow, level window
-// exceeded) makes the CTA redo that tile with the sequential stack machine on the carried stack, so
-// the result is always the sequential definition's.
+// id). A tile is consumed in windows: the first position where a rule fails (region mismatch, negative
+// height, bad region id, depth overflow, level window exceeded) cuts the window there; the prefix is
+// redone on its own (nothing of it had been committed), the offending marker goes through the
+// sequential stack machine on the carried stack, and a new window starts after it, so the result is
+// always the sequential definition's.
 #include "argus_internal.cuh"
 #include "argus_pair_common.cuh"
+
+#include <mutex>
 
 namespace {
 
@@ -54,13 +58,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
   return false;
 }
 
-#ifdef ARGUS_TILE_TIMING
-__device__ unsigned long long g_tile_timing[8];
-#define TT_MARK(i) do { if (tid == 0) { const long long c__ = clock64(); tt[i] += (unsigned long long)(c__ - tlast); tlast = c__; } } while (0)
-#else
-#define TT_MARK(i) do { } while (0)
-#endif
-
 constexpr int kLevelWindow = 32;  // begins of a tile may sit at levels [lbase, lbase + 32)
 constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 1 sink for "no parent", padding
 constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
@@ -92,7 +89,7 @@ __device__ __forceinline__ bool tile_pop_work(const ArgusPairArgs& a, int p, u64
     if (*done >= a.num_streams) return false;
     const u64 t = *tail;
     if (t != seen) { seen = t; idle = 0; }
-    if (++idle > (1u << 19)) {  // ~1 s without any hand-over anywhere
+    if (++idle > a.poll_limit) {  // ~1 s without any hand-over anywhere
       argus_set_error(a.status, ARGUS_ERR_TIMEOUT, 0, slot);
       return false;
     }
@@ -129,9 +126,9 @@ struct TileSmem {
   u32 cur_rec;                     // hand-over record of the stream being walked (kNoRec: none)
   u64 n_int;                       // written by the sequential redo path
   int ch;
-  int badpos;                      // first position of the window where the parallel rules fail (INT_MAX = none)
+  int badpos[2];                   // first position of the window where the parallel rules fail (INT_MAX = none); windows alternate
+                                   // between the two, so that one can be reset while stragglers still read the other
   int dead, failed;
-  u32 hot[2];                      // fused aggregation: the two regions whose count and sums threads keep in registers
 };
 
 // Latest begin of the tile at level L and position < pos (pos <= T); -1 if there is none. Written without
@@ -185,7 +182,7 @@ __device__ __forceinline__ void tile_fetch(const ArgusPairArgs& a, uint4* dst, c
   }
 }
 
-template <int NT, int E, int MINB, bool FUSE, bool RING = false>
+template <int NT, int E, int MINB, bool RING = false>
 __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   using SM = TileSmem<NT, E>;
   constexpr int T = SM::T, NW = SM::NW, NWORDS = SM::NWORDS, MAXI = SM::MAXI, NI = SM::NI;
@@ -199,39 +196,13 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     mbar_init(&sm.bar[1], 1);
     fence_mbar_init();
     sm.dead = 0;
+    sm.badpos[0] = sm.badpos[1] = 0x7fffffff;
   }
   __syncthreads();
   u32 ph0 = 0, ph1 = 0;  // mbarrier phase parities
+  int bp = 0;            // which of sm.badpos the next window uses
   const u64 off0 = a.stream_offsets[0];
   u32 tot_ctx = 0, tot_rev = 0, tot_clamp = 0;
-  // fused aggregation / overlap selection (first pass only): compact table and pair bitmap follow TileSmem
-  // (pointers into shared memory stay plain locals derived from the shared array, so that the compiler keeps
-  // their address space; a generic pointer would turn every table access into a generic load or atomic)
-  ArgusAggCell* const tabp = reinterpret_cast<ArgusAggCell*>(smem_raw + ((sizeof(SM) + 15) & ~(size_t)15));
-  u32* const pairbitsp = reinterpret_cast<u32*>(tabp + (FUSE && a.fuse.warp_tab ? a.num_regions : 0u));  // no table, no room for it
-  u32* const pairs_sm = pairbitsp + (a.num_regions + 31) / 32;  // copy of the (producer, consumer) list: [2 K]
-  const bool has_tab = FUSE && !a.redo && a.fuse.warp_tab != nullptr;
-  const bool has_pairs = FUSE && !a.redo && a.fuse.ov_spans != nullptr && a.fuse.num_pairs != 0;
-  u64* row = nullptr;      // global row of the current stream in the warp-scope table
-  u32 sm_index = 0;        // SM of the current stream's CTA
-  u64 ovc_base = 0;        // warp-uniform: current chunk of the global overlap span list
-  u32 ovc_used = a.fuse.ov_chunk;  // list slots a warp reserves at a time; none held yet
-  u32 hot0 = 0xffffffffu, hot1 = 0xffffffffu;  // hot regions of the current stream, private partial sums
-  u64 hsi0 = 0, hsi1 = 0, hse0 = 0, hse1 = 0;
-  if (has_pairs) {
-    for (u32 i = tid; i < (a.num_regions + 31) / 32; i += NT) pairbitsp[i] = 0;
-    __syncthreads();
-    for (u32 i = tid; i < 2 * a.fuse.num_pairs; i += NT) {
-      const u32 r = a.fuse.pairs[i];
-      pairs_sm[i] = r;
-      if (r < a.num_regions) atomicOr(&pairbitsp[r >> 5], 1u << (r & 31));
-    }
-    __syncthreads();
-  }
-#ifdef ARGUS_TILE_TIMING
-  unsigned long long tt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  long long tlast = clock64();
-#endif
 
   for (;;) {
     if (tid == 0) {
@@ -272,11 +243,11 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
     int ch = 0;          // carried stack height (uniform)
     u64 n_int = 0;       // intervals of this stream so far (uniform)
     bool stream_failed = false;
-    // Long streams are walked a chunk at a time (never when the aggregation table lives in this kernel: it
-    // belongs to the stream). A resumed stream takes its state from the record; a new one reserves a record.
+    // Long streams are walked a chunk at a time. A resumed stream takes its state from the record; a new one
+    // reserves a record.
     u32 ti0 = 0;
     constexpr u32 kChunkTiles = (kChunkEvents + T - 1) / T;
-    bool chunked = !FUSE && a.queue != nullptr && ntiles > kChunkTiles;
+    bool chunked = a.queue != nullptr && ntiles > kChunkTiles;
     if (rec != kNoRec) {
       const ArgusStreamRecord* r = a.records + rec;
       ti0 = __ldcg(&r->next_tile);
@@ -298,20 +269,6 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       if (rec == kNoRec) chunked = false;  // cannot happen (one record per long stream); then the stream is walked whole
     }
     const u32 ti_end = chunked && ti0 + kChunkTiles < ntiles ? ti0 + kChunkTiles : ntiles;
-    if (FUSE && !a.redo) {
-      if (has_tab) {
-        argus_fuse_init(tabp, a.num_regions, tid, NT);
-        row = a.fuse.warp_tab + (size_t)s * a.num_regions * kAggCellWords;
-        hot0 = hot1 = 0xffffffffu; hsi0 = hsi1 = hse0 = hse1 = 0;
-        if (tid < 2) sm.hot[tid] = 0xffffffffu;
-      }
-      if (has_pairs) {
-        const u32 m = a.fuse.cta_sm[s / a.fuse.warps_per_cta];
-        if (m >= a.fuse.num_sms && tid == 0) argus_set_error(a.status, ARGUS_ERR_INVALID_ARG, s, m);
-        sm_index = m < a.fuse.num_sms ? m : 0;
-      }
-      __syncthreads();
-    }
     if (tid == 0 && ti0 < ti_end) {  // first tile of this chunk, into the buffer its index selects
       const u32 start = ti0 * (u32)T;
       tile_fetch<RING>(a, (ti0 & 1) ? sm.evall + T + 2 * kCar : sm.evall, src, ring_first, start,
@@ -332,13 +289,11 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         const u32 nstart = tile_start + T;
         tile_fetch<RING>(a, b ? ev0 : ev1, src, ring_first, nstart, (n - nstart) < (u32)T ? (n - nstart) : (u32)T, &sm.bar[b ^ 1]);
       }
-      TT_MARK(0);
       {
         const bool ok = mbar_wait_bounded(&sm.bar[b], b ? ph1 : ph0);
         if (b) ph1 ^= 1; else ph0 ^= 1;
         if (!ok) sm.dead = 1;
       }
-      TT_MARK(1);
 
       // The tile is consumed in windows [w0, wend). A well-nested tile is one window. When the parallel
       // rules fail first at position p, the window is cut there: [w0, p) is redone in parallel (it is well
@@ -361,7 +316,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         }
         if (tid < kLevelWindow) sm.summ[tid] = 0;
         if (tid < ch) accb[cbase + tid] = sm.cchild[cpar][tid];  // a cut window may have added to these: start clean
-        if (tid == 0) { sm.badpos = 0x7fffffff; sm.failed = 0; accb[cbase + kSink] = 0; }
+        if (tid == 0) { sm.failed = 0; accb[cbase + kSink] = 0; }
         // block prefix sum of (begins, ends), 16 bits each: one barrier
         const u32 mine_cnt = (u32)nb | ((u32)ne << 16);
         u32 incl_cnt = mine_cnt;
@@ -404,16 +359,15 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             }
             rank += is_e ? 1 : 0;
             h += is_b ? 1 : (is_e ? -1 : 0);
-            if (viol && !seen) { atomicMin(&sm.badpos, e); seen = true; }
+            if (viol && !seen) { atomicMin(&sm.badpos[bp], e); seen = true; }
           }
         }
         __syncthreads();
-        TT_MARK(2);
 
         // ---------------- phase B: one thread per end marker: find begin and parent, feed the parent's child time ---
         u32 refs[NI];
         {
-          const int first_bad = sm.badpos;  // violations found so far; ends at or after it need no work
+          const int first_bad = sm.badpos[bp];  // violations found so far; ends at or after it need no work
 #pragma unroll
           for (int i = 0; i < NI; ++i) {
             const int rk = tid + i * NT;
@@ -431,9 +385,9 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               const int q_in = tile_latest_begin<NT, E>(sm, L - 1, lbase, e);
               const int partner = p_car ? (L < ch ? cbase + L : kBadRef) : p_in;
               const int parent = L == 0 ? cbase + kSink : (q_in >= 0 ? q_in : (L - 1 < ch ? cbase + L - 1 : kBadRef));
-              if (partner == kBadRef || parent == kBadRef) { atomicMin(&sm.badpos, e); continue; }
+              if (partner == kBadRef || parent == kBadRef) { atomicMin(&sm.badpos[bp], e); continue; }
               const uint4 pe = evb[partner];
-              if ((pe.z >> 1) != (ee.z >> 1)) { atomicMin(&sm.badpos, e); continue; }
+              if ((pe.z >> 1) != (ee.z >> 1)) { atomicMin(&sm.badpos[bp], e); continue; }
               const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
               if (ts > bts) {  // 64-bit add as two native 32-bit shared atomics; each carry is propagated exactly once
                 const u64 dlt = ts - bts;
@@ -448,17 +402,20 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           }
         }
         __syncthreads();
-        TT_MARK(3);
         if (sm.dead) {  // a bulk copy never arrived: report and leave (uniform decision)
-          if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
+          if (tid == 0) {
+            argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, tile_start);
+            atomicAdd(&a.ctl->n_done[a.redo ? 1 : 0], 1u);  // CTAs that poll for hand-overs must not wait for this stream
+          }
           return;
         }
-        const int badpos = sm.badpos;
+        const int badpos = sm.badpos[bp];
+        bp ^= 1;
+        if (tid == 0) sm.badpos[bp] = 0x7fffffff;  // nobody reads or reports into it before the next window's barriers
 
         if (badpos >= wend) {
           // ---------------- phase C: exclusive time, parent region, interval records; carried stack -------------
           const u64 pos0 = out_base + n_int;
-          u32 ovmask = 0;  // bit i: this thread's i-th interval belongs to a designated overlap region
 #pragma unroll
           for (int i = 0; i < NI; ++i) {
             const int rk = tid + i * NT;
@@ -487,56 +444,6 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               } else if (!a.redo) {
                 a.ctl->spec_overflow = 1;
               }
-              if (FUSE && !a.redo) {
-                const u32 f_region = pe.z >> 1;
-                if (has_pairs && incl && ((pairbitsp[f_region >> 5] >> (f_region & 31)) & 1u)) ovmask |= 1u << i;
-                if (has_tab) {
-                  ArgusAggCell& cell = tabp[f_region];
-                  if (f_region == hot0) { hsi0 += incl; hse0 += excl; }
-                  else if (f_region == hot1) { hsi1 += incl; hse1 += excl; }
-                  else argus_fuse_agg_sums(cell, incl, excl);
-                  argus_fuse_agg_rest(cell, row, f_region, incl, flags);
-                }
-              }
-            }
-          }
-          // Overlap selection: intervals of a designated region are rare in most traces, so the loop above only
-          // notes them; when some lane of the warp has one, the warp appends their spans together here.
-          if (has_pairs && __any_sync(0xffffffffu, ovmask != 0)) {
-#pragma unroll
-            for (int i = 0; i < NI; ++i) {
-              const bool cand = (ovmask >> i) & 1u;
-              if (!__ballot_sync(0xffffffffu, cand)) continue;
-              u32 f_region = 0xffffffffu;
-              u64 f_begin = 0, f_end = 0;
-              if (cand) {
-                const u32 d = sm.desc[tid + i * NT];
-                const uint4 ee = evb[d & 0xffffu];
-                const uint4 pe = evb[(int)(short)(refs[i] & 0xffffu)];
-                f_region = pe.z >> 1;
-                f_begin = (u64)pe.x | ((u64)pe.y << 32);
-                f_end = (u64)ee.x | ((u64)ee.y << 32);
-              }
-              for (u32 k = 0; k < 2 * a.fuse.num_pairs; ++k) {
-                const bool sel = cand && pairs_sm[k] == f_region;
-                const u32 bal = __ballot_sync(0xffffffffu, sel);
-                if (!bal) continue;
-                const u32 c = __popc(bal);
-                if (ovc_used + c > a.fuse.ov_chunk) {
-                  u64 nb64 = 0;
-                  if (lane == 0) nb64 = atomicAdd(a.fuse.ov_count, (u64)a.fuse.ov_chunk);
-                  ovc_base = __shfl_sync(0xffffffffu, nb64, 0);
-                  ovc_used = 0;
-                }
-                if (sel) {
-                  const u64 slot = ovc_base + ovc_used + __popc(bal & ((1u << lane) - 1u));
-                  if (slot < a.fuse.ov_capacity) {
-                    a.fuse.ov_spans[slot] = make_ulonglong2(f_begin, f_end);
-                    a.fuse.ov_seg[slot] = ((k >> 1) * a.fuse.num_sms + sm_index) * 2 + (k & 1u);
-                  }
-                }
-                ovc_used += c;
-              }
             }
           }
           const int new_ch = ch + win_nb - win_ne;
@@ -547,22 +454,6 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             sm.cchild[cpar ^ 1][tid] = accb[from];
             sm.cidx[cpar ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[cpar][tid];
           }
-          if (has_tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0 && warp == 0) {
-            // top two regions by count so far (counts may still be moving: only a heuristic)
-            u32 best = 0, second = 0;
-            for (u32 r = lane; r < a.num_regions; r += 32) {
-              u32 cnt = *reinterpret_cast<volatile u32*>(&tabp[r].count_out);
-#pragma unroll
-              for (u32 j = 0; j < kAggWindow; ++j) cnt += *reinterpret_cast<volatile u32*>(&tabp[r].h[j]);
-              const u32 key = ((cnt > 0xffffu ? 0xffffu : cnt) << 16) | r;
-              if (key > best) { second = best; best = key; } else if (key > second) { second = key; }
-            }
-            const u32 top = __reduce_max_sync(0xffffffffu, best);
-            const u32 cand = best == top ? second : best;
-            const u32 next = __reduce_max_sync(0xffffffffu, cand);
-            if (lane == 0) { sm.hot[0] = (top >> 16) ? (top & 0xffffu) : 0xffffffffu; sm.hot[1] = (next >> 16) ? (next & 0xffffu) : 0xffffffffu; }
-          }
-          const bool pick_hot = has_tab && hot0 == 0xffffffffu && ti == 0 && w0 == 0;
           small_streak = (wend - w0 < 32) ? small_streak + 1 : 0;
           ch = new_ch;
           n_int += (u64)win_ne;
@@ -570,8 +461,6 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           w0 = wend;
           wend = tn;
           __syncthreads();
-          if (pick_hot) { hot0 = sm.hot[0]; hot1 = sm.hot[1]; }
-          TT_MARK(4);
         } else if (badpos > w0) {
           wend = badpos;  // [w0, badpos) is well nested: do it again on its own (nothing was committed yet)
         } else {
@@ -585,15 +474,12 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           }
           __syncthreads();
           if (tid == 0) {
-            ArgusFuseCtx fx;  // the sequential machine is shared with the other pairing kernels and takes the context as a struct
-            fx.tab = has_tab ? tabp : nullptr; fx.pairbits = has_pairs ? pairbitsp : nullptr; fx.row = row; fx.sm_index = sm_index;
             ArgusSeqState st;
             st.h = ch; st.n_int = n_int; st.n_ctx = st.n_rev = st.n_clamp = 0; st.failed = false;
             bool ok = true;
             for (int e = w0; e < w0 + nseq && ok; ++e) {
               const uint4 pe = evb[e];
-              ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w,
-                                  (FUSE && !a.redo) ? &fx : nullptr);
+              ok = argus_seq_step(a, sm.fstk, st, s, gpos0, out_base, tile_start + (u32)e, (u64)pe.x | ((u64)pe.y << 32), pe.z, pe.w);
             }
             tot_ctx += st.n_ctx; tot_rev += st.n_rev; tot_clamp += st.n_clamp;
             sm.ch = st.h;
@@ -632,7 +518,10 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
 
     __syncthreads();
     if (sm.dead) {
-      if (tid == 0) argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, 0);
+      if (tid == 0) {
+        argus_set_error(a.status, ARGUS_ERR_TIMEOUT, s, 0);
+        atomicAdd(&a.ctl->n_done[a.redo ? 1 : 0], 1u);
+      }
       return;
     }
     if (!stream_failed && ti_end < ntiles) {
@@ -658,18 +547,9 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       }
       if (tid == 0) atomicAdd(&a.ctl->n_done[a.redo ? 1 : 0], 1u);
     }
-    if (has_tab) {
-      if (hot0 != 0xffffffffu) argus_fuse_agg_sums(tabp[hot0], hsi0, hse0);
-      if (hot1 != 0xffffffffu) argus_fuse_agg_sums(tabp[hot1], hsi1, hse1);
-      __syncthreads();
-      argus_fuse_flush(tabp, row, a.num_regions, tid, NT);
-    }
     __syncthreads();
   }  // streams
 
-#ifdef ARGUS_TILE_TIMING
-  if (tid == 0 && !a.redo) for (int i = 0; i < 8; ++i) atomicAdd(&g_tile_timing[i], tt[i]);
-#endif
   if (!a.redo) {
     tot_ctx = __reduce_add_sync(0xffffffffu, tot_ctx);
     tot_rev = __reduce_add_sync(0xffffffffu, tot_rev);
@@ -682,38 +562,35 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
   }
 }
 
-template <int NT, int E, int MINB, bool FUSE, bool RING = false>
+// The shared-memory opt-in and the occupancy of one instantiation belong to one device: looked up once per
+// device, under a lock (two host threads may make their first call at the same time).
+template <int NT, int E, int MINB, bool RING>
 int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
-  // the shared-memory opt-in and the occupancy belong to one device: cached per device, redone when the size changes
   constexpr int kMaxDevices = 64;
   static int grid_of[kMaxDevices];
-  static size_t smem_of[kMaxDevices];
-  size_t smem = ((sizeof(TileSmem<NT, E>) + 15) & ~(size_t)15) + 128;
-  if (FUSE) smem += (a.fuse.warp_tab ? (size_t)a.num_regions * sizeof(ArgusAggCell) : 0) + ((a.num_regions + 31) / 32) * 4 + (size_t)a.fuse.num_pairs * 8 + 16;
+  static std::mutex mu;
+  constexpr size_t smem = ((sizeof(TileSmem<NT, E>) + 15) & ~(size_t)15) + 128;
   int dev = 0;
   ARGUS_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return ARGUS_ERR_INVALID_ARG;
-  if (!grid_of[dev] || smem_of[dev] != smem) {
-    ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, FUSE, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int sms = 0, per_sm = 0;
-    ARGUS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB, FUSE, RING>, NT, smem));
-    if (per_sm < 1) return ARGUS_ERR_CUDA;
-    if (per_sm > MINB) per_sm = MINB;
-    grid_of[dev] = sms * per_sm;
-    smem_of[dev] = smem;
+  int grid_cache;
+  {
+    std::lock_guard<std::mutex> lk(mu);
+    if (!grid_of[dev]) {
+      ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_pair_tiled<NT, E, MINB, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      int sms = 0, per_sm = 0;
+      ARGUS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+      ARGUS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pair_tiled<NT, E, MINB, RING>, NT, smem));
+      if (per_sm < 1) return ARGUS_ERR_CUDA;
+      if (per_sm > MINB) per_sm = MINB;
+      grid_of[dev] = sms * per_sm;
+    }
+    grid_cache = grid_of[dev];
   }
-  const int grid_cache = grid_of[dev];
   const u32 grid = a.num_streams < (u32)grid_cache ? a.num_streams : (u32)grid_cache;
-  k_pair_tiled<NT, E, MINB, FUSE, RING><<<grid, NT, smem, stream>>>(a);
+  k_pair_tiled<NT, E, MINB, RING><<<grid, NT, smem, stream>>>(a);
   ARGUS_CHECK_LAUNCH();
   return ARGUS_OK;
-}
-
-template <int NT, int E, int MINB>
-int launch_tiled_any(const ArgusPairArgs& a, cudaStream_t stream) {
-  const bool fuse = !a.redo && (a.fuse.warp_tab || a.fuse.ov_spans);
-  return fuse ? launch_tiled<NT, E, MINB, true>(a, stream) : launch_tiled<NT, E, MINB, false>(a, stream);
 }
 
 int g_variant = 0;
@@ -722,39 +599,16 @@ int g_variant = 0;
 
 bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0; }
 
-bool argus_pair_tiled_can_fuse(uint32_t num_regions) { return num_regions <= kFuseMaxRegions; }
-bool argus_pair_tiled_can_fuse_overlap(uint32_t num_pairs) { return num_pairs <= kFuseMaxPairs; }
-
-#ifdef ARGUS_TILE_TIMING
-// Debug build only: cycles thread 0 of every CTA spent per phase (other, wait, A, B, C), summed; resets them.
-extern "C" int argus_debug_tile_timing(unsigned long long* out8) {
-  if (cudaMemcpyFromSymbol(out8, g_tile_timing, 64) != cudaSuccess) return ARGUS_ERR_CUDA;
-  unsigned long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (cudaMemcpyToSymbol(g_tile_timing, z, 64) != cudaSuccess) return ARGUS_ERR_CUDA;
-  return ARGUS_OK;
-}
-#endif
-
-// Tile shape used by the tiled kernel: 0 = automatic; 1..5 select the other compiled shapes
-// <threads, events per thread, CTAs per SM> (tuning and test aid; results do not depend on it).
+// Tile shape used by the tiled kernel: 0 = the default; 1..3 select the other compiled shapes
+// <threads, events per thread, CTAs per SM> (test aid: tiles end at other places; results do not depend on it).
 extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
-  if (a.ring_written) return launch_tiled<128, 5, 6, false, true>(a, stream);  // ring container: plain pairing, one shape
+  if (a.ring_written) return launch_tiled<128, 5, 6, true>(a, stream);  // ring container: one shape
   switch (g_variant) {
-    case 1: return launch_tiled_any<192, 5, 4>(a, stream);
-    case 2: return launch_tiled_any<320, 5, 2>(a, stream);
-    case 3: return launch_tiled_any<64, 5, 8>(a, stream);
-    case 4: return launch_tiled_any<256, 7, 2>(a, stream);
-    case 5: return launch_tiled_any<160, 5, 5>(a, stream);
-    default: {
-      // automatic. Plain pairing: six CTAs of 128 threads per SM (with streams walked in chunks the number of
-      // streams per SM does not have to divide evenly). With the aggregation table inside the kernel: four CTAs
-      // of 192 threads, or two of 320 when the table is large enough to cost CTA slots.
-      const bool hooks = !a.redo && (a.fuse.warp_tab || a.fuse.ov_spans);
-      if (!hooks) return launch_tiled_any<128, 5, 6>(a, stream);
-      const bool big_table = a.fuse.warp_tab && (size_t)a.num_regions * sizeof(ArgusAggCell) > 6 * 1024;
-      return big_table ? launch_tiled_any<320, 5, 2>(a, stream) : launch_tiled_any<192, 5, 4>(a, stream);
-    }
+    case 1: return launch_tiled<192, 5, 4, false>(a, stream);
+    case 2: return launch_tiled<64, 5, 8, false>(a, stream);
+    case 3: return launch_tiled<256, 7, 2, false>(a, stream);
+    default: return launch_tiled<128, 5, 6, false>(a, stream);  // six CTAs of 128 threads per SM
   }
 }

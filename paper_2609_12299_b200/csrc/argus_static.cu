@@ -44,7 +44,7 @@ extern "C" int argus_pair_intervals_static(const argus_event_t* events, uint64_t
   argus_prof_suppress(+1);
   const int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals,
                                      interval_capacity, interval_offsets, ambig, ambig_capacity, ambig_offsets, status,
-                                     g_scratch_ptr[dev], kStaticScratchBytes, cuda_stream, 0, nullptr, true, nullptr);
+                                     g_scratch_ptr[dev], kStaticScratchBytes, cuda_stream, 0, true);
   argus_prof_suppress(-1);
   return rc;
 }

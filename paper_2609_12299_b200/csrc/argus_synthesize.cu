@@ -1,13 +1,10 @@
 // argus_synthesize.cu — the whole hot path in one call: pair -> aggregate -> overlap.
 //
-// Pairing runs plain and writes, beside every 48-byte interval record, an 8-byte digest (region, both
-// durations, a flag bit); then ONE pass over the digests both aggregates the intervals and selects the overlap
-// spans. Hosting the table in the pairing kernel (which is bound by instruction issue and occupancy, not by
-// HBM) measured slower on every trace shape, and so did a pass over the records themselves (six times the
-// bytes). The pairing kernel's own hooks (aggregate and select while the interval is in registers: the interval
-// array is never read back) remain for calls that ask for overlap without tables and as a tuning choice
-// (argus_set_synthesize_mode). More than 400 regions or 128 pairs: the three plain calls. Results are identical
-// in every mode. argus_synthesize_ring is the same pipeline on a ring container.
+// Pairing writes, beside every 48-byte interval record, an 8-byte digest (region, both durations, a flag
+// bit); then ONE pass over the digests both aggregates the intervals and selects the overlap spans (a pass
+// over the records themselves reads six times the bytes). More than 400 regions or 128 pairs, or a call that
+// asks for no table: the three plain calls. Results are identical in every mode. argus_synthesize_ring is the
+// same pipeline on a ring container.
 #include "argus_internal.cuh"
 
 namespace {
@@ -28,8 +25,8 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
   L.agg = o; L.agg_bytes = argus_aggregate_workspace_bytes(num_events / 2, num_streams, num_regions); o += argus_align_up(L.agg_bytes, 256);
   // The span list: warps reserve slots in chunks and leave some unused, so the list is longer than the spans it
   // may hold, by a quarter or by one smallest chunk for every warp that can append, whichever is more
-  // (one block of 8 warps per stream in the aggregation passes; at most 148 x 8 blocks of 10 in the pairing kernel).
-  const uint64_t warps = (uint64_t)num_streams * 8 > 148ull * 8 * 10 ? (uint64_t)num_streams * 8 : 148ull * 8 * 10;
+  // (the aggregation passes run at most one block of 8 warps per stream).
+  const uint64_t warps = (uint64_t)num_streams * 8 > 1024 ? (uint64_t)num_streams * 8 : 1024;
   L.list_slack = num_pairs ? (max_overlap_spans / 4 > warps * 32 ? max_overlap_spans / 4 : warps * 32) : 0;
   L.list_chunk = 256;
   while (L.list_chunk > 32 && warps * L.list_chunk > L.list_slack) L.list_chunk >>= 1;
@@ -51,9 +48,8 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
 
 }  // namespace
 
-// Where argus_synthesize aggregates and selects overlap spans: -1 automatic, 0 inside the pairing kernel,
-// 1 in one pass over the intervals' digests, 2 the plain calls, 3 in one pass over the interval records
-// (tuning and test aid; results are identical).
+// Where argus_synthesize aggregates and selects overlap spans: -1 automatic, 1 in one pass over the intervals'
+// digests, 2 the plain calls, 3 in one pass over the interval records (test aid; results are identical).
 extern "C" void argus_set_synthesize_mode(int mode) { g_synth_mode = mode; }
 
 extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint32_t num_regions,
@@ -82,62 +78,37 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
   if (workspace_bytes < L.total) return ARGUS_ERR_WORKSPACE;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   char* ws = (char*)workspace;
-  const size_t row_bytes = (size_t)num_regions * sizeof(argus_agg_t);
-  argus_agg_t* warp_work = warp_tab ? warp_tab : (argus_agg_t*)(ws + L.agg);
-  argus_agg_t* cta_work = cta_tab ? cta_tab : (argus_agg_t*)(ws + L.agg + argus_align_up((size_t)num_streams * row_bytes, 256));
   const bool want_agg = warp_tab || cta_tab || sm_tab || kernel_tab;
 
   ArgusFuseArgs f;
   f.warp_tab = nullptr; f.cta_sm = cta_sm; f.warps_per_cta = warps_per_cta; f.num_sms = num_sms;
   f.pairs = pairs; f.num_pairs = num_pairs; f.ov_spans = nullptr; f.ov_seg = nullptr; f.ov_capacity = 0; f.ov_count = nullptr; f.ov_chunk = L.list_chunk;
-  // where aggregation and overlap selection happen: 0 = in the pairing kernel, 1 = in one pass over the
-  // intervals after plain pairing, 2 = the plain calls
-  const bool can_fuse = num_streams > 0 && !ring_written &&  // the kernel that reads rings has no hooks
-                        argus_pair_tiled_can_fuse(num_regions) && argus_pair_tiled_can_fuse_overlap(num_pairs);
-  int mode = 2;
-  if (num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs)) mode = 1;
-  else if (can_fuse) mode = 0;
-  if (g_synth_mode == 0 && can_fuse) mode = 0;  // tuning aid: a forced mode applies when the inputs allow it
-  if ((g_synth_mode == 1 || g_synth_mode == 3) && num_streams > 0 && want_agg &&
-      argus_aggregate_can_select_overlap(num_regions, num_pairs))
-    mode = 1;
-  if (g_synth_mode == 2) mode = 2;
+  // where aggregation and overlap selection happen: 1 = in one pass over the intervals (their digests, or the
+  // records themselves) after pairing, 2 = the plain calls
+  const bool can_one_pass = num_streams > 0 && want_agg && argus_aggregate_can_select_overlap(num_regions, num_pairs);
+  int mode = can_one_pass ? 1 : 2;
+  if (g_synth_mode == 2) mode = 2;  // test aid: a forced mode applies when the inputs allow it
   const bool list = mode != 2 && num_pairs;
-  if (mode == 0 && want_agg) {
-    f.warp_tab = (u64*)warp_work;
-    ARGUS_CUDA_TRY(cudaMemsetAsync(warp_work, 0, (size_t)num_streams * row_bytes, stream));
-  }
   if (list) {
     f.ov_spans = (ulonglong2*)(ws + L.list_spans);
     f.ov_seg = (u32*)(ws + L.list_seg);
     f.ov_capacity = L.list_capacity;
     f.ov_count = (u64*)(ws + L.list_count);
     ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_count, 0, 256, stream));
-    // the pairing kernel's hooks leave unused slots of their chunks untouched: those must read as "no span"; the
-    // aggregation passes tag them themselves
-    if (mode == 0) ARGUS_CUDA_TRY(cudaMemsetAsync(ws + L.list_seg, 0xff, (size_t)L.list_capacity * 4 + 4, stream));
   }
-  bool fused = false;
   const bool use_digest = mode == 1 && L.digest_capacity != 0 && g_synth_mode != 3;
   int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals, interval_capacity,
                                interval_offsets, ambig, ambig_capacity, ambig_offsets, status, ws + L.pair, L.pair_bytes,
-                               cuda_stream, ring_written ? 2 : 0, mode == 0 && (f.warp_tab || f.ov_spans) ? &f : nullptr,
-                               ring_written == nullptr, &fused, use_digest ? (uint64_t*)(ws + L.digest) : nullptr,
-                               L.digest_capacity, ring_written, ring_capacity);
+                               cuda_stream, ring_written ? 2 : 0, ring_written == nullptr,
+                               use_digest ? (uint64_t*)(ws + L.digest) : nullptr, L.digest_capacity, ring_written, ring_capacity);
   if (rc != ARGUS_OK) return rc;
-  if (mode == 0 && !fused) mode = 2;  // the pairing front end chose a kernel without the hooks
 
   if (want_agg) {
-    if (mode == 0) {
-      rc = argus_internal_agg_finish(ambig, ambig_offsets, num_streams, warps_per_cta, cta_sm, num_sms, num_regions, warp_work,
-                                     cta_work, cta_tab != nullptr, sm_tab, kernel_tab, status, cuda_stream);
-    } else {
-      rc = argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta,
-                                           cta_sm, num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab,
-                                           nullptr, nullptr, status, ws + L.agg, L.agg_bytes, cuda_stream, false,
-                                           mode == 1 && list ? &f : nullptr,
-                                           use_digest ? (const uint64_t*)(ws + L.digest) : nullptr, interval_capacity);
-    }
+    rc = argus_internal_aggregate_scoped(intervals, interval_offsets, ambig, ambig_offsets, num_streams, warps_per_cta,
+                                         cta_sm, num_sms, num_regions, nullptr, warp_tab, cta_tab, sm_tab, kernel_tab,
+                                         nullptr, nullptr, status, ws + L.agg, L.agg_bytes, cuda_stream, false,
+                                         mode == 1 && list ? &f : nullptr,
+                                         use_digest ? (const uint64_t*)(ws + L.digest) : nullptr, interval_capacity);
     if (rc != ARGUS_OK) return rc;
   }
   if (num_pairs) {

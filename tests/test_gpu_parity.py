@@ -338,7 +338,7 @@ def _synthesize_matches(spec, ev, offs, **kw):
     return res, st
 
 
-@pytest.fixture(params=[-1, 0, 1, 2, 3], ids=["auto", "in-pairing-kernel", "one-pass-digests", "plain-calls", "one-pass-records"])
+@pytest.fixture(params=[-1, 1, 2, 3], ids=["auto", "one-pass-digests", "plain-calls", "one-pass-records"])
 def synth_mode(request):
     """Where argus_synthesize aggregates and selects overlap spans; results must not depend on it."""
     from paper_2609_12299_b200.binding import argus_set_synthesize_mode
@@ -634,7 +634,7 @@ def test_synthesize_long_streams(idx, ctas, iters):
     _synthesize_matches(spec, ev, offs)
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_other_tile_shapes_give_the_same_result(variant):
     """The compiled alternatives to the default tile shape (threads x events per thread x CTAs per SM), on a
     malformed trace with streams several tiles long and on the one-call pipeline in every mode."""
@@ -644,7 +644,7 @@ def test_other_tile_shapes_give_the_same_result(variant):
     argus_set_tile_variant(variant)
     try:
         assert_pair_matches(ev, offs, spec.num_regions, KERNEL_TILED)
-        for mode in (0, 1):
+        for mode in (1, 2):
             argus_set_synthesize_mode(mode)
             _synthesize_matches(spec, ev, offs)
     finally:
