@@ -108,7 +108,9 @@ __global__ void __launch_bounds__(kScanThreads) k_pair_offsets(ArgusPairArgs a) 
     const u64 ex = argus_block_exclusive_scan<u64>(c, sh, &total);
     if (s < a.num_streams) {
       const u64 fin = carry + ex;
-      a.interval_offsets[s] = fin;
+      // (beyond the capacity only when the call ends with ARGUS_ERR_CAPACITY: offsets then stay inside the array, so
+      // that a call chained behind this one without a host check reads nothing it must not)
+      a.interval_offsets[s] = fin < a.interval_capacity ? fin : a.interval_capacity;
       const u64 lo = a.stream_offsets[s];
       if (lo >= off0 && fin != ((lo - off0) >> 1) && c != 0) mismatch = 1;
     }
@@ -116,7 +118,7 @@ __global__ void __launch_bounds__(kScanThreads) k_pair_offsets(ArgusPairArgs a) 
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    a.interval_offsets[a.num_streams] = carry;
+    a.interval_offsets[a.num_streams] = carry < a.interval_capacity ? carry : a.interval_capacity;
     a.ctl->total_intervals = carry;
     a.status->intervals_required = carry;
     if (carry > a.interval_capacity) {
@@ -225,7 +227,8 @@ __global__ void __launch_bounds__(256) k_ambig_offsets(AmbigArgs g) {
   if (g.p.ctl->n_notes == 0) { g.ambig_offsets[s] = 0; return; }
   const u64 off0 = g.p.stream_offsets[0];
   const u64 o = g.p.stream_offsets[s];
-  g.ambig_offsets[s] = o >= off0 ? ambig_rank(g, o - off0) : 0;
+  const u64 r = o >= off0 ? ambig_rank(g, o - off0) : 0;
+  g.ambig_offsets[s] = r < g.ambig_capacity ? r : g.ambig_capacity;  // inside the array also after ARGUS_ERR_CAPACITY
 }
 
 struct Layout {

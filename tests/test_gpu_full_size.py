@@ -1,7 +1,12 @@
 """Parity at the full benchmark sizes, in the launch configuration bench.py times (argus_synthesize on
-a trace generated in GPU memory): sampled CTAs are regenerated on the host (the generator is
-bit-identical on host and device), run through the CPU oracle one by one and compared bit for bit;
-properties that hold at any size are checked on the whole output."""
+a trace generated in GPU memory): EVERY CTA is regenerated on the host (the generator is bit-identical
+on host and device), run through the CPU oracle on its own and compared bit for bit (intervals,
+ambiguity records, warp and CTA rows, SM row and overlap), one CTA per host thread so that host memory
+stays bounded; the oracle's per-CTA tables are merged in plain numpy (sum / min / max) and compared with
+the SM- and kernel-scope tables; properties that hold at any size are checked on the whole output."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -27,16 +32,16 @@ def _run_full(spec):
     return res, st, n, d_off.cpu().numpy().view(np.uint64)
 
 
-def _check_cta(spec, res, offs, c):
+def _check_cta(spec, res, offs, c, host):
     """Everything the path produced for CTA `c` against the oracle run on that CTA alone."""
     W, R = spec.warps_per_cta, spec.num_regions
     s0, s1 = c * W, (c + 1) * W
-    ev = tg.host_streams(spec, offs, s0, s1)
+    ev = tg.host_streams(spec, offs, s0, s1, nthreads=1)
     sub = (offs[s0:s1 + 1] - offs[s0]).astype(np.uint64)
     rc, o_iv, o_ioffs, o_am, o_aoffs, o_st = oracle.pair(ev, sub, R, ambig_cap=max(len(ev) // 16, 4096))
     assert rc == 0 and int(o_st["code"]) == 0
-    ioffs = res.pair.interval_offsets.cpu().numpy().view(np.uint64)
-    aoffs = res.pair.ambig_offsets.cpu().numpy().view(np.uint64)
+    del ev
+    ioffs, aoffs = host["ioffs"], host["aoffs"]
     assert np.array_equal(ioffs[s0:s1 + 1] - ioffs[s0], o_ioffs)
     assert np.array_equal(aoffs[s0:s1 + 1] - aoffs[s0], o_aoffs)
     g_iv = res.pair.intervals[int(ioffs[s0]) * 48:int(ioffs[s1]) * 48].cpu().numpy().view(argus.INTERVAL_DTYPE)
@@ -57,9 +62,38 @@ def _check_cta(spec, res, offs, c):
         g_sm = res.agg.sm[c * row:(c + 1) * row].cpu().numpy().view(argus.AGG_DTYPE).reshape(1, R)
         assert g_sm.tobytes() == o_tabs["sm"].tobytes(), f"SM row {c} differs"
         _, o_ov, _ = oracle.overlap(o_iv, o_ioffs, W, np.zeros(1, np.uint32), 1, spec.overlap_pairs)
-        g_ov = res.overlap_numpy(spec.num_sms)[:, c]
+        g_ov = host["overlap"][:, c]
         assert g_ov.tobytes() == o_ov[:, 0].tobytes(), f"overlap of SM {c} differs"
-    return len(o_iv), len(o_am)
+    return len(o_iv), len(o_am), o_tabs["cta"][0].copy()
+
+
+_ADD = ("count", "sum_incl", "sum_excl", "n_unmatched_begin", "n_unmatched_end", "n_flagged", "hist")
+
+
+def _merge(rows):
+    """Rows of per-CTA oracle tables ([k][R]) into one row: additive fields summed, min / max taken."""
+    out = rows[0].copy()
+    for f in _ADD:
+        out[f] = np.sum([r[f] for r in rows], axis=0, dtype=np.uint64)
+    out["min_incl"] = np.min([r["min_incl"] for r in rows], axis=0)
+    out["max_incl"] = np.max([r["max_incl"] for r in rows], axis=0)
+    return out
+
+
+def _check_every_cta(spec, res, offs):
+    """All CTAs against the oracle (one CTA per host thread), then the SM and kernel tables against the merged
+    per-CTA oracle tables. Returns the intervals and ambiguity records compared."""
+    host = {"ioffs": res.pair.interval_offsets.cpu().numpy().view(np.uint64),
+            "aoffs": res.pair.ambig_offsets.cpu().numpy().view(np.uint64), "overlap": res.overlap_numpy(spec.num_sms)}
+    with ThreadPoolExecutor(max_workers=min(os.cpu_count() or 1, 16)) as pool:
+        done = list(pool.map(lambda c: _check_cta(spec, res, offs, c, host), range(spec.num_ctas)))
+    rows = [d[2] for d in done]
+    sm_want = np.stack([_merge([rows[c] for c in range(spec.num_ctas) if spec.cta_sm[c] == m]) for m in range(spec.num_sms)])
+    assert res.agg.table_numpy("sm").tobytes() == sm_want.tobytes(), "SM table differs from the merged oracle tables"
+    ker_want = _merge(rows)[None]
+    assert res.agg.table_numpy("kernel").tobytes() == ker_want.tobytes(), "kernel table differs from the merged oracle tables"
+    assert int(host["ioffs"][-1]) == sum(d[0] for d in done) and int(host["aoffs"][-1]) == sum(d[1] for d in done)
+    return sum(d[0] for d in done), sum(d[1] for d in done)
 
 
 def _check_global(spec, res, st, n, well_formed):
@@ -88,44 +122,41 @@ def _check_global(spec, res, st, n, well_formed):
     del warp
 
 
-def test_decode_megakernel_full_size_sampled():
-    """The bench workload: 1.23 G events (19.65 GB), 202 regions."""
+def test_decode_megakernel_full_size():
+    """The bench workload: 1.23 G events (19.65 GB), 202 regions; all 148 CTAs."""
     spec = tg.config(3)
     res, st, n, offs = _run_full(spec)
     assert n == 1_228_177_408
     _check_global(spec, res, st, n, well_formed=True)
-    for c in (0, 73, 147):
-        ni, na = _check_cta(spec, res, offs, c)
-        assert ni == spec.warps_per_cta * 259_328 and na == 0
+    ni, na = _check_every_cta(spec, res, offs)
+    assert ni == spec.num_streams * 259_328 and na == 0
     del res
     torch.cuda.empty_cache()
 
 
-def test_attention_full_size_sampled():
+def test_attention_full_size():
     spec = tg.config(2)
     res, st, n, offs = _run_full(spec)
     assert n == 153_513_888
     _check_global(spec, res, st, n, well_formed=True)
-    for c in (0, 101, 147):
-        _check_cta(spec, res, offs, c)
+    _check_every_cta(spec, res, offs)
     ov = res.overlap_numpy(spec.num_sms)
     assert np.all(ov["overlap_ns"] > 0)  # producer and consumer spans do overlap on every SM in this trace
     del res
     torch.cuda.empty_cache()
 
 
-def test_persistent_gemm_full_size_sampled():
+def test_persistent_gemm_full_size():
     spec = tg.config(1)
     res, st, n, offs = _run_full(spec)
     assert n == 68_672_000
     _check_global(spec, res, st, n, well_formed=True)
-    for c in (0, 64, 147):
-        _check_cta(spec, res, offs, c)
+    _check_every_cta(spec, res, offs)
     del res
     torch.cuda.empty_cache()
 
 
-def test_malformed_full_size_sampled():
+def test_malformed_full_size():
     """Dropped ends, duplicated begins and truncated streams at full size: ambiguity records, the
     second (re-basing) pass and the sequential redo of tiles that are not well nested."""
     spec = tg.config(4)
@@ -134,11 +165,9 @@ def test_malformed_full_size_sampled():
     _check_global(spec, res, st, n, well_formed=False)
     lens = np.diff(offs)
     truncated = np.nonzero(lens < np.where(np.arange(spec.num_streams) % 12 < 2, 72000, 32000) * 0.99)[0]
-    ctas = sorted({0, 147} | {int(s) // spec.warps_per_cta for s in truncated[:3]})
-    amb = 0
-    for c in ctas:
-        amb += _check_cta(spec, res, offs, c)[1]
-    assert amb > 0
+    assert len(truncated) > 0
+    ni, na = _check_every_cta(spec, res, offs)
+    assert na == int(st["ambig_required"]) > 0
     del res
     torch.cuda.empty_cache()
 

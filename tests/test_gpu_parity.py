@@ -556,6 +556,33 @@ def test_synthesize_interval_capacity_too_small(synth_mode):
     _synthesize_matches(spec, ev, offs)
 
 
+def test_synthesize_ambiguity_capacity_too_small(synth_mode):
+    """Fewer ambiguity slots than a malformed trace needs: ARGUS_ERR_CAPACITY with the required count; the offsets the
+    call leaves behind stay inside the arrays, so the aggregation behind it (no host check in between) reads nothing
+    beyond them; the same buffers work again with enough room."""
+    spec = tg.config(4).scaled(3, 300)
+    ev, offs = tg.generate_host(spec)
+    rc, o_iv, o_ioffs, o_am, o_aoffs, o_st = oracle.pair(ev, offs, spec.num_regions)
+    assert len(o_am) > 40
+    d_ev, d_off = to_dev(ev, offs)
+    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(DEV)
+    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(DEV)
+    cap = len(o_am) // 3
+    res = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms, pairs,
+                                 ambig_capacity=cap)
+    st = res.fetch_status()
+    assert int(st["code"]) == 4 and int(st["ambig_required"]) == len(o_am)
+    assert int(res.pair.ambig_offsets.cpu().numpy().view(np.uint64).max()) <= cap
+    # the plain chain: pairing that overflows, then aggregation of what it left, without looking at the status
+    pr = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions, ambig_capacity=cap, interval_capacity=len(o_iv) // 2)
+    ag = argus.argus_aggregate(pr.intervals, pr.interval_offsets, pr.ambig, pr.ambig_offsets, spec.warps_per_cta, cta_sm,
+                               spec.num_sms, spec.num_regions)
+    torch.cuda.synchronize()
+    assert int(pr.fetch_status()["code"]) == 4
+    assert int(pr.interval_offsets.cpu().numpy().view(np.uint64).max()) <= len(o_iv) // 2
+    _synthesize_matches(spec, ev, offs)
+
+
 def test_overlap_offsets_beyond_the_interval_array_are_reported():
     spec = tg.config(1).scaled(2, 40)
     ev, offs = tg.generate_host(spec)

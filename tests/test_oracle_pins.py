@@ -259,6 +259,7 @@ def test_aggregate_matches_numpy_groupby_and_rollup():
         hist = np.zeros((ncell, 64), np.uint64)
         np.add.at(hist, (cell, bins), 1)
         assert np.array_equal(tab["hist"].reshape(ncell, 64), hist)
+        assert np.array_equal(tab["n_flagged"].ravel(), np.bincount(cell[iv["flags"] != 0], minlength=ncell).astype(np.uint64))
         akeys = fn(am["stream"].astype(np.int64)) * R + (am["tag"] >> 1).astype(np.int64)
         ub = np.bincount(akeys[am["kind"] != 1], minlength=ncell).astype(np.uint64)
         ue = np.bincount(akeys[am["kind"] == 1], minlength=ncell).astype(np.uint64)
