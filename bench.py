@@ -27,7 +27,13 @@ if ROOT not in sys.path:
 METRIC = "marker events/sec (pair+aggregate, 1 B200) and % of HBM roofline"  # the step also runs the overlap stage
 UNIT = "events/s"
 ALG_BYTES_PER_EVENT = 40.0  # 16 B event read + 48 B interval written per 2 events
-NCU_DRAM_BYTES_PER_EVENT = (614.276352e6 + 1018.343e6) / 38380544  # pairing kernel, ncu capture summarised in profiles/
+# DRAM traffic of the pairing kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum of one launch)
+# on a small case of the bench workload; the full trace is too large for a multi-pass capture, and the kernel's
+# traffic grows in proportion to the events, so the JSON line scales it to a full launch and says so.
+TRAFFIC_CAPTURE = {"workload": "decode_megakernel", "iters": 8, "events": 38380544, "dram_bytes_read": 614.679808e6,
+                   "dram_bytes_write": 1018.509e6, "kernel": "k_pair_tiled<128,5,6>",
+                   "command": "ncu --set full --clock-control none -k regex:k_pair_tiled -c 1 python bench.py --workload 3 "
+                              "--iters 8 --steps 1 --no-e2e --no-cpu-baseline --no-other"}
 
 
 def load_peaks():
@@ -165,6 +171,8 @@ def main():
     ap.add_argument("--three-calls", action="store_true",
                     help="time argus_pair_intervals + argus_aggregate + argus_overlap instead of the one-call argus_synthesize")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-other", action="store_true",
+                    help="skip the secondary records (three plain calls, corrupted marker, the other trace shapes)")
     ap.add_argument("--no-combine", action="store_true",
                     help="N > 1: do not combine the ranks' kernel-scope tables at the end of every step")
     args = ap.parse_args()
@@ -189,9 +197,6 @@ def main():
     import paper_2609_12299_b200 as argus
 
     argus.load_library()  # raises if the CUDA library was not built: there is no fallback
-    if os.environ.get("ARGUS_TILE_VARIANT"):
-        from paper_2609_12299_b200.binding import argus_set_tile_variant
-        argus_set_tile_variant(int(os.environ["ARGUS_TILE_VARIANT"]))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device")
     dev = torch.device("cuda", local_rank)
@@ -205,72 +210,91 @@ def main():
     d_ev, d_off = tg.generate_cuda(spec, dev)
     n_events = d_ev.numel() // 16
     S = spec.num_streams
-    cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(dev)
-    pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(dev)
-    icap = n_events // 2
-    acap = max(n_events // 64, 4096)
-    ov_ws = torch.empty(min(argus.argus_overlap_workspace_bytes(icap, S, len(spec.overlap_pairs), spec.num_sms),
-                            2 << 30), dtype=torch.uint8, device=dev)
-    state = {"pair": None, "agg": None, "syn": None}
-    mos = max(n_events // 8, 1 << 16)  # overlap spans the one-call pipeline may select
-
-    def step_three_calls():
-        state["pair"] = p = argus.argus_pair_intervals(d_ev, d_off, spec.num_regions, interval_capacity=icap,
-                                                       ambig_capacity=acap, out=state["pair"])
-        state["agg"] = argus.argus_aggregate(p.intervals, p.interval_offsets, p.ambig, p.ambig_offsets,
-                                             spec.warps_per_cta, cta_sm, spec.num_sms, spec.num_regions, out=state["agg"])
-        state["ov"] = argus.argus_overlap(p.intervals, icap, p.interval_offsets, spec.warps_per_cta, cta_sm, spec.num_sms,
-                                          pairs, workspace=ov_ws)
-
-    def step_one_call():
-        state["syn"] = r = argus.argus_synthesize(d_ev, d_off, spec.num_regions, spec.warps_per_cta, cta_sm, spec.num_sms,
-                                                  pairs, interval_capacity=icap, ambig_capacity=acap,
-                                                  max_overlap_spans=mos, out=state["syn"])
-        state["pair"], state["agg"], state["ov"] = r.pair, r.agg, (r.overlap, r.status)
-
-    local_step = step_three_calls if args.three_calls else step_one_call
     combine = world > 1 and not args.no_combine
-
-    def step():
-        local_step()
-        if combine:  # the path's one exchange step: R x 576 bytes, all-reduced (sum / min / max)
-            combine_kernel_tables(state["agg"].kernel, world)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    st = state["pair"].fetch_status()
-    if int(st["code"]) != 0:
-        raise RuntimeError(f"device status after warm-up: {st}")
+    class Runner:
+        """One workload resident on the device: its step functions and their output buffers (allocated once)."""
 
+        def __init__(self, spec, d_ev, d_off):
+            self.spec, self.d_ev, self.d_off = spec, d_ev, d_off
+            self.n = d_ev.numel() // 16
+            self.cta_sm = torch.from_numpy(spec.cta_sm.view(np.int32)).to(dev)
+            self.pairs = torch.from_numpy(spec.overlap_pairs.view(np.int32)).to(dev)
+            self.icap = self.n // 2
+            self.acap = max(self.n // 64, 4096)
+            self.mos = max(self.n // 8, 1 << 16)  # overlap spans the one-call pipeline may select
+            self.state = {"pair": None, "agg": None, "syn": None, "ov": None}
+            self.ov_ws = None
+
+        def step_three_calls(self):
+            sp, st = self.spec, self.state
+            if self.ov_ws is None:
+                self.ov_ws = torch.empty(min(argus.argus_overlap_workspace_bytes(self.icap, sp.num_streams, len(sp.overlap_pairs),
+                                                                                 sp.num_sms), 2 << 30), dtype=torch.uint8, device=dev)
+            st["pair"] = p = argus.argus_pair_intervals(self.d_ev, self.d_off, sp.num_regions, interval_capacity=self.icap,
+                                                        ambig_capacity=self.acap, out=st["pair"])
+            st["agg"] = argus.argus_aggregate(p.intervals, p.interval_offsets, p.ambig, p.ambig_offsets, sp.warps_per_cta,
+                                              self.cta_sm, sp.num_sms, sp.num_regions, out=st["agg"])
+            st["ov"] = argus.argus_overlap(p.intervals, self.icap, p.interval_offsets, sp.warps_per_cta, self.cta_sm, sp.num_sms,
+                                           self.pairs, workspace=self.ov_ws)
+
+        def step_one_call(self):
+            sp, st = self.spec, self.state
+            st["syn"] = r = argus.argus_synthesize(self.d_ev, self.d_off, sp.num_regions, sp.warps_per_cta, self.cta_sm,
+                                                   sp.num_sms, self.pairs, interval_capacity=self.icap, ambig_capacity=self.acap,
+                                                   max_overlap_spans=self.mos, out=st["syn"])
+            st["pair"], st["agg"], st["ov"] = r.pair, r.agg, (r.overlap, r.status)
+
+        def check_status(self, where):
+            for name in ("pair", "agg"):
+                code = int(argus.argus_status_fetch(self.state[name].status)["code"])
+                if code != 0:
+                    raise RuntimeError(f"device status {code} in {name} {where}")
+            if int(argus.argus_status_fetch(self.state["ov"][1])["code"]) != 0:
+                raise RuntimeError(f"device status in overlap {where}")
+
+        def timed(self, local_step, steps, warmup, exchange=False, sampler=None):
+            """`warmup` untimed steps, then `steps` steps between CUDA events; kernel times from the library's own events."""
+            def step():
+                local_step()
+                if exchange:  # the path's one exchange step: R x 576 bytes, all-reduced (sum / min / max)
+                    combine_kernel_tables(self.state["agg"].kernel, world)
+            for _ in range(warmup):
+                step()
+            barrier()
+            self.check_status("after warm-up")
+            argus.argus_profile_read()
+            argus.argus_profile_enable(True)
+            launches0 = argus.argus_launch_count()
+            if sampler:
+                sampler.start()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                step()
+            e1.record()
+            barrier()
+            if sampler:
+                sampler.stop()
+            launches = argus.argus_launch_count() - launches0
+            argus.argus_profile_enable(False)
+            prof_ms, prof_n = argus.argus_profile_read()
+            self.check_status("after the timed region")
+            kernel_ms = {k: prof_ms[k] / max(prof_n[k], 1) for k in ("pair", "aggregate", "overlap")}
+            return e0.elapsed_time(e1), launches, kernel_ms, step
+
+    main_run = Runner(spec, d_ev, d_off)
+    local_step = main_run.step_three_calls if args.three_calls else main_run.step_one_call
     sampler = ClockSampler(dev)
-    argus.argus_profile_read()
-    argus.argus_profile_enable(True)
-    launches0 = argus.argus_launch_count()
-    sampler.start()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    sampler.stop()
-    launches = argus.argus_launch_count() - launches0
-    argus.argus_profile_enable(False)
-    prof_ms, prof_n = argus.argus_profile_read()
-    ms_total = e0.elapsed_time(e1)
-    for name in ("pair", "agg"):
-        code = int(argus.argus_status_fetch(state[name].status)["code"])
-        if code != 0:
-            raise RuntimeError(f"device status {code} in {name} after the timed region")
-    if int(argus.argus_status_fetch(state["ov"][1])["code"]) != 0:
-        raise RuntimeError("device status in overlap after the timed region")
+    ms_total, launches, kernel_ms, step = main_run.timed(local_step, args.steps, args.warmup, combine, sampler)
+    state = main_run.state
+    prof_pair_ms = kernel_ms["pair"]
 
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
@@ -278,16 +302,21 @@ def main():
 
     # roofline of the dominant kernel (the pairing kernel): algorithmic bytes / its own launch time
     peak, peak_src = load_peaks()
-    pair_ms = prof_ms["pair"] / max(prof_n["pair"], 1)
+    pair_ms = prof_pair_ms
     achieved = ALG_BYTES_PER_EVENT * n_events / (pair_ms * 1e-3) / 1e9 if pair_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "tiled pairing kernel (k_pair_tiled)", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "peak_source": peak_src,
-                "traffic": NCU_DRAM_BYTES_PER_EVENT * n_events if args.workload == 3 else None,
-                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on a 38.4 M-event "
-                                  "case of the same trace, scaled by events (profiles/)",
+    step_gbs = ALG_BYTES_PER_EVENT * n_events / (ms_per_step * 1e-3) / 1e9
+    scaled = (TRAFFIC_CAPTURE["dram_bytes_read"] + TRAFFIC_CAPTURE["dram_bytes_write"]) / TRAFFIC_CAPTURE["events"] * n_events
+    roofline = {"bound": "hbm", "kernel": "tiled pairing kernel (k_pair_tiled), the dominant kernel, timed alone",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "frac_of_8TBs_nominal": achieved / 8000.0, "peak_source": peak_src,
+                "traffic": scaled if spec.name == TRAFFIC_CAPTURE["workload"] else None,
+                "traffic_source": "ncu capture of one launch on a smaller case of the same trace, scaled by events",
+                "traffic_capture": TRAFFIC_CAPTURE,
                 "ms_per_launch": pair_ms, "algorithmic_bytes_per_event": ALG_BYTES_PER_EVENT,
-                "pipeline_frac": ALG_BYTES_PER_EVENT * n_events / (ms_per_step * 1e-3) / 1e9 / peak}
-    kernel_ms = {k: prof_ms[k] / max(prof_n[k], 1) for k in ("pair", "aggregate", "overlap")}
+                # the whole step (every kernel of pair + aggregate + overlap) by the accounting of a fused pair + aggregate
+                "step": {"achieved": step_gbs, "frac": step_gbs / peak, "frac_of_8TBs_nominal": step_gbs / 8000.0,
+                         "ms": ms_per_step},
+                "pipeline_frac": step_gbs / peak}
     if kernel_ms["aggregate"] > 0:
         # the pass over the intervals' digests (aggregation + overlap span selection): 8 B read per interval; it is
         # bound by instruction issue and shared-memory atomics, the HBM figure is given for scale
@@ -304,6 +333,7 @@ def main():
         pin_off = torch.empty(S + 1, dtype=torch.int64, pin_memory=True)
         pin_off.copy_(d_off)
         agg = state["agg"]
+        # tables, overlap, offsets and status come back; the interval array (48 B per interval) stays on the device
         outs = [agg.kernel, agg.sm, agg.cta, state["ov"][0], state["pair"].interval_offsets, state["pair"].status]
         pin_out = [torch.empty(o.numel(), dtype=o.dtype, pin_memory=True) for o in outs]
         torch.cuda.synchronize(dev)
@@ -329,8 +359,51 @@ def main():
         e2e = {"value": whole_job_rate(n_events, world, ms / args.e2e_steps), "unit": UNIT,
                "h2d_bytes_per_step": int(pin_ev.numel() + pin_off.numel() * 8),
                "d2h_bytes_per_step": int(sum(p.numel() * p.element_size() for p in pin_out)),
-               "steps": args.e2e_steps, "ms_per_step": ms / args.e2e_steps}
+               "steps": args.e2e_steps, "ms_per_step": ms / args.e2e_steps,
+               "note": "host events in, tables + overlap + offsets + status out; the interval array stays on the device "
+                       f"(copying it back would add {n_events // 2 * 48} bytes per step)"}
         del pin_ev
+
+    # The other numbers the contract asks for, a few steps each (world size 1 only): the plain three-call sequence and
+    # a single corrupted marker on the bench workload, and the one-call step on the other trace shapes.
+    other = None
+    if world == 1 and not args.no_other and not args.three_calls:
+        other = []
+
+        def record(run, name, step_name, local, steps):
+            ms, _, kms, _ = run.timed(local, steps, 3)
+            per = ms / steps
+            gbs = ALG_BYTES_PER_EVENT * run.n / (per * 1e-3) / 1e9
+            other.append({"workload": name, "step": step_name, "events": run.n, "steps": steps, "ms_per_step": per,
+                          "events_per_s": run.n / (per * 1e-3), "pipeline_frac": gbs / peak, "kernel_ms": kms})
+
+        three = Runner(spec, d_ev, d_off)  # its own output buffers
+        record(three, spec.name, "argus_pair_intervals + argus_aggregate + argus_overlap (three plain calls)",
+               three.step_three_calls, max(args.steps // 2, 3))
+        del three
+        torch.cuda.empty_cache()
+        if spec.name == "decode_megakernel" and not args.iters:
+            # one end marker of stream 0 turned into the end of another region: stream 0 loses an interval, every later
+            # stream's base moves, and the second pairing pass has to re-write them
+            pos = (int(d_off[0].item()) + 5) * 16 + 8
+            old = int(d_ev[pos].item())
+            assert old == 7  # end of sync_wait (region 3)
+            d_ev[pos] = 5    # end of tile_work (region 2)
+            try:
+                record(main_run, spec.name + " with one corrupted end marker in stream 0", "argus_synthesize",
+                       main_run.step_one_call, max(args.steps // 2, 3))
+                other[-1]["ambig_required"] = int(state["pair"].fetch_status()["ambig_required"])
+            finally:
+                d_ev[pos] = old
+        for idx in (1, 2, 4):
+            if idx == args.workload:
+                continue
+            sp = tg.config(idx)
+            o_ev, o_off = tg.generate_cuda(sp, dev)
+            run = Runner(sp, o_ev, o_off)
+            record(run, sp.name, "argus_synthesize", run.step_one_call, 10)
+            del run, o_ev, o_off
+            torch.cuda.empty_cache()
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -377,7 +450,7 @@ def main():
                                 "argus_synthesize (pair + aggregate + overlap in one call)") + " on one trace per GPU",
                        "exchange": "kernel-scope tables of all ranks combined by all-reduce every step" if combine else "none"},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu_baseline, "kernel_ms": kernel_ms,
+            "cpu_baseline": cpu_baseline, "kernel_ms": kernel_ms, "other": other,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
