@@ -175,7 +175,15 @@ def main():
                     help="skip the secondary records (three plain calls, corrupted marker, the other trace shapes)")
     ap.add_argument("--no-combine", action="store_true",
                     help="N > 1: do not combine the ranks' kernel-scope tables at the end of every step")
+    ap.add_argument("--suite", default="main", choices=["main", "secondary"],
+                    help="secondary: timings of the entry points beyond the step (bench_secondary.py), one JSON line each")
+    ap.add_argument("--what", default="join", choices=["scoped", "pcmap", "ring", "join"], help="--suite secondary: which one")
+    ap.add_argument("--queries", type=int, default=2000, help="--suite secondary --what join: number of queries")
     args = ap.parse_args()
+    if args.suite == "secondary":
+        import bench_secondary
+        bench_secondary.run(args.what, iters=args.iters, queries=args.queries)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2609_12299_b200.multirank import combine_kernel_tables, max_over_ranks, rank_env, rank_spec, whole_job_rate

@@ -1,9 +1,10 @@
-"""Timings of the entry points beyond the benchmark's step, on one GPU, with CUDA events:
+"""Timings of the entry points beyond the benchmark's step, on one GPU, with CUDA events (the secondary
+suite of bench.py):
 
-    python -m paper_2609_12299_b200.measure scoped   # argus_aggregate_scoped / argus_overlap_scoped on trace 3
-    python -m paper_2609_12299_b200.measure pcmap    # PC-to-region mapping and attribution on a mapping run
-    python -m paper_2609_12299_b200.measure ring     # pairing from a ring container: packed copy first, or directly
-    python -m paper_2609_12299_b200.measure join     # cross-run join against a whole trace, plain and grouped by stream
+    python bench.py --suite secondary --what scoped   # argus_aggregate_scoped / argus_overlap_scoped on trace 3
+    python bench.py --suite secondary --what pcmap    # PC-to-region mapping and attribution on a mapping run
+    python bench.py --suite secondary --what ring     # pairing from a ring container: packed copy first, or directly
+    python bench.py --suite secondary --what join     # cross-run join against a whole trace: per query, grouped, hashed
 
 Each line printed is one JSON object: what ran, its time (best of the repetitions after warm-up), the
 algorithmic bytes it has to move and the fraction of the measured HBM copy bandwidth that amounts to.
@@ -18,11 +19,11 @@ import os
 import numpy as np
 import torch
 
-from . import binding as argus
-from . import tracegen as tg
-from .tracegen.mapping import mapping_trace
+import paper_2609_12299_b200.binding as argus
+from paper_2609_12299_b200 import tracegen as tg
+from paper_2609_12299_b200.tracegen.mapping import mapping_trace
 
-_ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+_ROOT = os.path.dirname(os.path.abspath(__file__))
 
 
 def _peak_gbs() -> float:
@@ -189,27 +190,21 @@ def run_join(iters: int, queries: int):
     ms = _time(lambda: argus.argus_join_samples_grouped(iv, idx, iv, offs, spec.num_streams), reps=3, warmup=1)
     _line(f"argus_join_samples_grouped, {queries} queries (every query reads its own stream's samples)", ms,
           queries * 32.0 * n_iv / spec.num_streams, intervals=n_iv, workload=spec.name)
+    ws = torch.empty(argus.load_library().argus_join_workspace_bytes(queries), dtype=torch.uint8, device=dev)
+    ms = _time(lambda: argus.argus_join_samples_hashed(iv, idx, iv, ws), reps=3, warmup=1)
+    _line(f"argus_join_samples_hashed, {queries} queries (one pass over the samples in whatever order they lie)", ms,
+          48.0 * n_iv, intervals=n_iv, workload=spec.name)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["scoped", "pcmap", "ring", "join"])
-    ap.add_argument("--queries", type=int, default=2000, help="`join`: queries of the grouped join")
-    ap.add_argument("--shift-tokens", type=int, default=100, help="`ring`: tokens written before the surviving records (0: no wrap)")
-    ap.add_argument("--iters", type=int, default=0, help="tokens per stream of the decode trace (0: full size for `scoped`, 24 for `pcmap`)")
-    ap.add_argument("--pcs", type=int, default=70_560)
-    ap.add_argument("--execs-per-begin", type=int, default=2)
-    a = ap.parse_args()
+def run(what: str, iters: int = 0, queries: int = 2000, shift_tokens: int = 100, pcs: int = 70_560, execs_per_begin: int = 2):
     argus.load_library()
-    if a.what == "scoped":
-        run_scoped(a.iters)
-    elif a.what == "ring":
-        run_ring(a.iters, a.shift_tokens)
-    elif a.what == "join":
-        run_join(a.iters, a.queries)
+    if what == "scoped":
+        run_scoped(iters)
+    elif what == "ring":
+        run_ring(iters, shift_tokens)
+    elif what == "join":
+        run_join(iters, queries)
+    elif what == "pcmap":
+        run_pcmap(iters or 24, pcs, execs_per_begin)
     else:
-        run_pcmap(a.iters or 24, a.pcs, a.execs_per_begin)
-
-
-if __name__ == "__main__":
-    main()
+        raise ValueError(what)

@@ -444,6 +444,22 @@ int argus_join_samples_grouped(const argus_interval_t* reference /*device*/, uin
                                argus_join_t* out /*device [Q]*/, argus_status_t* status /*device*/,
                                void* cuda_stream);
 
+/* The same join for probe-run samples in ANY order, in one pass over `samples` for all queries
+ * together (Section 3.5: evidence is joined by region identity and execution context, never by
+ * comparing timestamps across runs): the distinct (stream, region, ctx) keys of the queries go
+ * into a hash table in the workspace, every sample is read once and looked up, matching values
+ * are appended to their key's list (at most ARGUS_JOIN_MAX_SAMPLES are kept and ranked; count
+ * and sum stay exact, ARGUS_ERR_CAPACITY reports the overflow), and one block per query sorts
+ * and ranks. Cost: one read of `samples` whatever the number of queries. workspace: device
+ * memory, 256-byte aligned, argus_join_workspace_bytes(num_queries) bytes, owned by the caller,
+ * contents unspecified before and after. Same results as argus_join_samples. */
+size_t argus_join_workspace_bytes(uint32_t num_queries);
+int argus_join_samples_hashed(const argus_interval_t* reference /*device*/, uint64_t num_reference,
+                              const uint64_t* ref_index /*device [Q]*/, uint32_t num_queries,
+                              const argus_interval_t* samples /*device*/, uint64_t num_samples,
+                              argus_join_t* out /*device [Q]*/, argus_status_t* status /*device*/,
+                              void* workspace /*device*/, size_t workspace_bytes, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------------
  * Ring-buffer input — a second container for the marker records of Section 3.2: tracers
  * commonly give every warp a fixed slot of slot_capacity records and let it wrap. The paper

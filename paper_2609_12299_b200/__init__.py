@@ -11,7 +11,7 @@ from .binding import (AGG_DTYPE, AMBIG_DTYPE, EVENT_DTYPE, INTERVAL_DTYPE, OVERL
                       argus_version, library_path, load_library, pair_aggregate_host, argus_synthesize,
                       argus_synthesize_workspace_bytes, SynthesizeResult, argus_pair_intervals_static, ArgusScope,
                       ScopedAggregateResult, argus_aggregate_scoped, argus_overlap_scoped, encode_map_events,
-                      argus_map_pc_counts, argus_attribute, argus_join_samples, argus_join_samples_grouped, JOIN_DTYPE,
+                      argus_map_pc_counts, argus_attribute, argus_join_samples, argus_join_samples_grouped, argus_join_samples_hashed, JOIN_DTYPE,
                       argus_ring_linearise, argus_pair_intervals_ring, argus_synthesize_ring)
 
 __all__ = [
@@ -22,5 +22,5 @@ __all__ = [
     "argus_profile_enable", "argus_profile_read", "argus_synthesize", "argus_synthesize_workspace_bytes",
     "SynthesizeResult", "argus_pair_intervals_static", "ArgusScope", "ScopedAggregateResult", "argus_aggregate_scoped",
     "argus_overlap_scoped", "encode_map_events", "argus_map_pc_counts", "argus_attribute",
-    "argus_join_samples", "argus_join_samples_grouped", "JOIN_DTYPE", "argus_ring_linearise", "argus_pair_intervals_ring", "argus_synthesize_ring",
+    "argus_join_samples", "argus_join_samples_grouped", "argus_join_samples_hashed", "JOIN_DTYPE", "argus_ring_linearise", "argus_pair_intervals_ring", "argus_synthesize_ring",
 ]

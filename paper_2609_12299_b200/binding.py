@@ -80,6 +80,10 @@ def load_library():
     lib.argus_join_samples_grouped.argtypes = [vp, u64, vp, u32, vp, u64, vp, u32, u32, vp, vp, vp]
     lib.argus_join_samples_grouped.restype = ci
     lib.argus_join_samples.restype = ci
+    lib.argus_join_workspace_bytes.argtypes = [u32]
+    lib.argus_join_workspace_bytes.restype = sz
+    lib.argus_join_samples_hashed.argtypes = [vp, u64, vp, u32, vp, u64, vp, vp, vp, sz, vp]
+    lib.argus_join_samples_hashed.restype = ci
     lib.argus_ring_linearise.argtypes = [vp, u32, vp, u32, vp, u64, vp, vp, vp, vp]
     lib.argus_ring_linearise.restype = ci
     lib.argus_pair_intervals_ring.argtypes = [vp, u32, vp, u32, u32, vp, vp, vp, u64, vp, vp, u64, vp, vp, vp, sz, vp]
@@ -459,6 +463,25 @@ def argus_join_samples(reference: torch.Tensor, ref_index: torch.Tensor, samples
                                 samples.numel() // 48, _ptr(out), _ptr(status), _stream_ptr(dev))
     if rc != 0:
         raise ArgusError(rc, "argus_join_samples")
+    return out, status
+
+
+def argus_join_samples_hashed(reference: torch.Tensor, ref_index: torch.Tensor, samples: torch.Tensor,
+                              workspace: torch.Tensor | None = None):
+    """As argus_join_samples, in one pass over `samples` for all queries together (samples in any order)."""
+    lib = load_library()
+    dev = reference.device
+    Q = ref_index.numel()
+    out = _bytes(Q * 64, dev)
+    status = _bytes(64, dev)
+    need = lib.argus_join_workspace_bytes(Q)
+    if workspace is None:
+        workspace = _bytes(max(need, 256), dev)
+    rc = lib.argus_join_samples_hashed(_ptr(reference), reference.numel() // 48, _ptr(ref_index), Q, _ptr(samples),
+                                       samples.numel() // 48, _ptr(out), _ptr(status), _ptr(workspace), workspace.numel(),
+                                       _stream_ptr(dev))
+    if rc != 0:
+        raise ArgusError(rc, "argus_join_samples_hashed")
     return out, status
 
 
