@@ -21,10 +21,15 @@
  *   - All structs are plain little-endian PODs, naturally aligned, with no padding.
  *   - Every pointer named "device" below is a CUDA device pointer on the current device;
  *     `cuda_stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
- *   - The caller owns every buffer. The three operations allocate nothing, keep no state
- *     between calls, enqueue their kernels on `cuda_stream` and return without
+ *   - The caller owns every buffer. The operations allocate nothing, keep nothing of a call
+ *     for the next one, enqueue their kernels on `cuda_stream` and return without
  *     synchronising; results are valid once the stream reaches that point, so
  *     pair -> aggregate -> overlap on one stream needs no host synchronisation.
+ *   - What the library does keep: per device, the launch parameters of its kernels (looked
+ *     up on first use, under a lock) and, for argus_pair_intervals_static, the address of
+ *     its scratch array; process-wide, the test and measurement switches declared in
+ *     argus_testing.h. Host threads may call the operations concurrently, each call with
+ *     its own buffers, workspace and stream.
  *   - Return value: host-detectable errors (ARGUS_OK, ARGUS_ERR_INVALID_ARG,
  *     ARGUS_ERR_WORKSPACE, ARGUS_ERR_CUDA). Conditions found on the device are written to
  *     `status->code` (first error wins); on a device error the output arrays are
@@ -181,21 +186,6 @@ int argus_pair_intervals(const argus_event_t* events /*device*/, uint64_t num_ev
                          uint64_t* ambig_offsets /*device [S+1] out*/,
                          argus_status_t* status /*device*/, void* workspace /*device*/,
                          size_t workspace_bytes, void* cuda_stream);
-
-/* Same operation with an explicit kernel choice, for tests and profiling:
- * kernel_choice 0 = automatic, 1 = one thread per stream (sequential stack, any input),
- * 2 = tiled kernel (CTAs walk streams tile by tile, long streams a chunk at a time, and hand
- * the markers that break the nesting to the sequential stack). All choices produce identical
- * output. */
-int argus_pair_intervals_ex(const argus_event_t* events /*device*/, uint64_t num_events,
-                            const uint64_t* stream_offsets /*device [S+1]*/,
-                            uint32_t num_streams, uint32_t num_regions,
-                            argus_interval_t* intervals /*device*/, uint64_t interval_capacity,
-                            uint64_t* interval_offsets /*device [S+1] out*/,
-                            argus_ambiguity_t* ambig /*device*/, uint64_t ambig_capacity,
-                            uint64_t* ambig_offsets /*device [S+1] out*/,
-                            argus_status_t* status /*device*/, void* workspace /*device*/,
-                            size_t workspace_bytes, void* cuda_stream, int kernel_choice);
 
 /* ---------------------------------------------------------------------------------------
  * argus_pair_intervals_static — no counterpart in the paper: a convenience variant of
@@ -567,26 +557,6 @@ const char* argus_strerror(int code);
 
 /* Library version: major * 10000 + minor * 100 + patch. */
 int argus_version(void);
-
-/* Measurement helpers (host-side bookkeeping only; they change no result).
- * argus_launch_count: kernels this library has launched since it was loaded.
- * argus_profile_enable(1): from now on each operation records a CUDA event pair on its stream
- * around its dominant kernel (slot 0 = pairing kernel of argus_pair_intervals, 1 = per-stream
- * accumulation kernel of argus_aggregate, 2 = sort kernel of argus_overlap, 3 = reserved).
- * argus_profile_read: waits for the recorded events, writes per slot the summed kernel time in
- * milliseconds and the number of recorded launches (arrays of 4), and forgets them. */
-unsigned long long argus_launch_count(void);
-void argus_profile_enable(int on);
-int argus_profile_read(double* ms_total /*host [4]*/, unsigned long long* launches /*host [4]*/);
-
-/* Tuning and test aids (process-wide; results never depend on them).
- * argus_set_synthesize_mode: where argus_synthesize aggregates and selects overlap spans: -1 automatic,
- * 0 inside the pairing kernel, 1 in one pass over the intervals' digests, 2 the three plain operations,
- * 3 in one pass over the interval records. A mode the inputs do not allow falls back to the automatic choice.
- * argus_set_tile_variant: shape of the tiled pairing kernel, 0 = automatic, 1..5 = the other compiled
- * shapes <threads, events per thread, blocks per SM>: <192,5,4>, <320,5,2>, <64,5,8>, <256,7,2>, <160,5,5>. */
-void argus_set_synthesize_mode(int mode);
-void argus_set_tile_variant(int variant);
 
 #ifdef __cplusplus
 }

@@ -8,7 +8,7 @@
 namespace {
 std::atomic<unsigned long long> g_launches{0};
 std::atomic<int> g_prof_on{0};
-std::atomic<int> g_prof_suppress{0};
+thread_local int g_prof_suppress = 0;  // per host thread: a call that must not create events does not silence others
 std::mutex g_prof_mu;
 struct ProfPair { cudaEvent_t a, b; };
 std::vector<ProfPair> g_prof[ARGUS_PROF_SLOTS];
@@ -17,7 +17,7 @@ std::vector<ProfPair> g_prof[ARGUS_PROF_SLOTS];
 void argus_count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 void argus_prof_mark(int slot, cudaStream_t stream, int end) {
-  if (!g_prof_on.load(std::memory_order_relaxed) || g_prof_suppress.load(std::memory_order_relaxed) > 0 || slot < 0 ||
+  if (!g_prof_on.load(std::memory_order_relaxed) || g_prof_suppress > 0 || slot < 0 ||
       slot >= ARGUS_PROF_SLOTS)
     return;
   std::lock_guard<std::mutex> lk(g_prof_mu);
@@ -32,7 +32,7 @@ void argus_prof_mark(int slot, cudaStream_t stream, int end) {
   }
 }
 
-void argus_prof_suppress(int delta) { g_prof_suppress.fetch_add(delta); }
+void argus_prof_suppress(int delta) { g_prof_suppress += delta; }
 
 extern "C" unsigned long long argus_launch_count(void) { return g_launches.load(); }
 

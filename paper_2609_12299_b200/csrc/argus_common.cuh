@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "argus.h"
+#include "argus_testing.h"
 
 typedef unsigned long long u64;
 typedef unsigned int u32;

@@ -13,11 +13,13 @@
 
 #include <string.h>
 
+#include <atomic>
+
 namespace {
 
 constexpr int kScanThreads = 1024;
 constexpr u32 kWordsPerBlock = 1024;  // bitmap words per prefix block (32768 events)
-u32 g_poll_limit = 1u << 19;          // see argus_testing_set_poll_limit
+std::atomic<u32> g_poll_limit{1u << 19};  // see argus_testing_set_poll_limit
 
 // ---------------------------------------------------------------------------------------------
 // Reference-order kernel: one thread walks one stream with its stack in local memory.
@@ -264,6 +266,8 @@ Layout make_layout(uint64_t num_events, uint32_t num_streams, uint64_t ambig_cap
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream);
 bool argus_pair_tiled_usable(const ArgusPairArgs& a);
 
+extern "C" void argus_testing_set_poll_limit(unsigned int polls) { g_poll_limit.store(polls ? polls : 1u << 19); }
+
 extern "C" size_t argus_pair_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint64_t ambig_capacity) {
   return make_layout(num_events, num_streams, ambig_capacity).total;
 }
@@ -301,7 +305,7 @@ int argus_internal_pair(const argus_event_t* events, uint64_t num_events, const 
   a.redo = 0;
   a.queue = (u32*)(ws + L.queue); a.queue_capacity = L.queue_capacity;
   a.records = (ArgusStreamRecord*)(ws + L.records); a.record_capacity = L.record_capacity;
-  a.poll_limit = g_poll_limit;
+  a.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
   a.ring_written = (const u64*)ring_written; a.ring_capacity = ring_capacity;
   if (ring_written && (ring_capacity == 0 || kernel_choice == 1)) return ARGUS_ERR_INVALID_ARG;  // only the tiled kernel reads rings
   // a stream's intervals start at half its first event's position at the latest, so positions stay below num_events / 2 + 1

@@ -22,6 +22,7 @@
 #include "argus_internal.cuh"
 #include "argus_pair_common.cuh"
 
+#include <atomic>
 #include <mutex>
 
 namespace {
@@ -593,7 +594,7 @@ int launch_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   return ARGUS_OK;
 }
 
-int g_variant = 0;
+std::atomic<int> g_variant{0};
 
 }  // namespace
 
@@ -601,11 +602,11 @@ bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0;
 
 // Tile shape used by the tiled kernel: 0 = the default; 1..3 select the other compiled shapes
 // <threads, events per thread, CTAs per SM> (test aid: tiles end at other places; results do not depend on it).
-extern "C" void argus_set_tile_variant(int v) { g_variant = v; }
+extern "C" void argus_set_tile_variant(int v) { g_variant.store(v); }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
   if (a.ring_written) return launch_tiled<128, 5, 6, true>(a, stream);  // ring container: one shape
-  switch (g_variant) {
+  switch (g_variant.load(std::memory_order_relaxed)) {
     case 1: return launch_tiled<192, 5, 4, false>(a, stream);
     case 2: return launch_tiled<64, 5, 8, false>(a, stream);
     case 3: return launch_tiled<256, 7, 2, false>(a, stream);

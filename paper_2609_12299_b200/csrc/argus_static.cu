@@ -6,6 +6,8 @@
 // cudaFree or an allocating library routine.
 #include "argus_internal.cuh"
 
+#include <atomic>
+
 
 namespace {
 
@@ -15,7 +17,13 @@ constexpr size_t kStaticScratchBytes = 960 * 1024;
 static __device__ __align__(256) unsigned char g_pair_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_ptr[kMaxDevices];  // device address of g_pair_scratch, looked up once per device
+std::atomic<void*> g_scratch_ptr[kMaxDevices];  // device address of g_pair_scratch, looked up once per device
+                                                // (two threads that race here both find the same address)
+
+// The documented maxima fit the array together (the run-time check below is then never the one that refuses them).
+static_assert((size_t)ARGUS_STATIC_MAX_EVENTS / 8 * 2 + (size_t)ARGUS_STATIC_MAX_AMBIG * 8 +
+                  (size_t)ARGUS_STATIC_MAX_STREAMS * 12 + 64 * 1024 <= kStaticScratchBytes,
+              "bitmap + word prefixes + ambiguity notes + per-stream counters and order + queue, records and control block");
 
 }  // namespace
 
@@ -32,19 +40,19 @@ extern "C" int argus_pair_intervals_static(const argus_event_t* events, uint64_t
   int dev = 0;
   ARGUS_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return ARGUS_ERR_INVALID_ARG;
-  if (!g_scratch_ptr[dev]) {
+  void* scratch = g_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
     // The array's name is only a host-side handle; kernels need its address on the current device.
-    void* p = nullptr;
-    ARGUS_CUDA_TRY(cudaGetSymbolAddress(&p, g_pair_scratch));
-    if (!p) return ARGUS_ERR_CUDA;
-    g_scratch_ptr[dev] = p;
+    ARGUS_CUDA_TRY(cudaGetSymbolAddress(&scratch, g_pair_scratch));
+    if (!scratch) return ARGUS_ERR_CUDA;
+    g_scratch_ptr[dev].store(scratch, std::memory_order_release);
   }
   // The pipeline clears its control block, counters and bitmap itself at the start of every call.
-  // Kernel-time profiling would create CUDA events (an allocation), so it stays off in here.
+  // Kernel-time profiling would create CUDA events (an allocation), so it stays off in here (for this thread only).
   argus_prof_suppress(+1);
   const int rc = argus_internal_pair(events, num_events, stream_offsets, num_streams, num_regions, intervals,
                                      interval_capacity, interval_offsets, ambig, ambig_capacity, ambig_offsets, status,
-                                     g_scratch_ptr[dev], kStaticScratchBytes, cuda_stream, 0, true);
+                                     scratch, kStaticScratchBytes, cuda_stream, 0, true);
   argus_prof_suppress(-1);
   return rc;
 }

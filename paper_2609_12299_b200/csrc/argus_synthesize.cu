@@ -7,9 +7,11 @@
 // same pipeline on a ring container.
 #include "argus_internal.cuh"
 
+#include <atomic>
+
 namespace {
 
-int g_synth_mode = -1;  // -1 = automatic
+std::atomic<int> g_synth_mode_knob{-1};  // -1 = automatic
 
 struct SynLayout {
   size_t pair, pair_bytes, agg, agg_bytes, list_count, list_seg, list_spans, ov, ov_bytes, digest, total;
@@ -50,7 +52,7 @@ SynLayout syn_layout(uint64_t num_events, uint32_t num_streams, uint32_t num_reg
 
 // Where argus_synthesize aggregates and selects overlap spans: -1 automatic, 1 in one pass over the intervals'
 // digests, 2 the plain calls, 3 in one pass over the interval records (test aid; results are identical).
-extern "C" void argus_set_synthesize_mode(int mode) { g_synth_mode = mode; }
+extern "C" void argus_set_synthesize_mode(int mode) { g_synth_mode_knob.store(mode); }
 
 extern "C" size_t argus_synthesize_workspace_bytes(uint64_t num_events, uint32_t num_streams, uint32_t num_regions,
                                                    uint64_t ambig_capacity, uint32_t num_pairs, uint32_t num_sms,
@@ -76,6 +78,7 @@ static int synthesize_impl(const argus_event_t* events, uint64_t num_events, con
   if (num_pairs && (!pairs || !overlap_out)) return ARGUS_ERR_INVALID_ARG;
   const SynLayout L = syn_layout(num_events, num_streams, num_regions, ambig_capacity, num_pairs, num_sms, max_overlap_spans);
   if (workspace_bytes < L.total) return ARGUS_ERR_WORKSPACE;
+  const int g_synth_mode = g_synth_mode_knob.load(std::memory_order_relaxed);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   char* ws = (char*)workspace;
   const bool want_agg = warp_tab || cta_tab || sm_tab || kernel_tab;

@@ -652,6 +652,27 @@ def test_long_streams_walked_in_chunks():
     assert int(pr.last_status["ambig_required"]) > 0
 
 
+def test_bounded_wait_for_a_hand_over_runs_out_and_the_call_returns():
+    """A block of the tiled kernel that has no stream left polls for hand-overs of long streams, and gives up after a
+    bounded number of polls. With the limit set to almost nothing the wait runs out while the long stream's block is
+    still busy: the call returns, the status says ARGUS_ERR_TIMEOUT, nothing hangs, and with the default limit the same
+    buffers give the oracle's result."""
+    lib = argus.load_library()
+    rng = np.random.default_rng(36)
+    evs = [random_wellformed(rng, 600_000, 6, max_height=8), random_wellformed(rng, 40, 6, max_height=3)]
+    offs = np.cumsum([0] + [len(e) for e in evs]).astype(np.uint64)
+    ev = np.concatenate(evs)
+    d_ev, d_off = to_dev(ev, offs)
+    lib.argus_testing_set_poll_limit(1)
+    try:
+        pr = argus.argus_pair_intervals(d_ev, d_off, 6, kernel=KERNEL_TILED)
+        st = pr.fetch_status()
+    finally:
+        lib.argus_testing_set_poll_limit(0)
+    assert int(st["code"]) == 8  # ARGUS_ERR_TIMEOUT
+    assert_pair_matches(ev, offs, 6, KERNEL_TILED)
+
+
 @pytest.mark.parametrize("idx,ctas,iters", [(3, 1, 40), (4, 2, 3000)])
 def test_synthesize_long_streams(idx, ctas, iters):
     """The one-call pipeline on streams of 80 K to 110 K events (several hand-overs each), bit for bit."""

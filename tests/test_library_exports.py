@@ -8,8 +8,8 @@ import paper_2609_12299_b200 as argus
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "argus.h")).read()
+def _declared_functions(header="argus.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(argus_[a-z_]+)\s*\(", text)))
 
@@ -22,6 +22,40 @@ def test_header_symbols_are_exported():
     lib = ctypes.CDLL(argus.library_path())
     for n in names:
         assert hasattr(lib, n), f"{n} is declared in argus.h but not exported"
+    # the product header holds no test or tuning aid; those live in argus_testing.h and are exported too
+    aids = _declared_functions("argus_testing.h")
+    assert {"argus_pair_intervals_ex", "argus_set_tile_variant", "argus_set_synthesize_mode", "argus_profile_enable",
+            "argus_profile_read", "argus_launch_count", "argus_testing_set_poll_limit"} <= set(aids)
+    assert not (set(aids) & set(names))
+    for n in aids:
+        assert hasattr(lib, n), f"{n} is declared in argus_testing.h but not exported"
+
+
+def test_first_calls_from_two_threads():
+    """Two host threads make their first calls at the same time (argument validation only, no GPU): the per-device
+    caches and the switches are safe to touch concurrently."""
+    import threading
+    lib = argus.load_library()
+    rcs = []
+
+    def work():
+        for _ in range(200):
+            rcs.append(lib.argus_pair_intervals(None, 0, None, 0, 1, None, 0, None, None, 0, None, None, None, 0, None))
+            lib.argus_set_tile_variant(0)
+            lib.argus_testing_set_poll_limit(0)
+            rcs.append(lib.argus_pair_intervals_static(None, (1 << 20) + 1, None, 0, 1, None, 0, None, None, 0, None, None, None))
+    ts = [threading.Thread(target=work) for _ in range(2)]
+    [t.start() for t in ts]
+    [t.join() for t in ts]
+    assert set(rcs) == {1, 9}
+
+
+def test_static_entry_accepts_its_documented_maxima():
+    """2^20 events, 4,096 streams and 2^16 ambiguity records together fit the built-in scratch: the call gets past
+    its size checks (and then stops at the null pointers, or at the missing device on a CPU machine)."""
+    lib = argus.load_library()
+    rc = lib.argus_pair_intervals_static(None, 1 << 20, None, 4096, 1, None, 0, None, None, 1 << 16, None, None, None)
+    assert rc in (1, 3)
 
 
 def test_host_only_calls():
@@ -59,7 +93,7 @@ def test_header_is_plain_c():
     with tempfile.TemporaryDirectory() as d:
         src = os.path.join(d, "t.c")
         with open(src, "w") as f:
-            f.write('#include "argus.h"\nint main(void) { return sizeof(argus_agg_t) == 576 && sizeof(argus_interval_t) == 48 ? 0 : 1; }\n')
+            f.write('#include "argus.h"\n#include "argus_testing.h"\nint main(void) { return sizeof(argus_agg_t) == 576 && sizeof(argus_interval_t) == 48 ? 0 : 1; }\n')
         exe = os.path.join(d, "t")
         subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), src, "-o", exe])
         assert subprocess.call([exe]) == 0

@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2609_12299_b200 as argus
 from paper_2609_12299_b200 import tracegen as tg
 
@@ -28,6 +29,11 @@ def _run_both(spec):
     assert got.intervals_numpy().tobytes() == ref.intervals_numpy().tobytes()
     assert got.ambig_numpy().tobytes() == ref.ambig_numpy().tobytes()
     assert st_got.tobytes() == st_ref.tobytes()
+    # and directly against the oracle
+    rc, o_iv, o_ioffs, o_am, o_aoffs, _ = oracle.pair(ev, offs, spec.num_regions)
+    assert rc == 0
+    assert got.intervals_numpy().tobytes() == o_iv.tobytes() and got.ambig_numpy().tobytes() == o_am.tobytes()
+    assert np.array_equal(got.interval_offsets.cpu().numpy().view(np.uint64), o_ioffs)
     return len(ev), len(ref.ambig_numpy())
 
 
@@ -57,3 +63,35 @@ def test_static_scratch_entry_rejects_oversized_inputs():
     rc = lib.argus_pair_intervals_static(ev.data_ptr(), 1, off.data_ptr(), 1, 1, None, 0, out_off.data_ptr(), None,
                                          (1 << 16) + 1, out_off.data_ptr(), st.data_ptr(), None)
     assert rc == 9
+
+
+def test_static_scratch_entry_allocates_nothing():
+    """What the entry point is for: with the outputs allocated beforehand and one call behind it (the first call on a
+    device looks up the scratch array's address), a call through the C function leaves the device's free memory and
+    torch's allocator exactly as they were."""
+    spec = tg.config(1).scaled(num_ctas=3, iters=50)
+    ev, offs = tg.generate_host(spec)
+    d_ev = torch.from_numpy(ev.view(np.uint8).reshape(-1).copy()).to(DEV)
+    d_off = torch.from_numpy(offs.view(np.int64).copy()).to(DEV)
+    n, S = len(ev), spec.num_streams
+    iv = torch.empty(n // 2 * 48, dtype=torch.uint8, device=DEV)
+    am = torch.empty(4096 * 32, dtype=torch.uint8, device=DEV)
+    ioffs = torch.empty(S + 1, dtype=torch.int64, device=DEV)
+    aoffs = torch.empty(S + 1, dtype=torch.int64, device=DEV)
+    st = torch.empty(64, dtype=torch.uint8, device=DEV)
+    lib = argus.load_library()
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        return lib.argus_pair_intervals_static(d_ev.data_ptr(), n, d_off.data_ptr(), S, spec.num_regions, iv.data_ptr(), n // 2,
+                                               ioffs.data_ptr(), am.data_ptr(), 4096, aoffs.data_ptr(), st.data_ptr(), stream)
+    assert call() == 0
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    stats0 = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+    assert call() == 0
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == stats0
+    rc, o_iv, o_ioffs, _, _, _ = oracle.pair(ev, offs, spec.num_regions)
+    assert iv.cpu().numpy()[: len(o_iv) * 48].tobytes() == o_iv.tobytes()
