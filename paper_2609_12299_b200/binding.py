@@ -398,25 +398,6 @@ def argus_overlap_scoped(intervals: torch.Tensor, max_intervals: int, interval_o
     return out, status
 
 
-def encode_map_events(kind: np.ndarray, ident: np.ndarray, count: np.ndarray, exec_region: int) -> np.ndarray:
-    """Mapping-run records (kind 0 begin / 1 end of region `ident`, 2 = PC index `ident` executed `count`
-    times) in the marker encoding argus.h documents: an exec record becomes a begin/end pair of region
-    `exec_region` with ctx = PC index and ts 0 / count. Returns (events, source index of each event).
-    Argument marshalling only."""
-    kind = np.asarray(kind)
-    is_exec = kind == 2
-    reps = np.where(is_exec, 2, 1)
-    src = np.repeat(np.arange(len(kind)), reps)
-    second = np.zeros(len(src), dtype=bool)
-    second[np.cumsum(reps)[is_exec] - 1] = True           # the end half of every exec pair
-    ev = np.zeros(len(src), dtype=EVENT_DTYPE)
-    ex = is_exec[src]
-    ev["tag"] = np.where(ex, (exec_region << 1) | second, (np.asarray(ident)[src] << 1) | (kind[src] & 1)).astype(np.uint32)
-    ev["ctx"] = np.where(ex, np.asarray(ident)[src], 0).astype(np.uint32)
-    ev["ts"] = np.where(second, np.asarray(count)[src], 0).astype(np.uint64)
-    return ev, src
-
-
 def argus_map_pc_counts(intervals: torch.Tensor, interval_offsets: torch.Tensor, exec_region: int, num_pcs: int):
     """Returns (counts int64 tensor [(exec_region + 1), num_pcs] (bit pattern of u64), status uint8 [64])."""
     lib = load_library()
@@ -635,43 +616,3 @@ def argus_synthesize(events: torch.Tensor, stream_offsets: torch.Tensor, num_reg
     if rc != 0:
         raise ArgusError(rc, "argus_synthesize")
     return out
-
-
-def pair_aggregate_host(events: np.ndarray, stream_offsets: np.ndarray, num_regions: int, warps_per_cta: int,
-                        cta_sm: np.ndarray, num_sms: int, device="cuda:0", state: dict | None = None):
-    """End-to-end call with HOST buffers: copies the events (and offsets) to the device, runs
-    argus_pair_intervals + argus_aggregate, and copies the kernel-, SM- and CTA-scope tables, the
-    interval offsets and the status block back. `state` (a dict the caller keeps) caches pinned staging
-    and device buffers between calls. Returns (tables dict of numpy arrays, interval_offsets, status)."""
-    dev = torch.device(device)
-    st = state if state is not None else {}
-    n = len(events)
-    S = len(stream_offsets) - 1
-    key = (n, S, num_regions)
-    if st.get("key") != key:
-        st.clear()
-        st["key"] = key
-        st["pin_ev"] = torch.empty(max(n, 1) * 16, dtype=torch.uint8).pin_memory()
-        st["pin_off"] = torch.empty(S + 1, dtype=torch.int64).pin_memory()
-        st["dev_ev"] = torch.empty(max(n, 1) * 16, dtype=torch.uint8, device=dev)
-        st["dev_off"] = torch.empty(S + 1, dtype=torch.int64, device=dev)
-        st["cta_sm"] = torch.from_numpy(np.ascontiguousarray(cta_sm, dtype=np.uint32).view(np.int32)).to(dev)
-        st["pair"] = None
-        st["agg"] = None
-    ev_bytes = np.ascontiguousarray(events).view(np.uint8).reshape(-1)
-    if ev_bytes.ctypes.data != st["pin_ev"].data_ptr():
-        st["pin_ev"][: n * 16].numpy()[:] = ev_bytes
-    st["pin_off"].numpy()[:] = np.ascontiguousarray(stream_offsets, dtype=np.uint64).view(np.int64)
-    with torch.cuda.device(dev):
-        st["dev_ev"][: n * 16].copy_(st["pin_ev"][: n * 16], non_blocking=True)
-        st["dev_off"].copy_(st["pin_off"], non_blocking=True)
-        st["pair"] = argus_pair_intervals(st["dev_ev"][: n * 16], st["dev_off"], num_regions, out=st["pair"],
-                                          ambig_capacity=max(n // 64, 4096) if st["pair"] is None else None)
-        p = st["pair"]
-        st["agg"] = argus_aggregate(p.intervals, p.interval_offsets, p.ambig, p.ambig_offsets, warps_per_cta,
-                                    st["cta_sm"], num_sms, num_regions, out=st["agg"])
-        a = st["agg"]
-        tables = {lv: a.table_numpy(lv) for lv in ("kernel", "sm", "cta")}
-        ioffs = p.interval_offsets.cpu().numpy().view(np.uint64)
-        status = p.fetch_status()
-    return tables, ioffs, status

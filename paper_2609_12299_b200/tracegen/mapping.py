@@ -60,3 +60,22 @@ def decode_mapping_trace(events: np.ndarray, num_regions: int):
     count = np.where(ex[idx], events["ts"][nxt], 0).astype(np.uint64)
     removed_before = np.cumsum(~keep)
     return kind, ident, count, removed_before
+
+
+def encode_map_events(kind: np.ndarray, ident: np.ndarray, count: np.ndarray, exec_region: int) -> np.ndarray:
+    """Mapping-run records (kind 0 begin / 1 end of region `ident`, 2 = PC index `ident` executed `count`
+    times) in the marker encoding argus.h documents: an exec record becomes a begin/end pair of region
+    `exec_region` with ctx = PC index and ts 0 / count. Returns (events, source index of each event).
+    Input preparation: the library itself only ever sees marker records."""
+    kind = np.asarray(kind)
+    is_exec = kind == 2
+    reps = np.where(is_exec, 2, 1)
+    src = np.repeat(np.arange(len(kind)), reps)
+    second = np.zeros(len(src), dtype=bool)
+    second[np.cumsum(reps)[is_exec] - 1] = True           # the end half of every exec pair
+    ev = np.zeros(len(src), dtype=np.dtype([("ts", "<u8"), ("tag", "<u4"), ("ctx", "<u4")]))
+    ex = is_exec[src]
+    ev["tag"] = np.where(ex, (exec_region << 1) | second, (np.asarray(ident)[src] << 1) | (kind[src] & 1)).astype(np.uint32)
+    ev["ctx"] = np.where(ex, np.asarray(ident)[src], 0).astype(np.uint32)
+    ev["ts"] = np.where(second, np.asarray(count)[src], 0).astype(np.uint64)
+    return ev, src

@@ -7,6 +7,7 @@ import torch
 
 import oracle
 import paper_2609_12299_b200 as argus
+from paper_2609_12299_b200.tracegen.mapping import encode_map_events
 from test_oracle_map_pins import load_map_example, random_map_trace
 
 pytestmark = pytest.mark.gpu
@@ -14,7 +15,7 @@ DEV = "cuda:0"
 
 
 def gpu_counts(streams, R, P):
-    enc = [argus.encode_map_events(s["kind"], s["id"], s["count"], R)[0] for s in streams]
+    enc = [encode_map_events(s["kind"], s["id"], s["count"], R)[0] for s in streams]
     offs = np.cumsum([0] + [len(e) for e in enc]).astype(np.uint64)
     ev = np.concatenate(enc) if enc else np.zeros(0, argus.EVENT_DTYPE)
     d_ev = torch.from_numpy(ev.view(np.uint8).reshape(-1).copy()).to(DEV)
@@ -79,7 +80,7 @@ def test_attribution_shapes_and_extremes():
 
 def test_pc_index_out_of_range_is_reported():
     ev = np.array([(0, 0, 0), (2, 9, 1), (1, 0, 0)], dtype=oracle.MAP_EVENT)
-    enc = argus.encode_map_events(ev["kind"], ev["id"], ev["count"], 1)[0]
+    enc = encode_map_events(ev["kind"], ev["id"], ev["count"], 1)[0]
     d_ev = torch.from_numpy(enc.view(np.uint8).reshape(-1).copy()).to(DEV)
     d_off = torch.from_numpy(np.array([0, len(enc)], np.int64)).to(DEV)
     pr = argus.argus_pair_intervals(d_ev, d_off, 2)
