@@ -310,10 +310,11 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
 #pragma unroll
         for (int k = 0; k < E; ++k) {
           const int e = w0 + tid * E + k;
-          tags[k] = e < wend ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;  // all ones = no event
+          const bool valid = e < wend;
+          tags[k] = valid ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;
           if (!(tags[k] & 1u)) accb[e] = 0;  // child time is gathered at begins only
           (&sm.bm[0][0])[tid * E + k] = 0;  // kLevelWindow * NWORDS == T words
-          if (tags[k] != 0xffffffffu) { if (tags[k] & 1u) ++ne; else ++nb; }
+          if (valid) { if (tags[k] & 1u) ++ne; else ++nb; }
         }
         if (tid < kLevelWindow) sm.summ[tid] = 0;
         if (tid < ch) accb[cbase + tid] = sm.cchild[cpar][tid];  // a cut window may have added to these: start clean
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
 #pragma unroll
           for (int k = 0; k < E; ++k) {  // flat, so that begins and ends of a warp are handled by predication, not by two passes
             const int e = w0 + tid * E + k;
-            const bool valid = tags[k] != 0xffffffffu;
+            const bool valid = e < wend;  // (not "tag != all ones": that is a marker too, with a region id out of range)
             const bool is_e = valid && (tags[k] & 1u), is_b = valid && !(tags[k] & 1u);
             const int he = h - 1;            // level of the frame an end closes
             const int l = h - lbase;         // level of the frame a begin opens, inside the window

@@ -652,6 +652,21 @@ def test_long_streams_walked_in_chunks():
     assert int(pr.last_status["ambig_required"]) > 0
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_marker_with_all_ones_tag_is_a_bad_region(kernel):
+    """A tag of all ones is an end marker of region 2^31 - 1, not an absent event: reported like any region id out of range."""
+    rng = np.random.default_rng(37)
+    ev = random_wellformed(rng, 900, 5, max_height=4)
+    ev["tag"][1234] = 0xFFFFFFFF
+    offs = np.array([0, len(ev)], np.uint64)
+    rc, *_, o_st = oracle.pair(ev, offs, 5)
+    d_ev, d_off = to_dev(ev, offs)
+    pr = argus.argus_pair_intervals(d_ev, d_off, 5, kernel=kernel)
+    st = pr.fetch_status()
+    assert int(o_st["code"]) == 6 and int(st["code"]) == 6
+    assert (int(st["bad_stream"]), int(st["bad_event"])) == (int(o_st["bad_stream"]), int(o_st["bad_event"])) == (0, 1234)
+
+
 def test_bounded_wait_for_a_hand_over_runs_out_and_the_call_returns():
     """A block of the tiled kernel that has no stream left polls for hand-overs of long streams, and gives up after a
     bounded number of polls. With the limit set to almost nothing the wait runs out while the long stream's block is
