@@ -42,7 +42,7 @@ int argus_profile_read(double* ms_total /*host [4]*/, unsigned long long* launch
  * 1 in one pass over the intervals' digests, 2 the three plain operations, 3 in one pass over the interval
  * records. A mode the inputs do not allow falls back to the automatic choice.
  * argus_set_tile_variant: shape of the tiled pairing kernel, 0 = the default <128 threads, 5 events per
- * thread, 6 blocks per SM>, 1..3 = <192,5,4>, <64,5,8>, <256,7,2> (tiles end at other places).
+ * thread, 7 blocks per SM>, 1..3 = <192,5,4>, <64,5,8>, <256,7,2> (tiles end at other places).
  * argus_testing_set_poll_limit: polls after which a block of the tiled pairing kernel that waits for a
  * hand-over gives up with ARGUS_ERR_TIMEOUT (default 2^19, about a second; 0 restores the default). A test
  * sets it to a few polls to see the bounded wait run out and the call return with the status set. */

@@ -24,6 +24,7 @@
 
 #include <atomic>
 #include <mutex>
+#include <type_traits>
 
 namespace {
 
@@ -59,7 +60,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
   return false;
 }
 
-constexpr int kLevelWindow = 32;  // begins of a tile may sit at levels [lbase, lbase + 32)
+constexpr int kLevelWindow = 16;  // begins of a tile may sit at levels [lbase, lbase + 16)
 constexpr int kCar = 80;          // slots of a carried-frame block: 64 frames, 1 sink for "no parent", padding
 constexpr int kSink = 64;         // index of the sink slot inside a carried-frame block
 constexpr int kBadRef = 0x3fff;   // reference that marks a window as not well nested
@@ -111,9 +112,12 @@ struct TileSmem {
   static constexpr int NWORDS = T / 32;                 // bitmap words per level
   static constexpr int MAXI = T / 2 + ARGUS_MAX_DEPTH;  // intervals a well-nested tile can emit
   static constexpr int NI = (MAXI + NT - 1) / NT;       // intervals per thread in the emission phases
+  static constexpr int kDescShift = T <= 1024 ? 10 : 16;
+  using desc_t = typename std::conditional<(T <= 1024), unsigned short, u32>::type;
   uint4 evall[2 * T + 2 * kCar];
-  u64 accall[T + 4 * kCar];        // child time per frame, same index space shifted by 2 kCar
-  u32 desc[MAXI];                  // per end, in end order: event index | level << 16
+  u32 accall[T + 4 * kCar];        // child time each frame gathers in the current window (32 bits: an overflow cuts the
+                                   // window), same index space shifted by 2 kCar
+  desc_t desc[MAXI];               // per end, in end order: event index | level << kDescShift
   union {
     u32 bm[kLevelWindow][NWORDS];    // per level: bit e set = event e of the tile is a begin at that level
     ArgusFrame fstk[ARGUS_MAX_DEPTH];  // stack in the layout the sequential path uses (no bitmap is live while it runs)
@@ -284,7 +288,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
       uint4* const ev0 = sm.evall;
       uint4* const ev1 = sm.evall + T + 2 * kCar;
       const uint4* evb = b ? ev1 : ev0;                  // evb[ref] for every reference of this tile
-      u64* accb = sm.accall + 2 * kCar;                  // accb[ref], ref in [-2 kCar, T + 2 kCar)
+      u32* accb = sm.accall + 2 * kCar;                  // accb[ref], ref in [-2 kCar, T + 2 kCar)
       const int carlo = b ? -2 * kCar : T;               // reference of slot 0 of carried block 0, seen from this buffer
       if (tid == 0 && ti + 1 < ti_end) {  // prefetch the next tile into the other buffer
         const u32 nstart = tile_start + T;
@@ -313,11 +317,11 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           const bool valid = e < wend;
           tags[k] = valid ? reinterpret_cast<const u32*>(evb + e)[2] : 0xffffffffu;
           if (!(tags[k] & 1u)) accb[e] = 0;  // child time is gathered at begins only
-          (&sm.bm[0][0])[tid * E + k] = 0;  // kLevelWindow * NWORDS == T words
           if (valid) { if (tags[k] & 1u) ++ne; else ++nb; }
         }
+        for (int i = tid; i < kLevelWindow * NWORDS; i += NT) (&sm.bm[0][0])[i] = 0;
         if (tid < kLevelWindow) sm.summ[tid] = 0;
-        if (tid < ch) accb[cbase + tid] = sm.cchild[cpar][tid];  // a cut window may have added to these: start clean
+        if (tid < ch) accb[cbase + tid] = 0;  // what this window adds to the carried frames (a cut window starts clean again)
         if (tid == 0) { sm.failed = 0; accb[cbase + kSink] = 0; }
         // block prefix sum of (begins, ends), 16 bits each: one barrier
         const u32 mine_cnt = (u32)nb | ((u32)ne << 16);
@@ -340,7 +344,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
         const int win_nb = (int)(tot & 0xffffu);
         const int win_ne = (int)(tot >> 16) < MAXI ? (int)(tot >> 16) : MAXI;  // more ends than that means a violation earlier
         const int h0 = ch + (int)(ex & 0xffffu) - (int)(ex >> 16);
-        const int lbase = ch > 16 ? ch - 16 : 0;
+        const int lbase = ch > kLevelWindow / 2 ? ch - kLevelWindow / 2 : 0;
         {
           int h = h0, rank = (int)(ex >> 16);
           bool seen = false;  // this thread already reported a violation: later markers only keep `desc` complete
@@ -354,7 +358,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             // the parallel rules: known region id, height never negative, at most 64 frames, begins inside the level window
             const bool viol = (valid && (tags[k] >> 1) >= a.num_regions) || (is_e && he < 0) ||
                               (is_b && ((unsigned)l >= (unsigned)kLevelWindow || h >= ARGUS_MAX_DEPTH));
-            if (is_e && rank < MAXI) sm.desc[rank] = (u32)e | ((u32)(he & 0xff) << 16);
+            if (is_e && rank < MAXI) sm.desc[rank] = (typename SM::desc_t)((u32)e | ((u32)(he & 0x3f) << SM::kDescShift));
             if (is_b && !viol && !seen) {
               atomicOr(&sm.bm[l][e >> 5], 1u << (e & 31));
               atomicOr(reinterpret_cast<u32*>(&sm.summ[l]) + (e >> 10), 1u << ((e >> 5) & 31));
@@ -376,7 +380,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             refs[i] = 0;
             if (rk < win_ne) {
               const u32 d = sm.desc[rk];
-              const int e = (int)(d & 0xffffu), L = (int)(d >> 16);
+              const int e = (int)(d & ((1u << SM::kDescShift) - 1u)), L = (int)(d >> SM::kDescShift);
               if (e >= first_bad) continue;
               const uint4 ee = evb[e];  // needed after the lookups; asked for now, so that it arrives meanwhile
               // in the tile, or opened before this window (then so was its parent); selects, not branches
@@ -391,13 +395,13 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
               const uint4 pe = evb[partner];
               if ((pe.z >> 1) != (ee.z >> 1)) { atomicMin(&sm.badpos[bp], e); continue; }
               const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
-              if (ts > bts) {  // 64-bit add as two native 32-bit shared atomics; each carry is propagated exactly once
+              if (ts > bts) {
+                // the parent gathers what this window adds to its child time in 32 bits; an interval or a sum of 2^32 ticks
+                // cuts the window here, and the sequential machine (64-bit throughout) takes this marker
                 const u64 dlt = ts - bts;
-                u32* p = reinterpret_cast<u32*>(&accb[parent]);
-                const u32 lo32 = (u32)dlt, hi32 = (u32)(dlt >> 32);
-                const u32 old = atomicAdd(p, lo32);
-                if (hi32) atomicAdd(p + 1, hi32);
-                if (old + lo32 < old) atomicAdd(p + 1, 1u);
+                const u32 lo32 = (u32)dlt;
+                const u32 old = atomicAdd(&accb[parent], lo32);
+                if ((dlt >> 32) || old + lo32 < old) { atomicMin(&sm.badpos[bp], e); continue; }
               }
               refs[i] = ((u32)partner & 0xffffu) | ((u32)parent << 16);
             }
@@ -424,16 +428,16 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             if (rk < win_ne) {
               const u32 d = sm.desc[rk];
               const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
-              const uint4 ee = evb[d & 0xffffu];
+              const uint4 ee = evb[d & ((1u << SM::kDescShift) - 1u)];
               const uint4 pe = evb[partner];
               const u64 ts = (u64)ee.x | ((u64)ee.y << 32), bts = (u64)pe.x | ((u64)pe.y << 32);
-              const u64 child = accb[partner];
+              const bool carried = (u32)partner >= (u32)T;
+              const u64 child = (carried ? sm.cchild[cpar][partner - cbase] : 0ull) + accb[partner];
               u32 flags = 0;
               u64 incl = 0, excl = 0;
               if (ee.w != pe.w) { flags |= ARGUS_FLAG_CTX_MISMATCH; ++tot_ctx; }
               if (ts < bts) { flags |= ARGUS_FLAG_TIME_REVERSED; ++tot_rev; } else { incl = ts - bts; }
               if (child > incl) { flags |= ARGUS_FLAG_CHILD_CLAMPED; ++tot_clamp; } else { excl = incl - child; }
-              const bool carried = (u32)partner >= (u32)T;
               const u32 bidx = carried ? sm.cidx[cpar][partner - cbase] : tile_start + (u32)partner;
               const u32 preg = parent == cbase + kSink ? ARGUS_NONE : (reinterpret_cast<const u32*>(evb + parent)[2] >> 1);
               const u64 pos = pos0 + (u64)rk;
@@ -441,7 +445,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
                 uint4* q = reinterpret_cast<uint4*>(a.intervals + pos);
                 q[0] = make_uint4(pe.x, pe.y, (u32)incl, (u32)(incl >> 32));
                 q[1] = make_uint4((u32)excl, (u32)(excl >> 32), pe.z >> 1, pe.w);
-                q[2] = make_uint4(s, preg, bidx, (d >> 16) | (flags << 16));
+                q[2] = make_uint4(s, preg, bidx, (d >> SM::kDescShift) | (flags << 16));
                 if (a.digest) a.digest[pos] = argus_digest_pack(pe.z >> 1, incl, excl, flags);
               } else if (!a.redo) {
                 a.ctl->spec_overflow = 1;
@@ -453,7 +457,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
             const int e = tile_latest_begin<NT, E>(sm, tid, lbase, T);
             const int from = e >= 0 ? e : cbase + tid;
             car_next[tid] = evb[from];
-            sm.cchild[cpar ^ 1][tid] = accb[from];
+            sm.cchild[cpar ^ 1][tid] = (e >= 0 ? 0ull : sm.cchild[cpar][tid]) + accb[from];
             sm.cidx[cpar ^ 1][tid] = e >= 0 ? tile_start + (u32)e : sm.cidx[cpar][tid];
           }
           small_streak = (wend - w0 < 32) ? small_streak + 1 : 0;
@@ -606,11 +610,11 @@ bool argus_pair_tiled_usable(const ArgusPairArgs& a) { return a.num_streams > 0;
 extern "C" void argus_set_tile_variant(int v) { g_variant.store(v); }
 
 int argus_launch_pair_tiled(const ArgusPairArgs& a, cudaStream_t stream) {
-  if (a.ring_written) return launch_tiled<128, 5, 6, true>(a, stream);  // ring container: one shape
+  if (a.ring_written) return launch_tiled<128, 5, 7, true>(a, stream);  // ring container: one shape
   switch (g_variant.load(std::memory_order_relaxed)) {
     case 1: return launch_tiled<192, 5, 4, false>(a, stream);
     case 2: return launch_tiled<64, 5, 8, false>(a, stream);
     case 3: return launch_tiled<256, 7, 2, false>(a, stream);
-    default: return launch_tiled<128, 5, 6, false>(a, stream);  // six CTAs of 128 threads per SM
+    default: return launch_tiled<128, 5, 7, false>(a, stream);  // seven CTAs of 128 threads per SM
   }
 }
