@@ -667,6 +667,28 @@ def test_marker_with_all_ones_tag_is_a_bad_region(kernel):
     assert (int(st["bad_stream"]), int(st["bad_event"])) == (int(o_st["bad_stream"]), int(o_st["bad_event"])) == (0, 1234)
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_child_time_beyond_32_bits_inside_a_tile(kernel):
+    """The tiled kernel gathers what a window adds to a frame's child time in 32 bits and hands anything larger to
+    the sequential machine: children that add up to more than 2^32 ticks under one parent, a single interval longer
+    than 2^32 ticks, both inside one tile, and a frame carried over many tiles whose child time passes 2^32 on the way."""
+    rows, t = [], 1_700_000_000_000_000_000
+    rows.append((t, "B", 0, 1))
+    for i in range(6):                       # six children of 1.2e9 ticks each: 7.2e9 > 2^32 under region 0
+        rows.append((t + 10, "B", 1, 1)); t += 1_200_000_000; rows.append((t, "E", 1, 1))
+    rows.append((t + 5, "B", 2, 1)); t += 9_000_000_000; rows.append((t, "E", 2, 1))   # one interval of 9e9 ticks
+    rows.append((t + 7, "E", 0, 1))
+    rows.append((t + 8, "B", 3, 2))          # a frame that stays open over several tiles
+    for i in range(4000):
+        rows.append((t + 9, "B", 1, 2)); t += 3_000_000; rows.append((t, "E", 1, 2))  # 4000 x 3e6 = 1.2e10 in all
+    rows.append((t + 1, "E", 3, 2))
+    ev = make_events(rows)
+    offs = np.array([0, len(ev)], np.uint64)
+    pr, _ = assert_pair_matches(ev, offs, 4, kernel)
+    iv = pr.intervals_numpy()
+    assert int(iv["exclusive"][iv["region"] == 3][0]) < int(iv["inclusive"][iv["region"] == 3][0]) - (1 << 33)
+
+
 def test_bounded_wait_for_a_hand_over_runs_out_and_the_call_returns():
     """A block of the tiled kernel that has no stream left polls for hand-overs of long streams, and gives up after a
     bounded number of polls. With the limit set to almost nothing the wait runs out while the long stream's block is
