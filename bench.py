@@ -30,10 +30,10 @@ ALG_BYTES_PER_EVENT = 40.0  # 16 B event read + 48 B interval written per 2 even
 # DRAM traffic of the pairing kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum of one launch)
 # on a small case of the bench workload; the full trace is too large for a multi-pass capture, and the kernel's
 # traffic grows in proportion to the events, so the JSON line scales it to a full launch and says so.
-TRAFFIC_CAPTURE = {"workload": "decode_megakernel", "iters": 8, "events": 38380544, "dram_bytes_read": 614.679808e6,
-                   "dram_bytes_write": 1018.509e6, "kernel": "k_pair_tiled<128,5,6>",
-                   "command": "ncu --set full --clock-control none -k regex:k_pair_tiled -c 1 python bench.py --workload 3 "
-                              "--iters 8 --steps 1 --no-e2e --no-cpu-baseline --no-other"}
+TRAFFIC_CAPTURE = {"workload": "decode_megakernel", "iters": 8, "events": 38380544, "dram_bytes_read": 614.345216e6,
+                   "dram_bytes_write": 1019.052e6, "kernel": "k_pair_tiled<128,5,7>",
+                   "command": "ncu --set full --clock-control none -k regex:k_pair_tiled -s 6 -c 1 python bench.py --workload 3 "
+                              "--iters 8 --steps 1 --warmup 3 --no-e2e --no-cpu-baseline --no-other"}
 
 
 def load_peaks():
