@@ -123,8 +123,8 @@ def argus_set_tile_variant(v: int) -> None:
 
 
 def argus_set_synthesize_mode(mode: int) -> None:
-    """Where argus_synthesize aggregates: -1 automatic, 0 in the pairing kernel, 1 in one pass over the
-    intervals, 2 the plain calls (tuning and test aid; results are identical)."""
+    """Where argus_synthesize aggregates: -1 automatic, 1 in one pass over the intervals' digests, 2 the plain
+    calls, 3 in one pass over the interval records (test aid; results are identical)."""
     load_library().argus_set_synthesize_mode(int(mode))
 
 

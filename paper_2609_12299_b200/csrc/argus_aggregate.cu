@@ -4,7 +4,7 @@
 //                   kernel wrote beside the interval records (not the records) and gathers the stream's row
 //                   in 100-byte shared-memory cells, with per-lane copies of the most frequent regions' cells;
 //   k_agg_streams_compact : the same over the 48-byte records, with an optional scope: that stream's row in
-//                   the compact shared-memory form the fused pairing kernel uses (112 B per region, so
+//                   a compact shared-memory form (112 B per region: sums, min, max, a 16-bin window, so
 //                   several CTAs fit an SM), for up to kAggCompactRegions regions;
 //   k_agg_streams : the same with a full 576 B-per-region copy in shared memory when that fits, else on
 //                   the global row itself. Integer atomics only: the result does not depend on thread order.

@@ -1,12 +1,13 @@
-// argus_fuse.cuh — per-interval hooks that let the pairing kernel feed aggregation and overlap
-// selection while the interval is still in registers (no second read of the interval array).
+// argus_fuse.cuh — what the pairing kernels and the aggregation passes share: the compact shared-memory
+// form of a stream's row of the warp-scope table, the 8-byte digest of an interval, and the arguments of
+// overlap span selection.
 //
-// Aggregation: the CTA that walks a stream keeps that stream's row of the warp-scope table in
-// shared memory in a compact form (per region: sums, min, max, counts and a 16-bin window of the
-// 64-bin log2 histogram; bins outside the window go straight to the global row) and writes it to
-// the global row when the stream ends. All updates are integer atomics, so thread order is irrelevant.
-// Overlap: spans of intervals whose region appears in a (producer, consumer) pair are appended to a
-// global list tagged with their (pair, SM, role) segment; the overlap kernels take it from there.
+// Compact row: per region the sums, min, max, counts and a 16-bin window of the 64-bin log2 histogram
+// (bins outside the window go straight to the global row); the CTA that aggregates a stream keeps the row
+// in shared memory and writes it to the global row when the stream ends. All updates are integer atomics,
+// so thread order is irrelevant.
+// Overlap selection: spans of intervals whose region appears in a (producer, consumer) pair are appended to
+// a global list tagged with their (pair, SM, role) segment; the overlap kernels take it from there.
 #ifndef ARGUS_FUSE_CUH_
 #define ARGUS_FUSE_CUH_
 
@@ -14,8 +15,7 @@
 
 constexpr u32 kAggWindow = 16;          // histogram bins kept in shared memory per region
 constexpr u32 kAggUnset = 0xffffffffu;  // window base not chosen yet
-constexpr u32 kFuseMaxRegions = 256;    // fused aggregation keeps num_regions * 112 bytes in shared memory
-constexpr u32 kFuseMaxPairs = 128;      // fused overlap selection keeps the pair list (8 bytes a pair) in shared memory
+constexpr u32 kFuseMaxPairs = 128;      // span selection keeps the pair list (8 bytes a pair) in shared memory
 constexpr u32 kAggCellWords = 72;       // u64 words of one argus_agg_t
 
 struct ArgusAggCell {  // 112 bytes
@@ -25,7 +25,7 @@ struct ArgusAggCell {  // 112 bytes
 };
 
 struct ArgusFuseArgs {
-  u64* warp_tab;          // [S][R][72], zeroed before the kernel; null = no fused aggregation
+  u64* warp_tab;          // unused by span selection (kept for layout)
   const u32* cta_sm;      // [C]
   u32 warps_per_cta, num_sms;
   const u32* pairs;       // [K][2]
@@ -37,7 +37,7 @@ struct ArgusFuseArgs {
   u64* ov_count;          // spans appended so far (may exceed the capacity)
 };
 
-struct ArgusFuseCtx {     // per CTA, for the stream it is walking
+struct ArgusFuseCtx {     // per CTA, for the stream it is aggregating
   ArgusAggCell* tab;      // shared memory [R]; null = aggregation off
   const u32* pairbits;    // shared memory bitmap over regions: region appears in some pair; null = overlap off
   u64* row;               // global row of this stream in the warp-scope table
@@ -138,29 +138,6 @@ __device__ __forceinline__ void argus_fuse_flush(const ArgusAggCell* tab, u64* r
       }
     }
   }
-}
-
-// Appends the span of a selected interval once per (pair, role) it takes part in.
-__device__ __forceinline__ void argus_fuse_overlap(const ArgusFuseArgs& f, const ArgusFuseCtx& fx, u32 region, u64 t_begin,
-                                                   u64 incl) {
-  if (!incl || !((fx.pairbits[region >> 5] >> (region & 31)) & 1u)) return;
-  for (u32 k = 0; k < f.num_pairs; ++k) {
-#pragma unroll
-    for (u32 role = 0; role < 2; ++role) {
-      if (f.pairs[2 * k + role] != region) continue;
-      const u64 slot = atomicAdd(f.ov_count, 1ull);
-      if (slot < f.ov_capacity) {
-        f.ov_spans[slot] = make_ulonglong2(t_begin, t_begin + incl);
-        f.ov_seg[slot] = (k * f.num_sms + fx.sm_index) * 2 + role;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void argus_fuse_emit(const ArgusFuseArgs& f, const ArgusFuseCtx& fx, u32 region, u64 t_begin,
-                                                u64 incl, u64 excl, u32 flags) {
-  if (fx.tab) argus_fuse_aggregate(fx, region, incl, excl, flags);
-  if (fx.pairbits) argus_fuse_overlap(f, fx, region, t_begin, incl);
 }
 
 #endif  // ARGUS_FUSE_CUH_

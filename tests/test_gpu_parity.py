@@ -348,7 +348,7 @@ def synth_mode(request):
 
 
 @pytest.mark.parametrize("idx,ctas,iters", [(0, 4, 626), (1, 7, 300), (2, 3, 3), (3, 3, 9), (4, 9, 400)])
-def test_synthesize_fused_matches_oracle(idx, ctas, iters, synth_mode):
+def test_synthesize_matches_oracle_in_every_mode(idx, ctas, iters, synth_mode):
     """One-call pipeline in each of its modes."""
     spec = tg.config(idx).scaled(ctas, iters)
     ev, offs = tg.generate_host(spec)
