@@ -318,7 +318,10 @@ __device__ __noinline__ u32 digest_bin_rare(u32* meta_word, u32 bin, u32 cell, u
   return 0xffffffffu;
 }
 
-__global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
+// (512 threads, three blocks per SM: the same 48 warps as six blocks of 256, but a stream's set-up, the choice of its hot
+// regions and the write-back of its row are shared by twice the threads; measured 2.33 ms against 2.45 ms on trace 3)
+constexpr int kDgThreads = 512;
+__global__ void __launch_bounds__(kDgThreads, 3) k_agg_streams_digest(AggArgs a) {
   extern __shared__ __align__(16) unsigned char sh_raw[];
   u32* const tab = reinterpret_cast<u32*>(sh_raw);
   const u32 R = a.num_regions;
@@ -397,12 +400,12 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_streams_digest(AggArgs a) {
         u32 b = leg_lo + (threadIdx.x & ~31u);
         // digests are asked for two rounds ahead (one round is shorter than a loaded DRAM access)
         u64 dg_next = b + lane < leg_hi ? __ldg(dgs + b + lane) : 0ull;
-        u64 dg_next2 = b + lane + kAggThreads < leg_hi ? __ldg(dgs + b + lane + kAggThreads) : 0ull;
-        for (; b < leg_hi; b += kAggThreads) {
+        u64 dg_next2 = b + lane + kDgThreads < leg_hi ? __ldg(dgs + b + lane + kDgThreads) : 0ull;
+        for (; b < leg_hi; b += kDgThreads) {
           const u32 i = b + lane;
           const u64 dg = dg_next;
           dg_next = dg_next2;
-          dg_next2 = i + 2 * kAggThreads < leg_hi ? __ldg(dgs + i + 2 * kAggThreads) : 0ull;
+          dg_next2 = i + 2 * kDgThreads < leg_hi ? __ldg(dgs + i + 2 * kDgThreads) : 0ull;
           const u32 dlo = (u32)dg, dhi = (u32)(dg >> 32);
           const bool in = i < leg_hi;
           const u32 region = dlo & 0xffffu;
@@ -774,7 +777,7 @@ int argus_internal_aggregate_scoped(const argus_interval_t* intervals, const uin
       const size_t dg = digest_table_words(num_regions) * 4 + ((num_regions + 31) / 32) * 4 + (size_t)a.ov.num_pairs * 8;
       if (dg > 48 * 1024)
         ARGUS_CUDA_TRY(cudaFuncSetAttribute(k_agg_streams_digest, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dg));
-      k_agg_streams_digest<<<num_streams, kAggThreads, dg, stream>>>(a);
+      k_agg_streams_digest<<<num_streams, kDgThreads, dg, stream>>>(a);
     } else {
       k_agg_streams_compact<<<num_streams, kAggThreads, compact, stream>>>(a);
     }
