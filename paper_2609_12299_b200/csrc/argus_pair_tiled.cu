@@ -12,10 +12,13 @@
 //     before it, and its parent as the latest set bit one level down before that begin; when there
 //     is none in the tile, the frame is in the stack carried from earlier tiles;
 //   - every finished interval adds its inclusive time to its parent frame's accumulator (shared
-//     atomics), which gives exclusive time without ordering the threads.
+//     atomics), which gives exclusive time without ordering the threads. The accumulators hold what
+//     the current window adds, in 32 bits (a frame carried from earlier tiles brings its 64-bit child
+//     time along separately); an interval or a sum that does not fit breaks the rules below.
 // This is exact when the tile is well nested (every end meets the frame on top with the same region
 // id). A tile is consumed in windows: the first position where a rule fails (region mismatch, negative
-// height, bad region id, depth overflow, level window exceeded) cuts the window there; the prefix is
+// height, bad region id, depth overflow, level window exceeded, 2^32 ticks of child time in one
+// window) cuts the window there; the prefix is
 // redone on its own (nothing of it had been committed), the offending marker goes through the
 // sequential stack machine on the carried stack, and a new window starts after it, so the result is
 // always the sequential definition's.
