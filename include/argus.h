@@ -502,8 +502,8 @@ int argus_pair_intervals_ring(const argus_event_t* ring /*device [S][slot_capaci
  * argus_overlap. Pairing also writes an 8-byte digest of every interval into the workspace
  * (4 bytes per event), and one pass over the digests both aggregates the intervals and
  * selects the overlap spans (up to 400 regions and 128 pairs; beyond that the three
- * operations run one after the other). Any of the four tables may be NULL; without tables
- * the pairing kernel selects the overlap spans itself. num_pairs may be 0. max_overlap_spans bounds
+ * operations run one after the other). Any of the four tables may be NULL; without any
+ * table the overlap stage reads the interval records. num_pairs may be 0. max_overlap_spans bounds
  * the spans selected for overlap over all pairs (an interval counts once per pair and role
  * its region appears in); more than that -> ARGUS_ERR_CAPACITY with the count in
  * status->intervals_required. One status block reports the first error of any stage.
