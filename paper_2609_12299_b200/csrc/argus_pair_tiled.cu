@@ -379,7 +379,9 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           const int first_bad = sm.badpos[bp];  // violations found so far; ends at or after it need no work
 #pragma unroll
           for (int i = 0; i < NI; ++i) {
-            const int rk = tid + i * NT;
+            // (the last, partly filled round goes to the upper half of the block: the lower half has the block's
+            // other duties, and a barrier waits for the slowest warp)
+            const int rk = (i == NI - 1 ? (tid + NT / 2) % NT : tid) + i * NT;
             refs[i] = 0;
             if (rk < win_ne) {
               const u32 d = sm.desc[rk];
@@ -427,7 +429,7 @@ __global__ void __launch_bounds__(NT, MINB) k_pair_tiled(ArgusPairArgs a) {
           const u64 pos0 = out_base + n_int;
 #pragma unroll
           for (int i = 0; i < NI; ++i) {
-            const int rk = tid + i * NT;
+            const int rk = (i == NI - 1 ? (tid + NT / 2) % NT : tid) + i * NT;
             if (rk < win_ne) {
               const u32 d = sm.desc[rk];
               const int partner = (int)(short)(refs[i] & 0xffffu), parent = (int)(short)(refs[i] >> 16);
